@@ -1,0 +1,397 @@
+"""Pins for the CPU oracle: closed forms, invariants, brute force, finite differences and the
+paper's printed parameter counts.  None of these call the CUDA path."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import btx_oracle as o
+
+RNG = np.random.default_rng
+
+
+def small_problem(seed, T=24, d=12, F=20, E=4, scale_r=1.0):
+    r = RNG(seed)
+    x = r.standard_normal((T, d))
+    wr = r.standard_normal((E, d)) * scale_r
+    w1 = r.standard_normal((E, F, d)) * 0.3
+    w3 = r.standard_normal((E, F, d)) * 0.3
+    w2 = r.standard_normal((E, d, F)) * 0.3
+    dy = r.standard_normal((T, d))
+    return x, wr, w1, w3, w2, dy
+
+
+# ---- scalar re-statement used for brute force on tiny inputs ---------------------------------
+
+def scalar_ffn(xv, W1, W3, W2):
+    F, d = len(W1), len(xv)
+    a = []
+    for f in range(F):
+        h1 = sum(W1[f][c] * xv[c] for c in range(d))
+        h3 = sum(W3[f][c] * xv[c] for c in range(d))
+        a.append(h1 / (1.0 + math.exp(-h1)) * h3)
+    return [sum(W2[c][f] * a[f] for f in range(F)) for c in range(d)]
+
+
+def scalar_moe_token(xv, Wr, W1, W3, W2, k):
+    """Enumerate every k-subset; keep the one with the largest logit sum (lowest indices on a
+    tie); mix the experts of that subset with a softmax restricted to it."""
+    E, d = len(Wr), len(xv)
+    z = [sum(Wr[i][c] * xv[c] for c in range(d)) for i in range(E)]
+    best = None
+    for S in itertools.combinations(range(E), k):          # lexicographic = lowest indices first
+        s = sum(z[i] for i in S)
+        if best is None or s > best[0]:
+            best = (s, S)
+    S = best[1]
+    den = sum(math.exp(z[i]) for i in S)
+    y = [0.0] * d
+    for i in S:
+        gi = math.exp(z[i]) / den
+        yi = scalar_ffn(xv, W1[i], W3[i], W2[i])
+        for c in range(d):
+            y[c] += gi * yi[c]
+    return set(S), y
+
+
+# ---- closed forms -----------------------------------------------------------------------------
+
+def test_worked_example_closed_form():
+    # one token, d = 1, two experts; logits (ln 3, 0) -> gates (3/4, 1/4)
+    x = np.array([[1.0]])
+    wr = np.array([[math.log(3.0)], [0.0]])
+    w1 = np.array([[[1.0]], [[0.0]]])
+    w3 = np.array([[[2.0]], [[5.0]]])
+    w2 = np.array([[[1.0]], [[7.0]]])
+    out = o.moe_forward(x, wr, w1, w3, w2, k=2, alpha=0.01)
+    np.testing.assert_allclose(out["gates"], [[0.75, 0.25]], rtol=1e-14)
+    assert out["topk_idx"].tolist() == [[0, 1]]
+    # expert 0: silu(1)*2 = 2/(1+e^-1); expert 1: silu(0) = 0
+    np.testing.assert_allclose(out["y"], [[0.75 * 2.0 / (1.0 + math.exp(-1.0))]], rtol=1e-14)
+    # u = (3/4, 1/4) = p  ->  L = 0.01 * 2 * (9/16 + 1/16)
+    np.testing.assert_allclose(out["lb_loss"], 0.01 * 2 * (10.0 / 16.0), rtol=1e-14)
+
+
+def test_operand_orientation_non_square():
+    # W1, W3 are [F, d] and W2 is [d, F]: with F != d a transposed operand cannot even multiply,
+    # and a swapped W1/W3 changes the value below.
+    x = np.array([[1.0, 2.0]])
+    w1 = np.array([[1.0, 0.0], [0.0, 1.0], [1.0, 1.0]])        # h1 = (1, 2, 3)
+    w3 = np.array([[1.0, 1.0], [0.0, 0.5], [2.0, 0.0]])        # h3 = (3, 1, 2)
+    w2 = np.array([[1.0, 0.0, 1.0], [0.0, 2.0, -1.0]])
+    silu = lambda v: v / (1.0 + math.exp(-v))
+    a = [silu(1.0) * 3.0, silu(2.0) * 1.0, silu(3.0) * 2.0]
+    want = [a[0] + a[2], 2.0 * a[1] - a[2]]
+    np.testing.assert_allclose(o.swiglu_ffn(x, w1, w3, w2), [want], rtol=1e-14)
+
+
+def test_lb_loss_closed_forms():
+    ln3 = math.log(3.0)
+    # two tokens preferring different experts, top-1 of 2 (gate of a lone selected logit is 1)
+    z = np.array([[ln3, 0.0], [0.0, ln3]])
+    loss, u, p = o.lb_loss_from_logits(z, 1, o.ROUTE_TOPK, 0.01)
+    np.testing.assert_allclose(u, [0.5, 0.5]); np.testing.assert_allclose(p, [0.5, 0.5])
+    np.testing.assert_allclose(loss, 0.01, rtol=1e-14)
+    # both prefer expert 0: u = (1, 0), p = (3/4, 1/4): L = alpha * 2 * 3/4
+    z = np.array([[ln3, 0.0], [ln3, 0.0]])
+    loss, u, p = o.lb_loss_from_logits(z, 1, o.ROUTE_TOPK, 0.01)
+    np.testing.assert_allclose(loss, 0.015, rtol=1e-14)
+    # Switch gate is the full-softmax probability: u = (3/4, 0): L = alpha * 2 * 9/16
+    loss, u, p = o.lb_loss_from_logits(z, 1, o.ROUTE_SWITCH, 0.01)
+    np.testing.assert_allclose(u, [0.75, 0.0])
+    np.testing.assert_allclose(loss, 0.01 * 2 * 9.0 / 16.0, rtol=1e-14)
+
+
+def test_zero_router_ties_and_uniform_loss():
+    x, wr, w1, w3, w2, _ = small_problem(1)
+    for k in (1, 2, 3):
+        out = o.moe_forward(x, wr * 0.0, w1, w3, w2, k=k, alpha=0.01)
+        assert (out["topk_idx"] == np.arange(k)[None, :]).all()          # ties -> lowest indices in order
+        np.testing.assert_allclose(out["gates"], 1.0 / k)
+        np.testing.assert_allclose(out["probs"], 0.25)
+        np.testing.assert_allclose(out["lb_loss"], 0.01, rtol=1e-14)    # alpha * E * sum u_i / E
+    # signed zeros tie as well
+    z = np.array([[0.0, -0.0, 0.0, -0.0], [-0.0, 0.0, -0.0, 0.0]])
+    assert o.top_k_select(z, 2).tolist() == [[0, 1], [0, 1]]
+
+
+def test_dominant_expert_loss_tends_to_alpha_E():
+    z = np.tile(np.array([[40.0, 0.0, 0.0, 0.0]]), (5, 1))
+    loss, u, p = o.lb_loss_from_logits(z, 1, o.ROUTE_TOPK, 0.01)
+    np.testing.assert_allclose(loss, 0.04, rtol=1e-12)
+
+
+# ---- invariants -------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("routing,k", [(o.ROUTE_TOPK, 1), (o.ROUTE_TOPK, 2), (o.ROUTE_TOPK, 3), (o.ROUTE_SOFT, 4)])
+def test_identical_experts_reduce_to_dense_ffn(routing, k):
+    x, wr, w1, w3, w2, _ = small_problem(2)
+    w1 = np.repeat(w1[:1], 4, axis=0); w3 = np.repeat(w3[:1], 4, axis=0); w2 = np.repeat(w2[:1], 4, axis=0)
+    out = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing)
+    np.testing.assert_allclose(out["y"], o.swiglu_ffn(x, w1[0], w3[0], w2[0]), rtol=1e-12, atol=1e-14)
+
+
+def test_single_expert_is_dense_ffn():
+    x, wr, w1, w3, w2, _ = small_problem(3, E=1)
+    out = o.moe_forward(x, wr, w1, w3, w2, k=1, alpha=0.01)
+    np.testing.assert_allclose(out["y"], o.swiglu_ffn(x, w1[0], w3[0], w2[0]), rtol=1e-13)
+    np.testing.assert_allclose(out["lb_loss"], 0.01, rtol=1e-14)
+
+
+def test_sparse_evaluation_equals_literal_sum_over_all_experts():
+    x, wr, w1, w3, w2, _ = small_problem(4)
+    for routing, k in [(o.ROUTE_TOPK, 2), (o.ROUTE_SWITCH, 1), (o.ROUTE_SOFT, 4)]:
+        a = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing)["y"]
+        b = o.moe_forward_all_experts(x, wr, w1, w3, w2, k=k, routing=routing)
+        np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-14)
+
+
+def test_expert_relabelling():
+    x, wr, w1, w3, w2, dy = small_problem(5)
+    sigma = np.array([2, 0, 3, 1])                       # new expert j is old expert sigma[j]
+    a = o.moe_forward(x, wr, w1, w3, w2, k=2)
+    b = o.moe_forward(x, wr[sigma], w1[sigma], w3[sigma], w2[sigma], k=2)
+    np.testing.assert_allclose(a["y"], b["y"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(a["lb_loss"], b["lb_loss"], rtol=1e-13)
+    assert (sigma[b["topk_idx"]] == a["topk_idx"]).all()
+    ga = o.moe_backward(x, wr, w1, w3, w2, dy, k=2)
+    gb = o.moe_backward(x, wr[sigma], w1[sigma], w3[sigma], w2[sigma], dy, k=2)
+    np.testing.assert_allclose(ga["dx"], gb["dx"], rtol=1e-11, atol=1e-13)
+    for name in ("dw1", "dw3", "dw2", "dw_router"):
+        np.testing.assert_allclose(ga[name][sigma], gb[name], rtol=1e-11, atol=1e-13)
+
+
+@pytest.mark.parametrize("E,k", [(2, 1), (4, 2), (5, 3), (6, 2)])
+def test_brute_force_subsets(E, k):
+    r = RNG(10 + E)
+    T, d, F = 6, 3, 4
+    x = r.standard_normal((T, d)); wr = r.standard_normal((E, d))
+    w1 = r.standard_normal((E, F, d)); w3 = r.standard_normal((E, F, d)); w2 = r.standard_normal((E, d, F))
+    out = o.moe_forward(x, wr, w1, w3, w2, k=k)
+    for t in range(T):
+        S, y = scalar_moe_token(x[t].tolist(), wr.tolist(), w1.tolist(), w3.tolist(), w2.tolist(), k)
+        assert set(out["topk_idx"][t].tolist()) == S
+        np.testing.assert_allclose(out["y"][t], y, rtol=1e-12, atol=1e-13)
+        # slots are ordered by decreasing logit
+        zs = out["logits"][t][out["topk_idx"][t]]
+        assert (np.diff(zs) <= 0).all()
+
+
+def test_gate_equivalences():
+    r = RNG(6)
+    z = r.standard_normal((50, 4)) * 2
+    idx = o.top_k_select(z, 2)
+    g = o.gate_values(z, idx, o.ROUTE_TOPK)
+    p = o.full_softmax(z)
+    psel = np.take_along_axis(p, idx.astype(np.int64), axis=1)
+    np.testing.assert_allclose(g, psel / psel.sum(1, keepdims=True), rtol=1e-13)   # renormalised full softmax
+    idx4 = o.top_k_select(z, 4)
+    g4 = o.gate_values(z, idx4, o.ROUTE_SOFT)
+    np.testing.assert_allclose(o.dense_gates(idx4, g4, 4), p, rtol=1e-13)          # soft = top-E
+    idx1 = o.top_k_select(z, 1)
+    gs = o.gate_values(z, idx1, o.ROUTE_SWITCH)
+    np.testing.assert_allclose(gs[:, 0], p.max(axis=1), rtol=1e-13)                 # Switch gate
+    assert (idx1[:, 0] == np.argmax(p, axis=1)).all()
+    # softmax is shift invariant
+    np.testing.assert_allclose(o.full_softmax(z + 3.0), p, rtol=1e-12)
+
+
+def test_forward_bookkeeping():
+    x, wr, w1, w3, w2, _ = small_problem(7, T=40)
+    out = o.moe_forward(x, wr, w1, w3, w2, k=2)
+    np.testing.assert_allclose(out["gates"].sum(1), 1.0, rtol=1e-14)
+    np.testing.assert_allclose(out["u"].sum(), 1.0, rtol=1e-13)
+    np.testing.assert_allclose(out["p"].sum(), 1.0, rtol=1e-13)
+    counts, offsets, perm, inv = out["counts"], out["offsets"], out["perm"], out["inv_perm"]
+    assert counts.sum() == 80 and offsets[0] == 0 and offsets[-1] == 80
+    assert (np.diff(offsets) == counts).all()
+    assert (perm[inv] == np.arange(80)).all() and (inv[perm] == np.arange(80)).all()
+    flat = out["topk_idx"].reshape(-1)
+    for e in range(4):
+        rows = perm[offsets[e]:offsets[e + 1]]
+        assert (flat[rows] == e).all()
+        assert (np.diff(rows // 2) > 0).all()             # strictly increasing token index
+    # a hand-checked dispatch
+    idx = np.array([[1, 0], [0, 2], [1, 2]], dtype=np.int32)
+    c, off, pm, iv = o.dispatch(idx, 3)
+    assert c.tolist() == [2, 2, 2] and off.tolist() == [0, 2, 4, 6]
+    assert pm.tolist() == [1, 2, 0, 4, 3, 5] and iv.tolist() == [2, 0, 1, 4, 3, 5]
+
+
+# ---- gradients --------------------------------------------------------------------------------
+
+def total_loss(x, wr, w1, w3, w2, G, k, routing, alpha, lam, bias=None):
+    out = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing, alpha=alpha, router_bias=bias)
+    return float(np.sum(out["y"] * G)) + lam * out["lb_loss"]
+
+
+@pytest.mark.parametrize("routing,k", [(o.ROUTE_TOPK, 2), (o.ROUTE_TOPK, 1), (o.ROUTE_SWITCH, 1), (o.ROUTE_SOFT, 4)])
+def test_gradients_against_finite_differences(routing, k):
+    x, wr, w1, w3, w2, G = small_problem(8, T=10, d=6, F=7, E=4, scale_r=1.5)
+    bias = np.array([0.1, -0.2, 0.0, 0.3])
+    alpha, lam = 0.7, 1.3                     # large alpha so the loss terms are visible
+    # the point must be far from a routing boundary
+    z = o.router_logits(x, wr, bias)
+    zs = np.sort(z, axis=1)
+    assert np.min(np.diff(zs, axis=1)) > 1e-3
+    g = o.moe_backward(x, wr, w1, w3, w2, G, k=k, routing=routing, alpha=alpha, lb_grad_scale=lam,
+                       router_bias=bias)
+    r = RNG(99)
+    h = 1e-6
+    params = dict(x=x, wr=wr, w1=w1, w3=w3, w2=w2, bias=bias)
+    names = dict(x="dx", wr="dw_router", w1="dw1", w3="dw3", w2="dw2", bias="dbias")
+    for pname, arr in params.items():
+        for _ in range(6):
+            pos = tuple(int(r.integers(0, s)) for s in arr.shape)
+            old = arr[pos]
+            arr[pos] = old + h
+            lp = total_loss(x, wr, w1, w3, w2, G, k, routing, alpha, lam, bias)
+            arr[pos] = old - h
+            lm = total_loss(x, wr, w1, w3, w2, G, k, routing, alpha, lam, bias)
+            arr[pos] = old
+            fd = (lp - lm) / (2 * h)
+            an = g[names[pname]][pos]
+            assert abs(fd - an) <= 2e-6 * max(1.0, abs(fd)), (pname, pos, fd, an)
+
+
+def test_lb_gradient_alone_and_stopgrad():
+    r = RNG(11)
+    z = r.standard_normal((12, 4)) * 1.5
+    alpha = 0.5
+    for routing, k in [(o.ROUTE_TOPK, 2), (o.ROUTE_SWITCH, 1), (o.ROUTE_SOFT, 4)]:
+        dz = o.lb_loss_grad(z, k, routing, alpha)
+        h = 1e-6
+        for _ in range(8):
+            pos = (int(r.integers(0, 12)), int(r.integers(0, 4)))
+            zp = z.copy(); zp[pos] += h
+            zm = z.copy(); zm[pos] -= h
+            fd = (o.lb_loss_from_logits(zp, k, routing, alpha)[0] - o.lb_loss_from_logits(zm, k, routing, alpha)[0]) / (2 * h)
+            assert abs(fd - dz[pos]) < 1e-8
+        np.testing.assert_allclose(dz.sum(axis=1), 0.0, atol=1e-15)
+    # with u held constant only the p-term remains: gradient of alpha E sum_i u_i p_i(z) at fixed u
+    k, routing = 2, o.ROUTE_TOPK
+    dz = o.lb_loss_grad(z, k, routing, alpha, lb_stopgrad_u=True)
+    _, u, _ = o.lb_loss_from_logits(z, k, routing, alpha)
+    f = lambda zz: alpha * 4 * float(np.sum(u * o.full_softmax(zz).mean(axis=0)))
+    pos = (3, 1)
+    zp = z.copy(); zp[pos] += 1e-6
+    zm = z.copy(); zm[pos] -= 1e-6
+    assert abs((f(zp) - f(zm)) / 2e-6 - dz[pos]) < 1e-8
+
+
+def test_router_gradient_rows_sum_to_zero():
+    x, wr, w1, w3, w2, dy = small_problem(12)
+    for routing, k in [(o.ROUTE_TOPK, 2), (o.ROUTE_SWITCH, 1), (o.ROUTE_SOFT, 4)]:
+        g = o.moe_backward(x, wr, w1, w3, w2, dy, k=k, routing=routing, alpha=0.3)
+        np.testing.assert_allclose(g["dlogits"].sum(axis=1), 0.0, atol=1e-13)
+        np.testing.assert_allclose(g["dw_router"].sum(axis=0), 0.0, atol=1e-12)
+        np.testing.assert_allclose(g["dbias"].sum(), 0.0, atol=1e-12)
+
+
+def test_linearity_in_w2_and_gate_gradient_identity():
+    x, wr, w1, w3, w2, dy = small_problem(13)
+    a = o.moe_forward(x, wr, w1, w3, w2, k=2)
+    b = o.moe_forward(x, wr, w1, w3, 2.5 * w2, k=2)
+    np.testing.assert_allclose(b["y"], 2.5 * a["y"], rtol=1e-12, atol=1e-14)
+    ga = o.moe_backward(x, wr, w1, w3, w2, dy, k=2, alpha=0.0)
+    gb = o.moe_backward(x, wr, w1, w3, 2.5 * w2, dy, k=2, alpha=0.0)
+    np.testing.assert_allclose(gb["dw1"], 2.5 * ga["dw1"], rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(gb["dw2"], ga["dw2"], rtol=1e-11, atol=1e-13)
+    # d/d gate = <dY_t, FF_i(x_t)> = <W2_i^T dY_t, a_{t,i}>
+    idx = a["topk_idx"]
+    for t in (0, 5, 17):
+        for s in range(2):
+            e = idx[t, s]
+            _, _, _, act = o.swiglu_ffn(x[t:t + 1], w1[e], w3[e], w2[e], return_hidden=True)
+            np.testing.assert_allclose(ga["dgate"][t, s], float((dy[t] @ w2[e]) @ act[0]), rtol=1e-11)
+
+
+def test_slice_modes_agree_with_full_backward():
+    x, wr, w1, w3, w2, dy = small_problem(14, T=30)
+    for routing, k in [(o.ROUTE_TOPK, 2), (o.ROUTE_SWITCH, 1)]:
+        full = o.moe_backward(x, wr, w1, w3, w2, dy, k=k, routing=routing, alpha=0.2, lb_grad_scale=0.9)
+        fwd = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing, alpha=0.2)
+        tok = np.array([3, 4, 11, 29])
+        sl = o.moe_backward_token_slice(x, wr, w1, w3, w2, dy, fwd["topk_idx"], fwd["gates"], fwd["probs"],
+                                        fwd["u"], fwd["p"], tok, routing=routing, alpha=0.2, lb_grad_scale=0.9)
+        np.testing.assert_allclose(sl["dx"], full["dx"][tok], rtol=1e-11, atol=1e-13)
+        np.testing.assert_allclose(sl["dlogits"], full["dlogits"][tok], rtol=1e-11, atol=1e-14)
+        ys = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing, tokens=tok)["y"]
+        np.testing.assert_allclose(ys, fwd["y"][tok], rtol=1e-12, atol=1e-14)
+        J = np.array([0, 7, 19])
+        for e in range(4):
+            d1, d3, d2 = o.expert_wgrad_hidden_slice(x, w1, w3, w2, dy, fwd["topk_idx"], fwd["gates"], e, J)
+            np.testing.assert_allclose(d1, full["dw1"][e][J], rtol=1e-11, atol=1e-13)
+            np.testing.assert_allclose(d3, full["dw3"][e][J], rtol=1e-11, atol=1e-13)
+            np.testing.assert_allclose(d2, full["dw2"][e][:, J], rtol=1e-11, atol=1e-13)
+
+
+def test_logits_override_decides_routing():
+    x, wr, w1, w3, w2, _ = small_problem(15)
+    z32 = o.router_logits(x, wr).astype(np.float32)
+    z32[0, :] = [1.0, 1.0, 1.0, 0.0]                      # a three-way tie decided by index
+    out = o.moe_forward(x, wr, w1, w3, w2, k=2, logits=z32)
+    assert out["topk_idx"][0].tolist() == [0, 1]
+    np.testing.assert_allclose(out["gates"][0], [0.5, 0.5])
+
+
+# ---- merge ------------------------------------------------------------------------------------
+
+def test_merge_pins():
+    r = RNG(16)
+    seed_model = {"layers.0.attn.wq": r.standard_normal((8, 8)).astype(np.float32),
+                  "layers.0.ffn.w1": r.standard_normal((5, 8)).astype(np.float32),
+                  "norm": r.standard_normal(8).astype(np.float32)}
+    for n in (2, 4):                                      # power of two: exact
+        m = o.merge_models([seed_model] * n, "f32")
+        assert (m["layers.0.attn.wq"] == seed_model["layers.0.attn.wq"]).all()
+        assert (m["norm"] == seed_model["norm"]).all()
+        assert m["layers.0.ffn.w1"].shape == (n, 5, 8)
+        for e in range(n):
+            assert (m["layers.0.ffn.w1"][e] == seed_model["layers.0.ffn.w1"]).all()
+    m3 = o.merge_models([seed_model] * 3, "f32")          # (3 a)/3 may differ by an ulp
+    np.testing.assert_allclose(m3["norm"], seed_model["norm"], rtol=2e-7)
+    a = {"norm": np.array([1.0, 2.0, -4.0])}
+    b = {"norm": np.array([3.0, 2.5, 4.0])}
+    assert o.merge_models([a, b], "f32")["norm"].tolist() == [2.0, 2.25, 0.0]
+    # experts keep their order
+    ma = {"l.ffn.w2": np.full((2, 2), 1.0)}; mb = {"l.ffn.w2": np.full((2, 2), 2.0)}
+    st = o.merge_models([ma, mb], "f32")["l.ffn.w2"]
+    assert (st[0] == 1.0).all() and (st[1] == 2.0).all()
+
+
+def test_bf16_rounding_against_torch_and_ties():
+    # ties to even at 8 significant bits
+    v = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -9, -(1.0 + 2.0 ** -8), 0.0, 3.0e-40])
+    got = o.round_to_bf16(v)
+    assert got[:5].tolist() == [1.0, 1.0 + 2.0 ** -6, 1.0, -1.0, 0.0]
+    # fp32 inputs: torch's own float32 -> bfloat16 conversion is an independent implementation
+    r = RNG(17)
+    f = (r.standard_normal(20000) * np.exp(r.uniform(-20, 20, 20000))).astype(np.float32)
+    want = torch.from_numpy(f).to(torch.bfloat16).to(torch.float64).numpy()
+    assert (o.round_to_bf16(f.astype(np.float64)) == want).all()
+    # mean of bf16 values rounded once
+    a = torch.from_numpy(f[:1000]).to(torch.bfloat16)
+    b = torch.from_numpy(f[1000:2000]).to(torch.bfloat16)
+    m = o.merge_average([a.to(torch.float64).numpy(), b.to(torch.float64).numpy()], "bf16")
+    want = ((a.to(torch.float32) + b.to(torch.float32)) / 2).to(torch.bfloat16).to(torch.float64).numpy()
+    # a + b of two bf16 numbers is exact in fp32 unless their exponents differ by more than 16
+    close = np.abs(np.log2(np.abs(a.float().numpy()) / np.abs(b.float().numpy()))) < 14
+    assert (m[close] == want[close]).all()
+
+
+def test_table4_active_parameter_counts():
+    path = os.path.join(os.path.dirname(__file__), "golden", "table4_active_params.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 3
+    for name, k, printed in rows:
+        n = o.active_parameters(32, 4096, 11008, 32000, 4, int(k))
+        assert round(n / 1e9, 1) == float(printed), (name, n)
+    # the same table fixes the split used by the merge workload
+    shapes = o.llama_like_param_shapes(32, 4096, 11008, 32000)
+    ffn = sum(int(np.prod(s)) for n, s in shapes if ".ffn." in n)
+    other = sum(int(np.prod(s)) for n, s in shapes if ".ffn." not in n)
+    assert ffn == 4_328_521_728 and other == 2_409_893_888
