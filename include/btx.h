@@ -1,0 +1,142 @@
+/*
+ * btx.h -- C ABI of the B200 (sm_100a) MoE feed-forward hot path of Branch-Train-MiX
+ * (arXiv 2403.07816).
+ *
+ * General conventions
+ *   - Every tensor argument is a DEVICE pointer to caller-owned, row-major, contiguous memory,
+ *     16-byte aligned, unless its description says "host".  The library never allocates or
+ *     frees device memory and keeps no pointer after a call returns.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and return without
+ *     synchronising; arguments are validated on the host before anything is launched.
+ *   - Element type of x, weights, y, dy, dx is given by btx_moe_desc.dtype (BTX_F32: float,
+ *     BTX_BF16: bfloat16 with fp32 accumulation).  Logits, gates, probabilities, the loss and all
+ *     weight gradients are fp32.  Index outputs are int32.
+ *   - Errors: a btx_status is returned; nothing is launched when it is not BTX_OK.  Device-side
+ *     bounded waits that expire are recorded in the workspace and read with btx_device_status.
+ *
+ * Notation: T tokens, d = d_model, F = d_ff, E experts, k selected experts per token
+ * (k = E under BTX_ROUTE_SOFT), R = T*k assignments.
+ */
+#ifndef BTX_H_
+#define BTX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BTX_OK = 0,
+  BTX_ERR_INVALID_ARG = 1,   /* null required pointer, bad size, misaligned pointer          */
+  BTX_ERR_UNSUPPORTED = 2,   /* valid request outside what the kernels cover                 */
+  BTX_ERR_WORKSPACE = 3,     /* workspace / saved buffer smaller than btx_moe_sizes reports  */
+  BTX_ERR_ARCH = 4,          /* current device is not compute capability 10.x                */
+  BTX_ERR_CUDA = 5,          /* a CUDA runtime or driver call failed                         */
+  BTX_ERR_TIMEOUT = 6        /* a device-side bounded wait expired (see btx_device_status)   */
+} btx_status;
+
+typedef enum { BTX_F32 = 0, BTX_BF16 = 1 } btx_dtype;
+
+/* Routing function g (Section 3.2 and Section 3.3 "Routing method").
+ *   TOPK   g = softmax over the k largest logits, zero elsewhere (the paper's default, k = 2).
+ *   SWITCH k = 1; the gate is the full-softmax probability of the arg-max expert.
+ *   SOFT   g = softmax over all E experts (every expert active); desc.k is ignored.
+ * Ties between equal logits go to the lower expert index; slot 0 holds the largest logit. */
+typedef enum { BTX_ROUTE_TOPK = 0, BTX_ROUTE_SWITCH = 1, BTX_ROUTE_SOFT = 2 } btx_routing;
+
+typedef struct {
+  int32_t T, d_model, d_ff, E, k;
+  int32_t dtype;              /* btx_dtype                                                     */
+  int32_t routing;            /* btx_routing                                                   */
+  float   lb_alpha;           /* alpha of the load-balancing loss (Section 3.3; 0.01 in 4.1.1) */
+  int32_t lb_stopgrad_u;      /* 0: differentiate L_LB through u and p as printed; 1: u const  */
+  int32_t save_for_backward;  /* forward fills `saved` so that btx_moe_backward can run        */
+} btx_moe_desc;
+
+/* Optional routing outputs of btx_moe_forward; any member may be NULL.  All device pointers.
+ *   logits[T,E], probs[T,E] (full softmax), topk_idx[T,k], gates[T,k]; counts[E] tokens per
+ *   expert, offsets[E+1] exclusive scan; perm[R]: sorted row -> t*k+slot with rows ordered by
+ *   (expert ascending, token ascending); inv_perm[R] its inverse; u[E], p[E], lb_loss[1] of
+ *   Section 3.3. */
+typedef struct {
+  float*   logits;
+  int32_t* topk_idx;
+  float*   gates;
+  float*   probs;
+  int32_t* counts;
+  int32_t* offsets;
+  int32_t* perm;
+  int32_t* inv_perm;
+  float*   u;
+  float*   p;
+  float*   lb_loss;
+} btx_routing_out;
+
+/* Bytes of `workspace` (scratch, contents undefined afterwards; one size serves forward and
+ * backward) and of `saved` (forward -> backward state: routing, the expert-sorted copy of x and
+ * the two SwiGLU pre-activations).  Host pointers out.  Sizes are upper bounds that do not depend
+ * on the routing outcome. */
+btx_status btx_moe_sizes(const btx_moe_desc* desc, size_t* workspace_bytes, size_t* saved_bytes);
+
+/* FF_MoE(x) = sum_i g_i(W_l x) FF_i(x)  (Section 3.2), FF_i(x) = W2_i (silu(W1_i x) * W3_i x),
+ * evaluated only for the selected experts, plus the load-balancing loss of Section 3.3.
+ *   x[T,d]; w_router[E,d] (W_l); router_bias[E] fp32 or NULL (the paper has no bias);
+ *   w1,w3[E,F,d]; w2[E,d,F]; y[T,d] out.  `routing` may be NULL.  `saved` may be NULL when
+ *   desc.save_for_backward == 0.  d and F must be multiples of 8 in BF16 mode, of 4 in F32. */
+btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, const void* w_router,
+                           const float* router_bias, const void* w1, const void* w3, const void* w2,
+                           void* y, const btx_routing_out* routing, void* saved,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* Backward of btx_moe_forward for the scalar <y, dy> + lb_grad_scale * L_LB (MoE finetuning,
+ * Sections 1 and 3.2; the loss is added to the training loss with weight 1, Section 3.3).
+ * `saved` is the buffer the forward call filled with the same desc and inputs.
+ * Outputs: dx[T,d] (dtype); dw_router[E,d], dbias[E] (may be NULL), dw1,dw3[E,F,d], dw2[E,d,F],
+ * all fp32.  accumulate = 0 overwrites the weight gradients, 1 adds to them. */
+btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void* w_router,
+                            const float* router_bias, const void* w1, const void* w3, const void* w2,
+                            const void* dy, float lb_grad_scale, const void* saved,
+                            void* dx, float* dw_router, float* dbias,
+                            float* dw1, float* dw3, float* dw2, int32_t accumulate,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/* L_LB = alpha * E * sum_i u_i p_i with u_i the batch mean of the gate of expert i and p_i the
+ * batch mean of SoftMax_i (Section 3.3), from given fp32 logits[T,E] (bias, if any, already
+ * added).  Outputs loss[1], u[E], p[E]; dlogits[T,E] (d loss / d logits) unless NULL.
+ * Uses desc.T, E, k, routing, lb_alpha, lb_stopgrad_u.  Workspace: btx_lb_loss_workspace_size. */
+btx_status btx_lb_loss_workspace_size(const btx_moe_desc* desc, size_t* workspace_bytes);
+btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits, float* loss, float* u, float* p,
+                       float* dlogits, void* workspace, size_t workspace_bytes, void* stream);
+
+/* MiX merge (Section 3.2): the feed-forward matrices of the N expert LLMs become the experts of
+ * one MoE layer (kind FFN: dst[e*numel .. ] = src[e], bit for bit); every other parameter is the
+ * uniform mean over the N models (kind AVERAGE: fp32 sum in model order, divided by N, rounded
+ * once to dtype).  `items` is a HOST array; each item's `src` is a HOST array of N device
+ * pointers.  Sources and destinations must not overlap.  numel*sizeof(element) need not be a
+ * multiple of 16 for AVERAGE items; the pointers must be 16-byte aligned. */
+typedef enum { BTX_PARAM_AVERAGE = 0, BTX_PARAM_FFN = 1 } btx_param_kind;
+typedef struct {
+  int32_t kind;               /* btx_param_kind */
+  int32_t layer;              /* informational  */
+  uint64_t numel;             /* elements per source tensor */
+  const void* const* src;     /* host array of n_models device pointers */
+  void* dst;                  /* device; numel elements (AVERAGE) or n_models*numel (FFN) */
+} btx_merge_item;
+
+btx_status btx_merge_workspace_size(int32_t n_models, uint64_t n_items, size_t* workspace_bytes);
+btx_status btx_merge(int32_t n_models, int32_t dtype, const btx_merge_item* items, uint64_t n_items,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream` and reads the status word that kernels of earlier calls left in
+ * `workspace`: *device_status (host) is BTX_OK or BTX_ERR_TIMEOUT. */
+btx_status btx_device_status(const void* workspace, void* stream, int32_t* device_status);
+
+const char* btx_status_string(btx_status s);
+int32_t btx_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BTX_H_ */

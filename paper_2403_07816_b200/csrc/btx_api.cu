@@ -1,0 +1,265 @@
+// C ABI entry points: argument validation, the buffer plan, and the launch sequences of the
+// forward and backward passes (see include/btx.h for the contract of every call).
+#include <cstdio>
+#include <cstring>
+
+#include "btx_common.cuh"
+
+namespace btx {
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
+  if (!desc || !pl) return BTX_ERR_INVALID_ARG;
+  if (desc->T < 1 || desc->E < 1) return BTX_ERR_INVALID_ARG;
+  if (!routing_only && (desc->d_model < 1 || desc->d_ff < 1)) return BTX_ERR_INVALID_ARG;
+  if (desc->dtype != BTX_F32 && desc->dtype != BTX_BF16) return BTX_ERR_INVALID_ARG;
+  if (desc->routing < BTX_ROUTE_TOPK || desc->routing > BTX_ROUTE_SOFT) return BTX_ERR_INVALID_ARG;
+  int k = desc->routing == BTX_ROUTE_SOFT ? desc->E : desc->k;
+  if (k < 1 || k > desc->E) return BTX_ERR_INVALID_ARG;
+  if (desc->routing == BTX_ROUTE_SWITCH && k != 1) return BTX_ERR_INVALID_ARG;
+  if (desc->E > kMaxExperts) return BTX_ERR_UNSUPPORTED;
+  const int gran = desc->dtype == BTX_BF16 ? 8 : 4;         // rows must be whole 16-byte vectors
+  if (!routing_only && (desc->d_model % gran || desc->d_ff % gran)) return BTX_ERR_UNSUPPORTED;
+  if ((long long)desc->T * k > (1ll << 28)) return BTX_ERR_UNSUPPORTED;
+
+  Plan& p = *pl;
+  memset(&p, 0, sizeof(p));
+  p.T = desc->T; p.E = desc->E; p.k = k; p.R = p.T * k;
+  p.d = routing_only ? 0 : desc->d_model;
+  p.F = routing_only ? 0 : desc->d_ff;
+  p.esize = desc->dtype == BTX_BF16 ? 2 : 4;
+  p.r_pad_max = (int)align_up((size_t)p.R + (size_t)p.E * (kRowTile - 1), kRowTile);
+  p.mt_max = p.r_pad_max / kRowTile;
+  p.nt_dact = desc->dtype == BTX_BF16 ? (p.F + 255) / 256 : (p.F + 63) / 64;
+  p.route_blocks = (p.T + 7) / 8;
+  if (p.route_blocks > 148 * 8) p.route_blocks = 148 * 8;
+  p.perm_blocks = (p.R + 1023) / 1024;
+  p.wr_chunks = (p.T + 127) / 128;
+
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  const size_t rp = (size_t)p.r_pad_max;
+  p.s_topk = take((size_t)p.R * 4);       p.s_gates = take((size_t)p.R * 4);
+  p.s_probs = take((size_t)p.T * p.E * 4); p.s_logits = take((size_t)p.T * p.E * 4);
+  p.s_u = take(p.E * 4);  p.s_p = take(p.E * 4);  p.s_loss = take(4);
+  p.s_counts = take(p.E * 4);  p.s_offsets = take((p.E + 1) * 4);  p.s_pad_offsets = take((p.E + 1) * 4);
+  p.s_tile_expert = take((size_t)p.mt_max * 4);
+  p.s_rowmap = take(rp * 4);  p.s_flat2row = take((size_t)p.R * 4);
+  p.s_perm = take((size_t)p.R * 4);  p.s_inv_perm = take((size_t)p.R * 4);
+  p.s_xs = take(rp * p.d * p.esize);
+  p.s_h1 = take(rp * p.F * p.esize);
+  p.s_h3 = take(rp * p.F * p.esize);
+  p.saved_bytes = o;
+
+  o = 0;
+  p.w_status = take(kStatusWords * 4);
+  p.w_route_part = take((size_t)p.route_blocks * 2 * p.E * 4);
+  p.w_perm_counts = take((size_t)p.perm_blocks * p.E * 4);
+  p.w_perm_base = take((size_t)p.perm_blocks * p.E * 4);
+  p.w_dz = take((size_t)p.T * p.E * 4);
+  p.w_dwr_part = take((size_t)p.wr_chunks * p.E * (p.d + 1) * 4);
+  p.w_dg_part = take((size_t)p.nt_dact * rp * 4);
+  // forward and backward scratch overlap: act | yp  vs  dys | dh1 | dh3 | ga | dxp
+  size_t base = o;
+  p.w_act = take(rp * p.F * p.esize);
+  p.w_yp = take((size_t)p.R * p.d * 4);
+  size_t fwd_end = o;
+  o = base;
+  p.w_dys = take(rp * p.d * p.esize);
+  p.w_dh1 = take(rp * p.F * p.esize);
+  p.w_dh3 = take(rp * p.F * p.esize);
+  p.w_ga = take(rp * p.F * p.esize);
+  p.w_dxp = take((size_t)p.R * p.d * 4);
+  if (o < fwd_end) o = fwd_end;
+  // a forward that keeps nothing for backward parks its "saved" state here
+  p.w_saved_fallback = take(p.saved_bytes);
+  p.workspace_bytes = o;
+  return BTX_OK;
+}
+
+static void resolve(const Plan& p, char* saved, char* ws, Buffers* b) {
+  b->topk = (int32_t*)(saved + p.s_topk);   b->gates = (float*)(saved + p.s_gates);
+  b->probs = (float*)(saved + p.s_probs);   b->logits = (float*)(saved + p.s_logits);
+  b->u = (float*)(saved + p.s_u);  b->p = (float*)(saved + p.s_p);  b->loss = (float*)(saved + p.s_loss);
+  b->counts = (int32_t*)(saved + p.s_counts);  b->offsets = (int32_t*)(saved + p.s_offsets);
+  b->pad_offsets = (int32_t*)(saved + p.s_pad_offsets);  b->tile_expert = (int32_t*)(saved + p.s_tile_expert);
+  b->rowmap = (int32_t*)(saved + p.s_rowmap);  b->flat2row = (int32_t*)(saved + p.s_flat2row);
+  b->perm = (int32_t*)(saved + p.s_perm);  b->inv_perm = (int32_t*)(saved + p.s_inv_perm);
+  b->xs = saved + p.s_xs;  b->h1 = saved + p.s_h1;  b->h3 = saved + p.s_h3;
+  b->status = (int32_t*)(ws + p.w_status);  b->route_part = (float*)(ws + p.w_route_part);
+  b->perm_counts = (int32_t*)(ws + p.w_perm_counts);  b->perm_base = (int32_t*)(ws + p.w_perm_base);
+  b->act = ws + p.w_act;  b->yp = (float*)(ws + p.w_yp);
+  b->dys = ws + p.w_dys;  b->dh1 = ws + p.w_dh1;  b->dh3 = ws + p.w_dh3;  b->ga = ws + p.w_ga;
+  b->dxp = (float*)(ws + p.w_dxp);
+  b->dg_part = (float*)(ws + p.w_dg_part);  b->dz = (float*)(ws + p.w_dz);  b->dwr_part = (float*)(ws + p.w_dwr_part);
+}
+
+static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+
+static btx_status check_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return BTX_ERR_CUDA;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return BTX_ERR_CUDA;
+  return major == 10 ? BTX_OK : BTX_ERR_ARCH;
+}
+
+#define BTX_CUDA_OK(expr) do { if ((expr) != cudaSuccess) return BTX_ERR_CUDA; } while (0)
+
+}  // namespace btx
+
+using namespace btx;
+
+extern "C" btx_status btx_moe_sizes(const btx_moe_desc* desc, size_t* workspace_bytes, size_t* saved_bytes) {
+  Plan p;
+  btx_status s = make_plan(desc, &p, false);
+  if (s != BTX_OK) return s;
+  if (workspace_bytes) *workspace_bytes = p.workspace_bytes;
+  if (saved_bytes) *saved_bytes = p.saved_bytes;
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, const void* w_router,
+                                      const float* router_bias, const void* w1, const void* w3, const void* w2,
+                                      void* y, const btx_routing_out* routing, void* saved, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+  Plan pl;
+  btx_status s = make_plan(desc, &pl, false);
+  if (s != BTX_OK) return s;
+  if (!x || !w_router || !w1 || !w3 || !w2 || !y || !workspace) return BTX_ERR_INVALID_ARG;
+  if (desc->save_for_backward && !saved) return BTX_ERR_INVALID_ARG;
+  if (misaligned(x) || misaligned(w_router) || misaligned(w1) || misaligned(w3) || misaligned(w2) || misaligned(y) ||
+      misaligned(workspace) || misaligned(saved))
+    return BTX_ERR_INVALID_ARG;
+  if (workspace_bytes < pl.workspace_bytes) return BTX_ERR_WORKSPACE;
+  if ((s = check_device()) != BTX_OK) return s;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = (char*)workspace;
+  char* sv = desc->save_for_backward ? (char*)saved : ws + pl.w_saved_fallback;
+  Buffers b;
+  resolve(pl, sv, ws, &b);
+
+  BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
+  BTX_CUDA_OK(launch_router(pl, desc->dtype, desc->routing, desc->lb_alpha, x, w_router, router_bias, nullptr, b, st));
+  BTX_CUDA_OK(launch_permute(pl, b, st));
+  BTX_CUDA_OK(launch_gather_rows(pl, x, b.xs, b, st));
+  if (desc->dtype == BTX_F32) {
+    BTX_CUDA_OK(launch_expert_forward_f32(pl, w1, w3, w2, b, desc->save_for_backward, st));
+  } else {
+    if ((s = launch_expert_forward_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
+  }
+  BTX_CUDA_OK(launch_combine(pl, desc->dtype, b.yp, y, st));
+
+  if (routing) {
+    auto out = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
+      return dst ? cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) : cudaSuccess;
+    };
+    BTX_CUDA_OK(out(routing->logits, b.logits, (size_t)pl.T * pl.E * 4));
+    BTX_CUDA_OK(out(routing->probs, b.probs, (size_t)pl.T * pl.E * 4));
+    BTX_CUDA_OK(out(routing->topk_idx, b.topk, (size_t)pl.R * 4));
+    BTX_CUDA_OK(out(routing->gates, b.gates, (size_t)pl.R * 4));
+    BTX_CUDA_OK(out(routing->counts, b.counts, pl.E * 4));
+    BTX_CUDA_OK(out(routing->offsets, b.offsets, (pl.E + 1) * 4));
+    BTX_CUDA_OK(out(routing->perm, b.perm, (size_t)pl.R * 4));
+    BTX_CUDA_OK(out(routing->inv_perm, b.inv_perm, (size_t)pl.R * 4));
+    BTX_CUDA_OK(out(routing->u, b.u, pl.E * 4));
+    BTX_CUDA_OK(out(routing->p, b.p, pl.E * 4));
+    BTX_CUDA_OK(out(routing->lb_loss, b.loss, 4));
+  }
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void* w_router,
+                                       const float* router_bias, const void* w1, const void* w3, const void* w2,
+                                       const void* dy, float lb_grad_scale, const void* saved, void* dx,
+                                       float* dw_router, float* dbias, float* dw1, float* dw3, float* dw2,
+                                       int32_t accumulate, void* workspace, size_t workspace_bytes, void* stream) {
+  (void)router_bias;   // the bias only shifts the logits; its gradient needs dz alone
+  Plan pl;
+  btx_status s = make_plan(desc, &pl, false);
+  if (s != BTX_OK) return s;
+  if (!x || !w_router || !w1 || !w3 || !w2 || !dy || !saved || !dx || !dw_router || !dw1 || !dw3 || !dw2 ||
+      !workspace)
+    return BTX_ERR_INVALID_ARG;
+  if (misaligned(x) || misaligned(w_router) || misaligned(w1) || misaligned(w3) || misaligned(w2) ||
+      misaligned(dy) || misaligned(saved) || misaligned(dx) || misaligned(dw_router) || misaligned(dw1) ||
+      misaligned(dw3) || misaligned(dw2) || misaligned(workspace))
+    return BTX_ERR_INVALID_ARG;
+  if (workspace_bytes < pl.workspace_bytes) return BTX_ERR_WORKSPACE;
+  if ((s = check_device()) != BTX_OK) return s;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  Buffers b;
+  resolve(pl, (char*)saved, (char*)workspace, &b);
+  BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
+  BTX_CUDA_OK(launch_gather_rows(pl, dy, b.dys, b, st));
+  if (desc->dtype == BTX_F32) {
+    BTX_CUDA_OK(launch_expert_backward_f32(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, st));
+  } else {
+    if ((s = launch_expert_backward_bf16(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, st)) != BTX_OK) return s;
+  }
+  BTX_CUDA_OK(launch_router_backward(pl, desc->dtype, desc->routing, desc->lb_alpha, lb_grad_scale,
+                                     desc->lb_stopgrad_u, 1, x, w_router, b, dx, dw_router, dbias, nullptr,
+                                     accumulate, st));
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_lb_loss_workspace_size(const btx_moe_desc* desc, size_t* workspace_bytes) {
+  Plan p;
+  btx_status s = make_plan(desc, &p, true);
+  if (s != BTX_OK) return s;
+  if (!workspace_bytes) return BTX_ERR_INVALID_ARG;
+  *workspace_bytes = p.workspace_bytes;
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits, float* loss, float* u, float* p,
+                                  float* dlogits, void* workspace, size_t workspace_bytes, void* stream) {
+  Plan pl;
+  btx_status s = make_plan(desc, &pl, true);
+  if (s != BTX_OK) return s;
+  if (!logits || !loss || !u || !p || !workspace) return BTX_ERR_INVALID_ARG;
+  if (misaligned(workspace)) return BTX_ERR_INVALID_ARG;
+  if (workspace_bytes < pl.workspace_bytes) return BTX_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = (char*)workspace;
+  Buffers b;
+  resolve(pl, ws + pl.w_saved_fallback, ws, &b);
+  BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
+  BTX_CUDA_OK(launch_router(pl, BTX_F32, desc->routing, desc->lb_alpha, nullptr, nullptr, nullptr, logits, b, st));
+  BTX_CUDA_OK(cudaMemcpyAsync(loss, b.loss, 4, cudaMemcpyDeviceToDevice, st));
+  BTX_CUDA_OK(cudaMemcpyAsync(u, b.u, pl.E * 4, cudaMemcpyDeviceToDevice, st));
+  BTX_CUDA_OK(cudaMemcpyAsync(p, b.p, pl.E * 4, cudaMemcpyDeviceToDevice, st));
+  if (dlogits) {
+    BTX_CUDA_OK(launch_router_backward(pl, BTX_F32, desc->routing, desc->lb_alpha, 1.0f, desc->lb_stopgrad_u, 0,
+                                       nullptr, nullptr, b, nullptr, nullptr, nullptr, dlogits, 0, st));
+  }
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_device_status(const void* workspace, void* stream, int32_t* device_status) {
+  if (!workspace || !device_status) return BTX_ERR_INVALID_ARG;
+  int32_t word = 0;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(&word, workspace, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return BTX_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return BTX_ERR_CUDA;
+  *device_status = word == 0 ? BTX_OK : BTX_ERR_TIMEOUT;
+  return BTX_OK;
+}
+
+extern "C" const char* btx_status_string(btx_status s) {
+  switch (s) {
+    case BTX_OK: return "ok";
+    case BTX_ERR_INVALID_ARG: return "invalid argument";
+    case BTX_ERR_UNSUPPORTED: return "unsupported configuration";
+    case BTX_ERR_WORKSPACE: return "workspace or saved buffer too small";
+    case BTX_ERR_ARCH: return "device is not compute capability 10.x";
+    case BTX_ERR_CUDA: return "CUDA call failed";
+    case BTX_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+extern "C" int32_t btx_version(void) { return 100; }

@@ -1,0 +1,100 @@
+// Shared declarations of the btx CUDA library: the internal buffer plan, kernel launchers
+// and small device helpers.  Nothing here is part of the public ABI (see include/btx.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "btx.h"
+
+namespace btx {
+
+constexpr int kRowTile = 128;        // expert segments of the sorted buffers are padded to this many rows
+constexpr int kMaxExperts = 32;
+constexpr int kStatusWords = 64;     // first 256 bytes of every workspace: device status block
+
+// ---------------------------------------------------------------------------------------------
+// Buffer plan.  All offsets are bytes from the start of `saved` / `workspace`.
+// ---------------------------------------------------------------------------------------------
+struct Plan {
+  int T, d, F, E, k, R;              // k = effective number of selected experts
+  int esize;                         // bytes per element of dtype
+  int r_pad_max;                     // upper bound of the padded sorted row count (multiple of 128)
+  int mt_max;                        // r_pad_max / 128
+  int nt_dact;                       // column tiles of the dgrad-2 GEMM (row-dot partials)
+  int route_blocks;                  // blocks of the router kernel (partial sums for u, p)
+  int perm_blocks;                   // blocks of the permutation kernels
+  int wr_chunks;                     // token chunks of the router-weight gradient
+  // saved
+  size_t s_topk, s_gates, s_probs, s_logits, s_u, s_p, s_loss, s_counts, s_offsets, s_pad_offsets,
+      s_tile_expert, s_rowmap, s_flat2row, s_perm, s_inv_perm, s_xs, s_h1, s_h3, saved_bytes;
+  // workspace
+  size_t w_status, w_route_part, w_perm_counts, w_perm_base, w_act, w_yp, w_dys, w_dh1, w_dh3, w_ga,
+      w_dxp, w_dg_part, w_dz, w_dwr_part, w_saved_fallback, workspace_bytes;
+};
+
+// routing_only: plan for btx_lb_loss (no expert buffers)
+btx_status make_plan(const btx_moe_desc* desc, Plan* plan, bool routing_only);
+
+// Pointers into saved/workspace resolved for one call.
+struct Buffers {
+  int32_t* topk;      float* gates;   float* probs;   float* logits;
+  float* u;           float* p;       float* loss;
+  int32_t* counts;    int32_t* offsets;   int32_t* pad_offsets;   int32_t* tile_expert;
+  int32_t* rowmap;    // padded sorted row -> flat assignment id (t*k+slot), -1 for padding rows
+  int32_t* flat2row;  // flat assignment id -> padded sorted row
+  int32_t* perm;      int32_t* inv_perm;
+  void* xs;  void* h1;  void* h3;
+  int32_t* status;    float* route_part;  int32_t* perm_counts;  int32_t* perm_base;
+  void* act;  float* yp;  void* dys;  void* dh1;  void* dh3;  void* ga;  float* dxp;
+  float* dg_part;  float* dz;  float* dwr_part;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Launchers (defined in the .cu files).
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, const void* x, const void* w_router,
+                          const float* bias, const float* given_logits, const Buffers& b, cudaStream_t st);
+cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st);
+cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st);
+cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, void* y, cudaStream_t st);
+cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float alpha, float lb_scale,
+                                   int stopgrad_u, int have_dg, const void* x, const void* w_router, const Buffers& b,
+                                   void* dx, float* dw_router, float* dbias, float* dlogits_out, int accumulate,
+                                   cudaStream_t st);
+
+// Expert GEMMs: SIMT fp32 kernels for BTX_F32, tcgen05 kernels for BTX_BF16.
+cudaError_t launch_expert_forward_f32(const Plan& pl, const void* w1, const void* w3, const void* w2,
+                                      const Buffers& b, int save, cudaStream_t st);
+cudaError_t launch_expert_backward_f32(const Plan& pl, const void* w1, const void* w3, const void* w2,
+                                       const Buffers& b, float* dw1, float* dw3, float* dw2, int accumulate,
+                                       cudaStream_t st);
+btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
+                                      const Buffers& b, int save, cudaStream_t st);
+btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
+                                       const Buffers& b, float* dw1, float* dw3, float* dw2, int accumulate,
+                                       cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float sigmoid_f32(float v) { return 1.0f / (1.0f + expf(-v)); }
+
+// a = silu(h1) * h3
+__device__ __forceinline__ float swiglu_f32(float h1, float h3) { return h1 * sigmoid_f32(h1) * h3; }
+
+// Given dact = dL/da: dh1 = dact*h3*s*(1+h1*(1-s)), dh3 = dact*h1*s
+__device__ __forceinline__ void swiglu_bwd_f32(float h1, float h3, float dact, float& dh1, float& dh3) {
+  float s = sigmoid_f32(h1);
+  dh1 = dact * h3 * s * (1.0f + h1 * (1.0f - s));
+  dh3 = dact * h1 * s;
+}
+
+}  // namespace btx

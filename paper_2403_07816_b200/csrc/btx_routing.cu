@@ -1,0 +1,498 @@
+// Router, load-balancing loss, token permutation, row gather / combine and router backward.
+// These are the bandwidth- and latency-bound steps around the expert GEMMs.
+//
+//   router      logits = W_l x (Section 3.2), top-k by repeated arg-max with ties to the lower
+//               index, gate softmax over the selected logits, full softmax, partial sums for
+//               the batch means u and p of Section 3.3
+//   finalize    u, p, L_LB = alpha E sum_i u_i p_i
+//   permutation histogram -> exclusive scan -> stable scatter of the R assignments into
+//               (expert ascending, token ascending) order; expert segments padded to 128 rows
+//   gather      rows of x (or dy) copied into the padded expert-sorted layout
+//   combine     y_t = sum over slots of the gate-scaled expert rows
+//   router bwd  d logits from d gates and the two L_LB terms; dW_l = dz^T x; dx += W_l^T dz
+#include "btx_common.cuh"
+
+namespace btx {
+
+namespace {
+
+constexpr int kRouterThreads = 256;
+constexpr int kRouterWarps = kRouterThreads / 32;
+constexpr int kPermThreads = 256;
+constexpr int kPermChunk = 1024;      // assignments per block of the permutation kernels
+
+template <typename T> struct Vec;     // 16-byte vectors of the element type
+template <> struct Vec<float> {
+  static constexpr int N = 4;
+  static __device__ __forceinline__ void load(const float* p, float (&v)[4]) {
+    float4 q = *reinterpret_cast<const float4*>(p);
+    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+  }
+};
+template <> struct Vec<__nv_bfloat16> {
+  static constexpr int N = 8;
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8]) {
+    uint4 q = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&q);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 f = __bfloat1622float2(h[i]);
+      v[2 * i] = f.x; v[2 * i + 1] = f.y;
+    }
+  }
+};
+
+// ---------------------------------------------------------------------------------------------
+// Router
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kRouterThreads)
+router_kernel(int Tn, int d, int E, int k, int routing, const T* __restrict__ x, const T* __restrict__ wr,
+              const float* __restrict__ bias, const float* __restrict__ given_logits,
+              float* __restrict__ logits, int32_t* __restrict__ topk, float* __restrict__ gates,
+              float* __restrict__ probs, float* __restrict__ route_part) {
+  __shared__ float zs[kRouterWarps][kMaxExperts];
+  __shared__ float red[kRouterWarps][kMaxExperts][2];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int VN = Vec<T>::N;
+  float u_acc = 0.f, p_acc = 0.f;      // lane e accumulates expert e over this warp's tokens
+
+  for (int t = blockIdx.x * kRouterWarps + warp; t < Tn; t += gridDim.x * kRouterWarps) {
+    if (given_logits != nullptr) {
+      if (lane < E) zs[warp][lane] = given_logits[(size_t)t * E + lane];
+    } else {
+      const T* xr = x + (size_t)t * d;
+      for (int eb = 0; eb < E; eb += 8) {
+        float acc[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+        for (int c = lane * VN; c < d; c += 32 * VN) {
+          float xv[VN];
+          Vec<T>::load(xr + c, xv);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (eb + j < E) {
+              float wv[VN];
+              Vec<T>::load(wr + (size_t)(eb + j) * d + c, wv);
+#pragma unroll
+              for (int v = 0; v < VN; ++v) acc[j] = fmaf(xv[v], wv[v], acc[j]);
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          float a = acc[j];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+          if (lane == 0 && eb + j < E) zs[warp][eb + j] = a + (bias ? bias[eb + j] : 0.f);
+        }
+      }
+    }
+    __syncwarp();
+    // Every lane runs the same selection on the shared logits; lane 0 writes the results.
+    const float* z = zs[warp];
+    uint32_t taken = 0;
+    int sel[kMaxExperts];
+    int first = 0;
+    // repeated arg-max: strict '>' keeps the lower index on ties
+    for (int j = 0; j < k; ++j) {
+      int best = -1;
+      float zb = 0.f;
+      for (int e = 0; e < E; ++e) {
+        if ((taken >> e) & 1u) continue;
+        float ze = z[e];
+        if (best < 0 || ze > zb) { best = e; zb = ze; }
+      }
+      taken |= 1u << best;
+      sel[j] = best;
+      if (j == 0) first = best;
+    }
+    const float zmax = z[first];
+    float psum = 0.f;
+    for (int e = 0; e < E; ++e) psum += expf(z[e] - zmax);
+    float my_p = (lane < E) ? expf(z[lane] - zmax) / psum : 0.f;
+    float my_g = 0.f;
+    if (routing == BTX_ROUTE_SWITCH) {
+      float g0 = expf(z[first] - zmax) / psum;
+      if (lane == first) my_g = g0;
+      if (lane == 0) { topk[t] = first; gates[t] = g0; }
+    } else {
+      float gsum = 0.f;
+      for (int j = 0; j < k; ++j) gsum += expf(z[sel[j]] - zmax);
+      for (int j = 0; j < k; ++j) {
+        float gj = expf(z[sel[j]] - zmax) / gsum;
+        if (sel[j] == lane) my_g = gj;
+        if (lane == 0) { topk[(size_t)t * k + j] = sel[j]; gates[(size_t)t * k + j] = gj; }
+      }
+    }
+    if (lane < E) {
+      probs[(size_t)t * E + lane] = my_p;
+      logits[(size_t)t * E + lane] = z[lane];
+      u_acc += my_g;
+      p_acc += my_p;
+    }
+    __syncwarp();
+  }
+  if (lane < E) { red[warp][lane][0] = u_acc; red[warp][lane][1] = p_acc; }
+  __syncthreads();
+  if (threadIdx.x < 2 * E) {
+    int e = threadIdx.x >> 1, which = threadIdx.x & 1;
+    float s = 0.f;
+    for (int w = 0; w < kRouterWarps; ++w) s += red[w][e][which];
+    route_part[(size_t)blockIdx.x * 2 * E + threadIdx.x] = s;
+  }
+}
+
+__global__ void lb_finalize_kernel(int Tn, int E, int nblocks, float alpha, const float* __restrict__ route_part,
+                                   float* __restrict__ u, float* __restrict__ p, float* __restrict__ loss) {
+  __shared__ double su[kMaxExperts], sp[kMaxExperts];
+  int tid = threadIdx.x;
+  if (tid < 2 * E) {
+    double s = 0.0;
+    for (int b = 0; b < nblocks; ++b) s += (double)route_part[(size_t)b * 2 * E + tid];
+    s /= (double)Tn;
+    if (tid & 1) { sp[tid >> 1] = s; p[tid >> 1] = (float)s; }
+    else { su[tid >> 1] = s; u[tid >> 1] = (float)s; }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double acc = 0.0;
+    for (int e = 0; e < E; ++e) acc += su[e] * sp[e];
+    loss[0] = (float)((double)alpha * (double)E * acc);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Permutation
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kPermThreads)
+perm_count_kernel(int R, int E, int nblocks, const int32_t* __restrict__ topk, int32_t* __restrict__ perm_counts) {
+  __shared__ int hist[kMaxExperts];
+  if (threadIdx.x < kMaxExperts) hist[threadIdx.x] = 0;
+  __syncthreads();
+  int base = blockIdx.x * kPermChunk;
+  int end = min(R, base + kPermChunk);
+  for (int i = base + threadIdx.x; i < end; i += kPermThreads) atomicAdd(&hist[topk[i]], 1);
+  __syncthreads();
+  if (threadIdx.x < E) perm_counts[threadIdx.x * nblocks + blockIdx.x] = hist[threadIdx.x];
+}
+
+__global__ void perm_scan_kernel(int E, int nblocks, int mt_max, const int32_t* __restrict__ perm_counts,
+                                 int32_t* __restrict__ perm_base, int32_t* __restrict__ counts,
+                                 int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
+                                 int32_t* __restrict__ tile_expert) {
+  __shared__ int scnt[kMaxExperts];
+  __shared__ int spad[kMaxExperts + 1];
+  int tid = threadIdx.x;
+  if (tid < E) {
+    int run = 0;
+    for (int b = 0; b < nblocks; ++b) {
+      perm_base[tid * nblocks + b] = run;
+      run += perm_counts[tid * nblocks + b];
+    }
+    scnt[tid] = run;
+    counts[tid] = run;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int o = 0, po = 0;
+    for (int e = 0; e < E; ++e) {
+      offsets[e] = o; pad_offsets[e] = po; spad[e] = po;
+      o += scnt[e];
+      po += (scnt[e] + kRowTile - 1) / kRowTile * kRowTile;
+    }
+    offsets[E] = o; pad_offsets[E] = po; spad[E] = po;
+  }
+  __syncthreads();
+  for (int mt = tid; mt < mt_max; mt += blockDim.x) {
+    int row = mt * kRowTile, ex = -1;
+    for (int e = 0; e < E; ++e)
+      if (row >= spad[e] && row < spad[e + 1]) ex = e;
+    tile_expert[mt] = ex;
+  }
+}
+
+__global__ void __launch_bounds__(kPermThreads)
+perm_scatter_kernel(int R, int E, int nblocks, const int32_t* __restrict__ topk, const int32_t* __restrict__ perm_base,
+                    const int32_t* __restrict__ offsets, const int32_t* __restrict__ pad_offsets,
+                    int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
+                    int32_t* __restrict__ flat2row) {
+  constexpr int NW = kPermThreads / 32;
+  __shared__ int running[kMaxExperts + 1];
+  __shared__ int wcnt[NW][kMaxExperts + 1];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x < E) running[threadIdx.x] = perm_base[threadIdx.x * nblocks + blockIdx.x];
+  const int base = blockIdx.x * kPermChunk;
+  const int end = min(R, base + kPermChunk);
+  for (int r0 = base; r0 < end; r0 += kPermThreads) {
+    for (int j = threadIdx.x; j < NW * (kMaxExperts + 1); j += kPermThreads) (&wcnt[0][0])[j] = 0;
+    __syncthreads();
+    int i = r0 + threadIdx.x;
+    int e = (i < end) ? topk[i] : E;                 // E = dummy bucket for idle lanes
+    unsigned same = __match_any_sync(0xffffffffu, e);
+    int rank = __popc(same & ((1u << lane) - 1u));
+    if (rank == 0) wcnt[warp][e] = __popc(same);
+    __syncthreads();
+    if (i < end) {
+      int before = 0;
+      for (int w = 0; w < warp; ++w) before += wcnt[w][e];
+      int within = running[e] + before + rank;
+      int r = offsets[e] + within;                   // tight sorted row
+      int rp = pad_offsets[e] + within;              // padded sorted row
+      perm[r] = i;
+      inv_perm[i] = r;
+      rowmap[rp] = i;
+      flat2row[i] = rp;
+    }
+    __syncthreads();
+    if (threadIdx.x < E) {
+      int s = 0;
+      for (int w = 0; w < NW; ++w) s += wcnt[w][threadIdx.x];
+      running[threadIdx.x] += s;
+    }
+    __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Gather into the padded sorted layout, combine out of it
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(int k, int row_vecs, const uint4* __restrict__ src, uint4* __restrict__ dst,
+                   const int32_t* __restrict__ rowmap, const int32_t* __restrict__ pad_offsets, int E) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total = pad_offsets[E];
+  for (int rp = blockIdx.x * 8 + warp; rp < total; rp += gridDim.x * 8) {
+    int flat = rowmap[rp];
+    uint4* o = dst + (size_t)rp * row_vecs;
+    if (flat < 0) {
+      for (int c = lane; c < row_vecs; c += 32) o[c] = make_uint4(0, 0, 0, 0);
+    } else {
+      const uint4* s = src + (size_t)(flat / k) * row_vecs;
+      for (int c = lane; c < row_vecs; c += 32) o[c] = s[c];
+    }
+  }
+}
+
+template <typename T> __device__ __forceinline__ void store4(T* p, float4 v);
+template <> __device__ __forceinline__ void store4<float>(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 q;
+  q.x = *reinterpret_cast<uint32_t*>(&a);
+  q.y = *reinterpret_cast<uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = q;
+}
+
+// y[t, :] = sum_slot rows[t*k + slot, :]   (+ sum_e dz[t,e] * wr[e, :] when dz != nullptr)
+template <typename T>
+__global__ void __launch_bounds__(256)
+combine_kernel(int Tn, int d, int k, int E, const float* __restrict__ rows, const float* __restrict__ dz,
+               const T* __restrict__ wr, T* __restrict__ y) {
+  const int vecs = d >> 2;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)Tn * vecs;
+       i += (size_t)gridDim.x * blockDim.x) {
+    int t = (int)(i / vecs), c = (int)(i % vecs) * 4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < k; ++s) {
+      float4 v = *reinterpret_cast<const float4*>(rows + ((size_t)t * k + s) * d + c);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    if (dz != nullptr) {
+      for (int e = 0; e < E; ++e) {
+        float g = dz[(size_t)t * E + e];
+        const T* w = wr + (size_t)e * d + c;
+        acc.x = fmaf(g, to_f32(w[0]), acc.x); acc.y = fmaf(g, to_f32(w[1]), acc.y);
+        acc.z = fmaf(g, to_f32(w[2]), acc.z); acc.w = fmaf(g, to_f32(w[3]), acc.w);
+      }
+    }
+    store4<T>(y + (size_t)t * d + c, acc);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Router backward
+// ---------------------------------------------------------------------------------------------
+// One thread per token: d gate of every slot (row-dot partials of the dgrad-2 epilogue summed in
+// tile order, plus the u-term of L_LB), then the softmax Jacobians and the p-term of L_LB.
+__global__ void __launch_bounds__(256)
+router_dz_kernel(int Tn, int E, int k, int routing, float alpha, float lb_scale, int stopgrad_u, int nt_dact,
+                 int r_pad_max, const int32_t* __restrict__ topk, const float* __restrict__ gates,
+                 const float* __restrict__ probs, const float* __restrict__ u, const float* __restrict__ p,
+                 const int32_t* __restrict__ flat2row, const float* __restrict__ dg_part,
+                 float* __restrict__ dz_out, float* __restrict__ dz_out2) {
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= Tn) return;
+  float dzv[kMaxExperts];
+  for (int e = 0; e < E; ++e) dzv[e] = 0.f;
+  const float lbc = lb_scale * alpha * (float)E / (float)Tn;
+  float dg[kMaxExperts];
+  for (int s = 0; s < k; ++s) {
+    float a = 0.f;
+    if (dg_part != nullptr) {
+      int rp = flat2row[(size_t)t * k + s];
+      for (int n = 0; n < nt_dact; ++n) a += dg_part[(size_t)n * r_pad_max + rp];
+    }
+    if (!stopgrad_u) a += lbc * p[topk[(size_t)t * k + s]];
+    dg[s] = a;
+  }
+  const float* pt = probs + (size_t)t * E;
+  if (routing == BTX_ROUTE_SWITCH) {
+    int sel = topk[t];
+    float ps = pt[sel];
+    for (int e = 0; e < E; ++e) dzv[e] = -dg[0] * ps * pt[e];
+    dzv[sel] += dg[0] * ps;
+  } else {
+    float inner = 0.f;
+    for (int s = 0; s < k; ++s) inner += gates[(size_t)t * k + s] * dg[s];
+    for (int s = 0; s < k; ++s) dzv[topk[(size_t)t * k + s]] = gates[(size_t)t * k + s] * (dg[s] - inner);
+  }
+  float pc = 0.f;
+  for (int e = 0; e < E; ++e) pc += pt[e] * (lbc * u[e]);
+  for (int e = 0; e < E; ++e) {
+    float v = dzv[e] + pt[e] * (lbc * u[e] - pc);
+    dz_out[(size_t)t * E + e] = v;
+    if (dz_out2 != nullptr) dz_out2[(size_t)t * E + e] = v;
+  }
+}
+
+constexpr int kWrTokens = 128;   // tokens per chunk of the router-weight gradient
+
+// partial[chunk][e][c] = sum over the chunk's tokens of dz[t,e] * x[t,c]; each thread owns 2 columns.
+template <typename T>
+__global__ void __launch_bounds__(256)
+router_dw_partial_kernel(int Tn, int d, int E, const T* __restrict__ x, const float* __restrict__ dz,
+                         float* __restrict__ part, float* __restrict__ bias_part) {
+  __shared__ float sdz[kWrTokens * kMaxExperts];
+  const int chunk = blockIdx.x;
+  const int t0 = chunk * kWrTokens, t1 = min(Tn, t0 + kWrTokens);
+  for (int i = threadIdx.x; i < (t1 - t0) * E; i += blockDim.x) sdz[i] = dz[(size_t)t0 * E + i];
+  __syncthreads();
+  const int c = (blockIdx.y * blockDim.x + threadIdx.x) * 2;
+  if (blockIdx.y == 0 && threadIdx.x < E) {
+    float s = 0.f;
+    for (int t = 0; t < t1 - t0; ++t) s += sdz[t * E + threadIdx.x];
+    bias_part[(size_t)chunk * E + threadIdx.x] = s;
+  }
+  if (c >= d) return;
+  for (int eb = 0; eb < E; eb += 8) {
+    float acc[8][2];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j][0] = acc[j][1] = 0.f;
+    for (int t = t0; t < t1; ++t) {
+      float x0 = to_f32(x[(size_t)t * d + c]), x1 = to_f32(x[(size_t)t * d + c + 1]);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (eb + j < E) {
+          float g = sdz[(t - t0) * E + eb + j];
+          acc[j][0] = fmaf(g, x0, acc[j][0]);
+          acc[j][1] = fmaf(g, x1, acc[j][1]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (eb + j < E) {
+        float* o = part + ((size_t)chunk * E + eb + j) * d + c;
+        o[0] = acc[j][0]; o[1] = acc[j][1];
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+router_dw_reduce_kernel(int d, int E, int chunks, const float* __restrict__ part, const float* __restrict__ bias_part,
+                        float* __restrict__ dw_router, float* __restrict__ dbias, int accumulate) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < E * d) {
+    float s = 0.f;
+    for (int ch = 0; ch < chunks; ++ch) s += part[(size_t)ch * E * d + i];
+    dw_router[i] = accumulate ? dw_router[i] + s : s;
+  }
+  if (dbias != nullptr && blockIdx.x == 0 && threadIdx.x < E) {
+    float s = 0.f;
+    for (int ch = 0; ch < chunks; ++ch) s += bias_part[(size_t)ch * E + threadIdx.x];
+    dbias[threadIdx.x] = accumulate ? dbias[threadIdx.x] + s : s;
+  }
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// Launchers
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, const void* x, const void* w_router,
+                          const float* bias, const float* given_logits, const Buffers& b, cudaStream_t st) {
+  if (dtype == BTX_BF16) {
+    router_kernel<__nv_bfloat16><<<pl.route_blocks, kRouterThreads, 0, st>>>(
+        pl.T, pl.d, pl.E, pl.k, routing, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, given_logits,
+        b.logits, b.topk, b.gates, b.probs, b.route_part);
+  } else {
+    router_kernel<float><<<pl.route_blocks, kRouterThreads, 0, st>>>(
+        pl.T, pl.d, pl.E, pl.k, routing, (const float*)x, (const float*)w_router, bias, given_logits, b.logits,
+        b.topk, b.gates, b.probs, b.route_part);
+  }
+  lb_finalize_kernel<<<1, 64, 0, st>>>(pl.T, pl.E, pl.route_blocks, alpha, b.route_part, b.u, b.p, b.loss);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(b.rowmap, 0xFF, (size_t)pl.r_pad_max * sizeof(int32_t), st);
+  if (e != cudaSuccess) return e;
+  perm_count_kernel<<<pl.perm_blocks, kPermThreads, 0, st>>>(pl.R, pl.E, pl.perm_blocks, b.topk, b.perm_counts);
+  perm_scan_kernel<<<1, 256, 0, st>>>(pl.E, pl.perm_blocks, pl.mt_max, b.perm_counts, b.perm_base, b.counts,
+                                      b.offsets, b.pad_offsets, b.tile_expert);
+  perm_scatter_kernel<<<pl.perm_blocks, kPermThreads, 0, st>>>(pl.R, pl.E, pl.perm_blocks, b.topk, b.perm_base,
+                                                               b.offsets, b.pad_offsets, b.perm, b.inv_perm, b.rowmap,
+                                                               b.flat2row);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st) {
+  int row_vecs = pl.d * pl.esize / 16;
+  int blocks = min(pl.r_pad_max / 8, 148 * 16);
+  gather_rows_kernel<<<blocks, 256, 0, st>>>(pl.k, row_vecs, (const uint4*)src, (uint4*)dst_sorted, b.rowmap,
+                                             b.pad_offsets, pl.E);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, void* y, cudaStream_t st) {
+  size_t n = (size_t)pl.T * (pl.d / 4);
+  int blocks = (int)min((n + 255) / 256, (size_t)148 * 32);
+  if (dtype == BTX_BF16)
+    combine_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, rows, nullptr, nullptr,
+                                                          (__nv_bfloat16*)y);
+  else
+    combine_kernel<float><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, rows, nullptr, nullptr, (float*)y);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float alpha, float lb_scale,
+                                   int stopgrad_u, int have_dg, const void* x, const void* w_router, const Buffers& b,
+                                   void* dx, float* dw_router, float* dbias, float* dlogits_out, int accumulate,
+                                   cudaStream_t st) {
+  router_dz_kernel<<<(pl.T + 255) / 256, 256, 0, st>>>(pl.T, pl.E, pl.k, routing, alpha, lb_scale, stopgrad_u,
+                                                       pl.nt_dact, pl.r_pad_max, b.topk, b.gates, b.probs, b.u, b.p,
+                                                       b.flat2row, have_dg ? b.dg_part : nullptr, b.dz, dlogits_out);
+  if (x == nullptr) return cudaGetLastError();     // loss-only gradient (btx_lb_loss)
+  dim3 grid(pl.wr_chunks, (pl.d / 2 + 255) / 256);
+  float* bias_part = b.dwr_part + (size_t)pl.wr_chunks * pl.E * pl.d;
+  size_t n = (size_t)pl.T * (pl.d / 4);
+  int cblocks = (int)min((n + 255) / 256, (size_t)148 * 32);
+  if (dtype == BTX_BF16) {
+    router_dw_partial_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(pl.T, pl.d, pl.E, (const __nv_bfloat16*)x, b.dz,
+                                                                  b.dwr_part, bias_part);
+    combine_kernel<__nv_bfloat16><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, b.dxp, b.dz,
+                                                           (const __nv_bfloat16*)w_router, (__nv_bfloat16*)dx);
+  } else {
+    router_dw_partial_kernel<float><<<grid, 256, 0, st>>>(pl.T, pl.d, pl.E, (const float*)x, b.dz, b.dwr_part,
+                                                          bias_part);
+    combine_kernel<float><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, b.dxp, b.dz, (const float*)w_router,
+                                                   (float*)dx);
+  }
+  router_dw_reduce_kernel<<<(pl.E * pl.d + 255) / 256, 256, 0, st>>>(pl.d, pl.E, pl.wr_chunks, b.dwr_part, bias_part,
+                                                                     dw_router, dbias, accumulate);
+  return cudaGetLastError();
+}
+
+}  // namespace btx
