@@ -1,0 +1,153 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element, on
+seeded inputs.  Routing and the dispatch permutation must be bit-exact when the oracle is fed the
+GPU's fp32 logits; floating-point outputs must satisfy max|err|/max|ref| <= 1e-5 in FP32 mode and
+<= 1e-2 in BF16 mode."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import btx_oracle as o
+from paper_2403_07816_b200 import binding as B
+from paper_2403_07816_b200 import synth
+from util import TOL, check_backward, check_forward, gpu_backward, gpu_forward, np64, rel_err
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+DTYPES = [torch.float32, torch.bfloat16]
+
+
+def run_case(T, d, F, E, k, dtype, seed, routing=B.ROUTE_TOPK, alpha=0.01, bias=None, lb_scale=1.0,
+             stopgrad_u=False, backward=True):
+    inp = synth.moe_inputs(T, d, F, E, seed, dtype, DEV)
+    tol = TOL[dtype]
+    kk = E if routing == B.ROUTE_SOFT else k
+    fwd = gpu_forward(inp, k, routing, alpha, bias, save=backward, stopgrad_u=stopgrad_u)
+    cpu, b64, z_gpu, ref = check_forward(inp, fwd, kk, routing, alpha, bias, tol)
+    if backward:
+        got = gpu_backward(inp, fwd, lb_scale, bias)
+        check_backward(cpu, b64, z_gpu, got, kk, routing, alpha, lb_scale, stopgrad_u, tol)
+    return inp, fwd, ref
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_tiny_config_forward_backward(dtype):
+    # T=256, d=256, F=688 (= 5*128 + 48: ragged column tiles), E=4, top-2, alpha = 0.01, seed 0
+    run_case(256, 256, 688, 4, 2, dtype, seed=0)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("T,d,F,E,k", [(37, 64, 72, 5, 3), (1, 128, 128, 4, 2), (300, 136, 264, 8, 2),
+                                        (129, 64, 64, 1, 1), (515, 192, 328, 3, 1)])
+def test_ragged_shapes(dtype, T, d, F, E, k):
+    run_case(T, d, F, E, k, dtype, seed=11, alpha=0.05, lb_scale=0.7)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_switch_routing(dtype):
+    run_case(200, 128, 136, 4, 1, dtype, seed=3, routing=B.ROUTE_SWITCH, alpha=0.02)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_soft_routing(dtype):
+    run_case(150, 128, 136, 4, 4, dtype, seed=3, routing=B.ROUTE_SOFT, alpha=0.02)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_router_bias_skew_and_empty_expert(dtype):
+    bias = torch.tensor([1.5, 0.0, -100.0, 0.2], dtype=torch.float32, device=DEV)   # expert 2 never chosen
+    inp, fwd, ref = run_case(260, 128, 200, 4, 2, dtype, seed=5, bias=bias)
+    assert int(fwd["routing"].counts[2].item()) == 0
+    assert int(fwd["routing"].counts[0].item()) > 130
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_lb_stopgrad_and_zero_alpha(dtype):
+    run_case(96, 64, 72, 4, 2, dtype, seed=6, alpha=0.3, stopgrad_u=True)
+    run_case(96, 64, 72, 4, 2, dtype, seed=6, alpha=0.0)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_accumulate_adds_to_existing_gradients(dtype):
+    inp = synth.moe_inputs(70, 64, 72, 4, 8, dtype, DEV)
+    fwd = gpu_forward(inp, 2)
+    cpu, b64, z_gpu, _ = check_forward(inp, fwd, 2, B.ROUTE_TOPK, 0.01, None, TOL[dtype])
+    got = gpu_backward(inp, fwd, accumulate=True, init=0.25)
+    check_backward(cpu, b64, z_gpu, got, 2, B.ROUTE_TOPK, 0.01, 1.0, False, TOL[dtype], base=0.25)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_tied_logits_go_to_lower_index_and_identical_experts(dtype):
+    # zero router: every logit ties -> experts (0, 1), gates 1/2, L_LB = alpha exactly;
+    # identical experts -> the layer equals the dense FFN
+    inp = synth.moe_inputs(64, 64, 72, 4, 9, dtype, DEV)
+    inp["w_router"].zero_()
+    for n in ("w1", "w3", "w2"):
+        inp[n][1:] = inp[n][:1]
+    fwd = gpu_forward(inp, 2, alpha=0.01, save=False)
+    r = fwd["routing"]
+    assert (r.topk_idx.cpu().numpy() == np.array([[0, 1]])).all()
+    assert (r.gates.cpu().numpy() == 0.5).all()
+    assert abs(float(r.lb_loss.item()) - 0.01) < 1e-8
+    dense = o.swiglu_ffn(np64(inp["x"]), np64(inp["w1"][0]), np64(inp["w3"][0]), np64(inp["w2"][0]))
+    assert rel_err(np64(fwd["y"]), dense) <= TOL[dtype]
+
+
+def test_results_are_deterministic_across_runs():
+    inp = synth.moe_inputs(256, 256, 688, 4, 0, torch.float32, DEV)
+    a = gpu_forward(inp, 2)
+    ga = gpu_backward(inp, a)
+    b = gpu_forward(inp, 2)
+    gb = gpu_backward(inp, b)
+    assert torch.equal(a["y"], b["y"])
+    for n in ga:
+        assert torch.equal(ga[n], gb[n]), n
+
+
+@pytest.mark.parametrize("routing,k", [(B.ROUTE_TOPK, 2), (B.ROUTE_SWITCH, 1), (B.ROUTE_SOFT, 4)])
+def test_lb_loss_entry_point(routing, k):
+    T, E, alpha = 333, 4, 0.01
+    g = torch.Generator(device="cpu").manual_seed(4)
+    logits = (torch.randn(T, E, generator=g) * 1.3).to(DEV)
+    desc = B.make_desc(T, 0, 0, E, k, torch.float32, routing, alpha)
+    ws = torch.empty(B.btx_lb_loss_workspace_size(desc), dtype=torch.uint8, device=DEV)
+    loss = torch.empty(1, device=DEV); u = torch.empty(E, device=DEV); p = torch.empty(E, device=DEV)
+    dz = torch.empty(T, E, device=DEV)
+    B.btx_lb_loss(desc, logits, loss, u, p, dz, ws)
+    z = logits.cpu().numpy()
+    kk = E if routing == B.ROUTE_SOFT else k
+    want, wu, wp = o.lb_loss_from_logits(z, kk, routing, alpha)
+    assert abs(loss.item() - want) <= 1e-5 * want
+    assert rel_err(u.cpu().numpy(), wu) <= 1e-5 and rel_err(p.cpu().numpy(), wp) <= 1e-5
+    assert rel_err(dz.cpu().numpy(), o.lb_loss_grad(z, kk, routing, alpha)) <= 1e-5
+
+
+@pytest.mark.parametrize("dtype,name", [(torch.float32, "f32"), (torch.bfloat16, "bf16")])
+def test_merge_toy_models(dtype, name):
+    # 4 seeded copies of a 2-layer d=256 toy model (vocab 1024) merged into one MoE model
+    models = synth.expert_models(4, 2, 256, 688, 1024, seed=0, dtype=dtype, device=DEV)
+    # one tensor with an odd element count exercises the scalar tail
+    for m, mod in enumerate(models):
+        mod["odd_tail"] = synth.normal((1003,), 0.02, 0, 999, dtype, DEV, layer=m)
+    out = {}
+    for n, t in models[0].items():
+        out[n] = torch.full(((4,) + tuple(t.shape)) if ".ffn." in n else tuple(t.shape), 7.0, dtype=dtype, device=DEV)
+    B.btx_merge(models, out)
+    torch.cuda.synchronize()
+    ref = o.merge_models([{n: np64(t) for n, t in m.items()} for m in models], name)
+    ulp = 2.0 ** -8 if dtype == torch.bfloat16 else 2.0 ** -24
+    for n in out:
+        got = np64(out[n])
+        if ".ffn." in n:
+            assert np.array_equal(got, ref[n]), n                  # copies are bit-exact
+        else:
+            # fp32 running sum vs one rounding of the exact mean: at most one unit in the last place
+            assert np.all(np.abs(got - ref[n]) <= ulp * np.abs(ref[n]) * 1.0001 + 1e-45), n
+            assert np.mean(got != ref[n]) < 2e-2, n
+    # identical models: the merge returns the seed bit for bit (N = 4 is a power of two)
+    same = [models[0]] * 4
+    B.btx_merge(same, out)
+    torch.cuda.synchronize()
+    for n in out:
+        if ".ffn." not in n:
+            assert torch.equal(out[n], models[0][n]), n
