@@ -1,5 +1,581 @@
+// BF16 expert GEMMs on the 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM,
+// operands staged in shared memory by TMA), one persistent warp-specialised kernel template.
+//
+//   warp 0      TMA producer: fills a 4-stage ring of (A 128x64, B 256x64) bf16 tiles
+//   warp 1      allocates TMEM, issues tcgen05.mma (one lane), commits to mbarriers
+//   warps 2-5   epilogue: tcgen05.ld of a 128x256 fp32 accumulator (one row per thread),
+//               fused element-wise work, stores.  Two accumulators (2 x 256 TMEM columns)
+//               let the epilogue of tile i overlap the main loop of tile i+1.
+//
+// Modes (all grouped by expert through the 128-row padded sorted layout):
+//   FWD1   [h1|h3] = Xs [W1;W3]^T, epilogue a = silu(h1)*h3        (Section 3.2, FF_i)
+//   FWD2   rows   = a W2^T, epilogue gate scale + scatter to t*k+slot rows
+//   DACT   dA'    = dYs W2, epilogue SwiGLU backward, g*a, row-dot <dA', a> (d gate)
+//   DX     dXs    = dh1 W1 + dh3 W3 (contraction over 2F), epilogue scatter
+//   WGRAD  dW_e   = P_e^T Q_e, contraction over the expert's token rows, fp32 output
+// Operands whose contraction index is not contiguous in memory (weights in DACT/DX, both
+// operands in WGRAD) are fed as MN-major shared-memory tiles, so nothing is ever transposed.
+//
+// Every mbarrier wait is bounded: after about two seconds it records BTX_ERR_TIMEOUT in the
+// workspace status word, raises a CTA-wide abort flag and the kernel drains and returns.
+#include <cuda.h>
+
 #include "btx_common.cuh"
+
 namespace btx {
-btx_status launch_expert_forward_bf16(const Plan&, const void*, const void*, const void*, const Buffers&, int, cudaStream_t) { return BTX_ERR_UNSUPPORTED; }
-btx_status launch_expert_backward_bf16(const Plan&, const void*, const void*, const void*, const Buffers&, float*, float*, float*, int, cudaStream_t) { return BTX_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int CHUNK_BYTES = 64 * BK * 2;                 // one 64x64 MN-major box
+constexpr int TC_THREADS = 192;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int GROUP_N = 8;                               // column tiles per raster group
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+enum TcMode { G_FWD1 = 0, G_FWD2 = 1, G_DACT = 2, G_DX = 3, G_WGRAD = 4 };
+
+struct TcParams {
+  int d, F, E, r_pad_max;
+  int n_tiles;                  // column tiles
+  int m_tiles;                  // WGRAD: row tiles per expert
+  int kb_total;                 // K blocks per tile (grouped modes)
+  int kb_half;                  // DX: K blocks of the first operand pair
+  int M, N;                     // output rows per expert (WGRAD) / columns
+  const int32_t* tile_expert;
+  const int32_t* pad_offsets;
+  const int32_t* rowmap;
+  const float* gates;
+  const __nv_bfloat16* h1;
+  const __nv_bfloat16* h3;
+  __nv_bfloat16* o0;
+  __nv_bfloat16* o1;
+  __nv_bfloat16* o2;
+  float* of;
+  float* dg_part;
+  int save, accumulate;
+  int32_t* status;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  unsigned long long t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(status, (int32_t)BTX_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  K-major: rows of 128 B, 8-row groups
+// 1024 B apart (stride offset).  MN-major: 64-element (128 B) runs along M/N, 8 contraction rows
+// per 1024 B group (stride offset), next 64-element run 8192 B further (leading offset).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
+  uint64_t dsc = (uint64_t)((addr & 0x3FFFFu) >> 4);
+  dsc |= (uint64_t)((mn_major ? CHUNK_BYTES : 16) >> 4) << 16;
+  dsc |= (uint64_t)(1024 >> 4) << 32;
+  dsc |= 1ull << 46;                                      // descriptor version of this architecture
+  dsc |= 2ull << 61;                                      // 128-byte swizzle
+  return dsc;
+}
+
+__device__ __forceinline__ uint4 pack8(const float* v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), e = __floats2bfloat162_rn(v[6], v[7]);
+  return make_uint4(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b),
+                    *reinterpret_cast<uint32_t*>(&c), *reinterpret_cast<uint32_t*>(&e));
+}
+__device__ __forceinline__ void unpack8(uint4 q, float* v) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&q);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 f = __bfloat1622float2(h[i]);
+    v[2 * i] = f.x; v[2 * i + 1] = f.y;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tile schedule: the same function is evaluated by the producer, the MMA issuer and the epilogue
+// ---------------------------------------------------------------------------------------------
+struct Tile {
+  int m0;        // first output row (padded sorted row, or row of the weight gradient)
+  int nt;        // column tile index
+  int e;         // expert
+  int k_base;    // WGRAD: first contraction row
+  int kb;        // K blocks
+};
+
+template <int MODE>
+__device__ __forceinline__ int total_tiles(const TcParams& p) {
+  if (MODE == G_WGRAD) return p.E * p.m_tiles * p.n_tiles;
+  return (p.pad_offsets[p.E] / BM) * p.n_tiles;
+}
+
+template <int MODE>
+__device__ __forceinline__ Tile get_tile(const TcParams& p, int t) {
+  Tile tl;
+  int mt_count, local = t;
+  if (MODE == G_WGRAD) {
+    mt_count = p.m_tiles;
+    tl.e = t / (p.m_tiles * p.n_tiles);
+    local = t - tl.e * p.m_tiles * p.n_tiles;
+  } else {
+    mt_count = p.pad_offsets[p.E] / BM;
+  }
+  // raster: groups of GROUP_N column tiles; inside a group rows advance slowest
+  const int full = p.n_tiles / GROUP_N;
+  const int in_full = full * mt_count * GROUP_N;
+  int g, width, rem;
+  if (local < in_full) { g = local / (mt_count * GROUP_N); rem = local - g * mt_count * GROUP_N; width = GROUP_N; }
+  else { g = full; rem = local - in_full; width = p.n_tiles - full * GROUP_N; }
+  const int mt = rem / width;
+  tl.nt = g * GROUP_N + rem - mt * width;
+  tl.m0 = mt * BM;
+  if (MODE == G_WGRAD) {
+    tl.k_base = p.pad_offsets[tl.e];
+    tl.kb = (p.pad_offsets[tl.e + 1] - tl.k_base) / BK;
+  } else {
+    tl.e = p.tile_expert[mt];
+    tl.k_base = 0;
+    tl.kb = p.kb_total;
+  }
+  return tl;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------------------------
+template <int MODE>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
+               const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
+               const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;                        // 1024-byte aligned ring
+  uint8_t* ctl = smem_raw + (tiles - raw) + STAGES * STAGE_BYTES;       // barriers behind the ring
+  const uint32_t bar_full = smem_u32(ctl);                              // STAGES x 8 B
+  const uint32_t bar_empty = bar_full + STAGES * 8;
+  const uint32_t bar_tfull = bar_empty + STAGES * 8;                    // 2 x 8 B
+  const uint32_t bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + STAGES * 16 + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + STAGES * 16 + 40);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr bool A_MN = (MODE == G_WGRAD);
+  constexpr bool B_MN = (MODE == G_DACT || MODE == G_DX || MODE == G_WGRAD);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + s * 8, 1); mbar_init(bar_empty + s * 8, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + a * 8, 1); mbar_init(bar_tempty + a * 8, 128); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int n_total = total_tiles<MODE>(p);
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer -------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_total && ok; t += gridDim.x) {
+        const Tile tl = get_tile<MODE>(p, t);
+        for (int kb = 0; kb < tl.kb; ++kb) {
+          if (!(ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status))) break;
+          const uint32_t full = bar_full + stage * 8;
+          const uint32_t sA = tiles + stage * STAGE_BYTES, sB = sA + A_BYTES;
+          mbar_expect_tx(full, STAGE_BYTES);
+          if (MODE == G_FWD1) {
+            tma_load_2d(sA, &tmA0, kb * BK, tl.m0, full);
+            tma_load_3d(sB, &tmB0, kb * BK, tl.nt * 128, tl.e, full);
+            tma_load_3d(sB + B_BYTES / 2, &tmB1, kb * BK, tl.nt * 128, tl.e, full);
+          } else if (MODE == G_FWD2) {
+            tma_load_2d(sA, &tmA0, kb * BK, tl.m0, full);
+            tma_load_3d(sB, &tmB0, kb * BK, tl.nt * BN, tl.e, full);
+          } else if (MODE == G_DACT) {
+            tma_load_2d(sA, &tmA0, kb * BK, tl.m0, full);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) tma_load_3d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + j * 64, kb * BK, tl.e, full);
+          } else if (MODE == G_DX) {
+            const bool second = kb >= p.kb_half;
+            const int kk = (second ? kb - p.kb_half : kb) * BK;
+            tma_load_2d(sA, second ? &tmA1 : &tmA0, kk, tl.m0, full);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              tma_load_3d(sB + j * CHUNK_BYTES, second ? &tmB1 : &tmB0, tl.nt * BN + j * 64, kk, tl.e, full);
+          } else {
+            const int row = tl.k_base + kb * BK;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) tma_load_2d(sA + j * CHUNK_BYTES, &tmA0, tl.m0 + j * 64, row, full);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) tma_load_2d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + j * 64, row, full);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer -------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
+                                 ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_total && ok; t += gridDim.x) {
+        const Tile tl = get_tile<MODE>(p, t);
+        if (tl.kb == 0) continue;
+        if (!(ok = mbar_wait(bar_tempty + acc * 8, acc_phase ^ 1u, abort_flag, p.status))) break;
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + acc * BN;
+        for (int kb = 0; kb < tl.kb; ++kb) {
+          if (!(ok = mbar_wait(bar_full + stage * 8, phase, abort_flag, p.status))) break;
+          tc_fence_after();
+          const uint32_t sA = tiles + stage * STAGE_BYTES, sB = sA + A_BYTES;
+          const uint64_t da = smem_desc(sA, A_MN), db = smem_desc(sB, B_MN);
+#pragma unroll
+          for (int k16 = 0; k16 < BK / 16; ++k16) {
+            // advance 16 contraction elements: 32 B inside a K-major row, 16 rows (2048 B) MN-major
+            const uint64_t ao = (uint64_t)((A_MN ? 2048 : 32) * k16 >> 4);
+            const uint64_t bo = (uint64_t)((B_MN ? 2048 : 32) * k16 >> 4);
+            tc_mma(tmem_d, da + ao, db + bo, idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          }
+          tc_commit(bar_empty + stage * 8);              // frees the stage when these MMAs retire
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(bar_tfull + acc * 8);
+        acc ^= 1u;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------- epilogue -------------------------------
+    const int q = warp & 3;                               // TMEM lane quarter this warp may read
+    const int row = q * 32 + lane;
+    uint32_t acc = 0, acc_phase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_total && ok; t += gridDim.x) {
+      const Tile tl = get_tile<MODE>(p, t);
+      const bool have_acc = tl.kb > 0;
+      if (have_acc) {
+        if (!(ok = mbar_wait(bar_tfull + acc * 8, acc_phase, abort_flag, p.status))) break;
+        tc_fence_after();
+      }
+      const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
+      const int rp = tl.m0 + row;
+      float v[32];
+
+      if (MODE == G_FWD1) {
+        float w[32], a[8];
+        const int F = p.F;
+        for (int c = 0; c < 128; c += 32) {
+          tc_ld32(taddr + c, v);
+          tc_ld32(taddr + 128 + c, w);
+          const int col = tl.nt * 128 + c;
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            if (col + g8 * 8 < F) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) a[i] = swiglu_f32(v[g8 * 8 + i], w[g8 * 8 + i]);
+              const size_t o = (size_t)rp * F + col + g8 * 8;
+              *reinterpret_cast<uint4*>(p.o0 + o) = pack8(a);
+              if (p.save) {
+                *reinterpret_cast<uint4*>(p.o1 + o) = pack8(v + g8 * 8);
+                *reinterpret_cast<uint4*>(p.o2 + o) = pack8(w + g8 * 8);
+              }
+            }
+          }
+        }
+      } else if (MODE == G_FWD2 || MODE == G_DX) {
+        const int flat = p.rowmap[rp];
+        const float g = (MODE == G_FWD2 && flat >= 0) ? p.gates[flat] : 1.0f;
+        const int N = p.N;
+        for (int c = 0; c < BN; c += 32) {
+          tc_ld32(taddr + c, v);                          // all lanes take part in the load
+          const int col = tl.nt * BN + c;
+          if (flat >= 0) {
+            float* o = p.of + (size_t)flat * N + col;
+#pragma unroll
+            for (int g4 = 0; g4 < 8; ++g4)
+              if (col + g4 * 4 < N)
+                *reinterpret_cast<float4*>(o + g4 * 4) =
+                    make_float4(g * v[g4 * 4], g * v[g4 * 4 + 1], g * v[g4 * 4 + 2], g * v[g4 * 4 + 3]);
+          }
+        }
+      } else if (MODE == G_DACT) {
+        const int flat = p.rowmap[rp];
+        const float g = flat >= 0 ? p.gates[flat] : 0.f;
+        const int F = p.F;
+        float rowdot = 0.f;
+        for (int c = 0; c < BN; c += 32) {
+          tc_ld32(taddr + c, v);
+          const int col = tl.nt * BN + c;
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            if (col + g8 * 8 < F) {
+              const size_t o = (size_t)rp * F + col + g8 * 8;
+              float h1[8], h3[8], d1[8], d3[8], ga[8];
+              unpack8(*reinterpret_cast<const uint4*>(p.h1 + o), h1);
+              unpack8(*reinterpret_cast<const uint4*>(p.h3 + o), h3);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float da = v[g8 * 8 + i];
+                const float a = swiglu_f32(h1[i], h3[i]);
+                swiglu_bwd_f32(h1[i], h3[i], g * da, d1[i], d3[i]);
+                ga[i] = g * a;
+                rowdot = fmaf(da, a, rowdot);
+              }
+              *reinterpret_cast<uint4*>(p.o0 + o) = pack8(d1);
+              *reinterpret_cast<uint4*>(p.o1 + o) = pack8(d3);
+              *reinterpret_cast<uint4*>(p.o2 + o) = pack8(ga);
+            }
+          }
+        }
+        p.dg_part[(size_t)tl.nt * p.r_pad_max + rp] = rowdot;
+      } else {  // WGRAD
+        const int N = p.N;
+        const bool row_ok = rp < p.M;
+        for (int c = 0; c < BN; c += 32) {
+          if (have_acc) tc_ld32(taddr + c, v);
+          else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = 0.f;
+          }
+          const int col = tl.nt * BN + c;
+          if (row_ok) {
+            float* o = p.of + ((size_t)tl.e * p.M + rp) * N + col;
+#pragma unroll
+            for (int g4 = 0; g4 < 8; ++g4) {
+              if (col + g4 * 4 < N) {
+                float4 r = make_float4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
+                if (p.accumulate) {
+                  const float4 old = *reinterpret_cast<const float4*>(o + g4 * 4);
+                  r.x += old.x; r.y += old.y; r.z += old.z; r.w += old.w;
+                }
+                *reinterpret_cast<float4*>(o + g4 * 4) = r;
+              }
+            }
+          }
+        }
+      }
+      if (have_acc) {
+        tc_fence_before();
+        mbar_arrive(bar_tempty + acc * 8);
+        acc ^= 1u;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side: tensor maps and launches
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)sym;
+  }
+  return fn;
+}
+
+// bf16 tensor [rows, cols] (2D) or [E, rows, cols] (3D), cols contiguous; box = (box_cols, box_rows[, 1])
+bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t experts, uint32_t box_cols,
+              uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {cols, rows, experts};
+  cuuint64_t strides[2] = {cols * 2, cols * rows * 2};
+  cuuint32_t box[3] = {box_cols, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const cuuint32_t rank = experts > 0 ? 3 : 2;
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <int MODE>
+btx_status launch_tc(const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0, const CUtensorMap& b1,
+                     const TcParams& p, int max_tiles, cudaStream_t st) {
+  if (cudaFuncSetAttribute(tc_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+    return BTX_ERR_CUDA;
+  int grid = sm_count();
+  if (grid > max_tiles) grid = max_tiles;
+  if (grid < 1) grid = 1;
+  tc_gemm_kernel<MODE><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a0, a1, b0, b1, p);
+  return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
+}
+
+TcParams base_params(const Plan& pl, const Buffers& b) {
+  TcParams p = {};
+  p.d = pl.d; p.F = pl.F; p.E = pl.E; p.r_pad_max = pl.r_pad_max;
+  p.tile_expert = b.tile_expert; p.pad_offsets = b.pad_offsets; p.rowmap = b.rowmap; p.gates = b.gates;
+  p.status = b.status;
+  return p;
+}
+
+}  // namespace
+
+btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
+                                      const Buffers& b, int save, cudaStream_t st) {
+  const uint64_t d = pl.d, F = pl.F, E = pl.E, RP = pl.r_pad_max;
+  CUtensorMap a, b0, b1;
+  btx_status s;
+  // GEMM-1: [h1|h3] = Xs [W1;W3]^T with the SwiGLU epilogue
+  if (!make_map(&a, b.xs, d, RP, 0, 64, 128) || !make_map(&b0, w1, d, F, E, 64, 128) ||
+      !make_map(&b1, w3, d, F, E, 64, 128))
+    return BTX_ERR_CUDA;
+  TcParams p = base_params(pl, b);
+  p.n_tiles = (pl.F + 127) / 128; p.kb_total = (pl.d + BK - 1) / BK; p.N = pl.F;
+  p.o0 = (__nv_bfloat16*)b.act; p.o1 = (__nv_bfloat16*)b.h1; p.o2 = (__nv_bfloat16*)b.h3; p.save = save;
+  if ((s = launch_tc<G_FWD1>(a, a, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
+  // GEMM-2: gate-scaled expert rows = act W2^T
+  if (!make_map(&a, b.act, F, RP, 0, 64, 128) || !make_map(&b0, w2, F, d, E, 64, 256)) return BTX_ERR_CUDA;
+  p.n_tiles = (pl.d + BN - 1) / BN; p.kb_total = (pl.F + BK - 1) / BK; p.N = pl.d; p.of = b.yp;
+  return launch_tc<G_FWD2>(a, a, b0, b0, p, pl.mt_max * p.n_tiles, st);
+}
+
+btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
+                                       const Buffers& b, float* dw1, float* dw3, float* dw2, int accumulate,
+                                       cudaStream_t st) {
+  const uint64_t d = pl.d, F = pl.F, E = pl.E, RP = pl.r_pad_max;
+  CUtensorMap a0, a1, b0, b1;
+  btx_status s;
+  TcParams p = base_params(pl, b);
+  // dgrad-2: dA' = dYs W2 (W2[d,F] read N-major), SwiGLU backward epilogue
+  if (!make_map(&a0, b.dys, d, RP, 0, 64, 128) || !make_map(&b0, w2, F, d, E, 64, 64)) return BTX_ERR_CUDA;
+  p.n_tiles = (pl.F + BN - 1) / BN; p.kb_total = (pl.d + BK - 1) / BK; p.N = pl.F;
+  p.h1 = (const __nv_bfloat16*)b.h1; p.h3 = (const __nv_bfloat16*)b.h3;
+  p.o0 = (__nv_bfloat16*)b.dh1; p.o1 = (__nv_bfloat16*)b.dh3; p.o2 = (__nv_bfloat16*)b.ga; p.dg_part = b.dg_part;
+  if ((s = launch_tc<G_DACT>(a0, a0, b0, b0, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
+  // dgrad-1: dXs = dh1 W1 + dh3 W3 (weights read N-major), scatter to t*k+slot rows
+  if (!make_map(&a0, b.dh1, F, RP, 0, 64, 128) || !make_map(&a1, b.dh3, F, RP, 0, 64, 128) ||
+      !make_map(&b0, w1, d, F, E, 64, 64) || !make_map(&b1, w3, d, F, E, 64, 64))
+    return BTX_ERR_CUDA;
+  p.n_tiles = (pl.d + BN - 1) / BN; p.kb_half = (pl.F + BK - 1) / BK; p.kb_total = 2 * p.kb_half; p.N = pl.d;
+  p.of = b.dxp;
+  if ((s = launch_tc<G_DX>(a0, a1, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
+  // wgrads: contraction over the expert's padded token rows, both operands MN-major
+  p.accumulate = accumulate;
+  if (!make_map(&a0, b.dys, d, RP, 0, 64, 64) || !make_map(&b0, b.ga, F, RP, 0, 64, 64)) return BTX_ERR_CUDA;
+  p.M = pl.d; p.N = pl.F; p.m_tiles = (pl.d + BM - 1) / BM; p.n_tiles = (pl.F + BN - 1) / BN; p.of = dw2;
+  if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
+  if (!make_map(&a0, b.dh1, F, RP, 0, 64, 64) || !make_map(&a1, b.dh3, F, RP, 0, 64, 64) ||
+      !make_map(&b0, b.xs, d, RP, 0, 64, 64))
+    return BTX_ERR_CUDA;
+  p.M = pl.F; p.N = pl.d; p.m_tiles = (pl.F + BM - 1) / BM; p.n_tiles = (pl.d + BN - 1) / BN; p.of = dw1;
+  if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
+  p.of = dw3;
+  return launch_tc<G_WGRAD>(a1, a1, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st);
+}
+
+}  // namespace btx

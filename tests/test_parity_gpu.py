@@ -15,6 +15,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 DTYPES = [torch.float32, torch.bfloat16]
+IDS = ["f32", "bf16"]
 
 
 def run_case(T, d, F, E, k, dtype, seed, routing=B.ROUTE_TOPK, alpha=0.01, bias=None, lb_scale=1.0,
@@ -30,30 +31,30 @@ def run_case(T, d, F, E, k, dtype, seed, routing=B.ROUTE_TOPK, alpha=0.01, bias=
     return inp, fwd, ref
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 def test_tiny_config_forward_backward(dtype):
     # T=256, d=256, F=688 (= 5*128 + 48: ragged column tiles), E=4, top-2, alpha = 0.01, seed 0
     run_case(256, 256, 688, 4, 2, dtype, seed=0)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 @pytest.mark.parametrize("T,d,F,E,k", [(37, 64, 72, 5, 3), (1, 128, 128, 4, 2), (300, 136, 264, 8, 2),
                                         (129, 64, 64, 1, 1), (515, 192, 328, 3, 1)])
 def test_ragged_shapes(dtype, T, d, F, E, k):
     run_case(T, d, F, E, k, dtype, seed=11, alpha=0.05, lb_scale=0.7)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 def test_switch_routing(dtype):
     run_case(200, 128, 136, 4, 1, dtype, seed=3, routing=B.ROUTE_SWITCH, alpha=0.02)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 def test_soft_routing(dtype):
     run_case(150, 128, 136, 4, 4, dtype, seed=3, routing=B.ROUTE_SOFT, alpha=0.02)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 def test_router_bias_skew_and_empty_expert(dtype):
     bias = torch.tensor([1.5, 0.0, -100.0, 0.2], dtype=torch.float32, device=DEV)   # expert 2 never chosen
     inp, fwd, ref = run_case(260, 128, 200, 4, 2, dtype, seed=5, bias=bias)
@@ -61,13 +62,13 @@ def test_router_bias_skew_and_empty_expert(dtype):
     assert int(fwd["routing"].counts[0].item()) > 130
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 def test_lb_stopgrad_and_zero_alpha(dtype):
     run_case(96, 64, 72, 4, 2, dtype, seed=6, alpha=0.3, stopgrad_u=True)
     run_case(96, 64, 72, 4, 2, dtype, seed=6, alpha=0.0)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 def test_accumulate_adds_to_existing_gradients(dtype):
     inp = synth.moe_inputs(70, 64, 72, 4, 8, dtype, DEV)
     fwd = gpu_forward(inp, 2)
@@ -76,7 +77,7 @@ def test_accumulate_adds_to_existing_gradients(dtype):
     check_backward(cpu, b64, z_gpu, got, 2, B.ROUTE_TOPK, 0.01, 1.0, False, TOL[dtype], base=0.25)
 
 
-@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 def test_tied_logits_go_to_lower_index_and_identical_experts(dtype):
     # zero router: every logit ties -> experts (0, 1), gates 1/2, L_LB = alpha exactly;
     # identical experts -> the layer equals the dense FFN
@@ -122,7 +123,7 @@ def test_lb_loss_entry_point(routing, k):
     assert rel_err(dz.cpu().numpy(), o.lb_loss_grad(z, kk, routing, alpha)) <= 1e-5
 
 
-@pytest.mark.parametrize("dtype,name", [(torch.float32, "f32"), (torch.bfloat16, "bf16")])
+@pytest.mark.parametrize("dtype,name", [(torch.float32, "f32"), (torch.bfloat16, "bf16")], ids=IDS)
 def test_merge_toy_models(dtype, name):
     # 4 seeded copies of a 2-layer d=256 toy model (vocab 1024) merged into one MoE model
     models = synth.expert_models(4, 2, 256, 688, 1024, seed=0, dtype=dtype, device=DEV)
@@ -134,16 +135,22 @@ def test_merge_toy_models(dtype, name):
         out[n] = torch.full(((4,) + tuple(t.shape)) if ".ffn." in n else tuple(t.shape), 7.0, dtype=dtype, device=DEV)
     B.btx_merge(models, out)
     torch.cuda.synchronize()
-    ref = o.merge_models([{n: np64(t) for n, t in m.items()} for m in models], name)
+    cpu_models = [{n: np64(t) for n, t in m.items()} for m in models]
+    ref = o.merge_models(cpu_models, name)
     ulp = 2.0 ** -8 if dtype == torch.bfloat16 else 2.0 ** -24
     for n in out:
         got = np64(out[n])
         if ".ffn." in n:
             assert np.array_equal(got, ref[n]), n                  # copies are bit-exact
         else:
-            # fp32 running sum vs one rounding of the exact mean: at most one unit in the last place
-            assert np.all(np.abs(got - ref[n]) <= ulp * np.abs(ref[n]) * 1.0001 + 1e-45), n
-            assert np.mean(got != ref[n]) < 2e-2, n
+            # The kernel sums in fp32 in model order: each of the N-1 additions rounds by at most
+            # 2^-24 of a partial sum (<= sum |src|); the store rounds once more to the storage type.
+            mean_abs = sum(np.abs(m[n]) for m in cpu_models) / len(cpu_models)
+            bound = ulp * np.abs(ref[n]) * 1.0001 + 3 * 2.0 ** -24 * mean_abs + 1e-45
+            assert np.all(np.abs(got - ref[n]) <= bound), n
+            assert rel_err(got, ref[n]) <= TOL[dtype]
+            if dtype == torch.bfloat16:
+                assert np.mean(got != ref[n]) < 1e-2, n            # the fp32 sum rarely flips a bf16 rounding
     # identical models: the merge returns the seed bit for bit (N = 4 is a power of two)
     same = [models[0]] * 4
     B.btx_merge(same, out)
