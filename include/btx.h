@@ -102,6 +102,22 @@ btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void*
                             float* dw1, float* dw3, float* dw2, int32_t accumulate,
                             void* workspace, size_t workspace_bytes, void* stream);
 
+/* One training step of the layer with HOST activations: copies x_host, dy_host ([T,d], dtype;
+ * pinned memory makes the copies asynchronous) into the device staging buffers x_dev, dy_dev,
+ * runs btx_moe_forward (saving for backward) and btx_moe_backward, and copies y, dx and the
+ * load-balancing loss back to y_host, dx_host, loss_host.  Weights, gradients, staging buffers,
+ * `saved` and `workspace` are device memory as in the two calls it composes; desc.save_for_backward
+ * must be 1.  Everything is enqueued on `stream`; the host results are valid after the stream
+ * has been synchronised. */
+btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_host, const void* dy_host,
+                             void* y_host, void* dx_host, float* loss_host,
+                             void* x_dev, void* dy_dev, void* y_dev, void* dx_dev,
+                             const void* w_router, const float* router_bias,
+                             const void* w1, const void* w3, const void* w2, float lb_grad_scale,
+                             float* dw_router, float* dbias, float* dw1, float* dw3, float* dw2,
+                             int32_t accumulate, void* saved, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
 /* L_LB = alpha * E * sum_i u_i p_i with u_i the batch mean of the gate of expert i and p_i the
  * batch mean of SoftMax_i (Section 3.3), from given fp32 logits[T,E] (bias, if any, already
  * added).  Outputs loss[1], u[E], p[E]; dlogits[T,E] (d loss / d logits) unless NULL.
@@ -132,6 +148,14 @@ btx_status btx_merge(int32_t n_models, int32_t dtype, const btx_merge_item* item
 /* Synchronises `stream` and reads the status word that kernels of earlier calls left in
  * `workspace`: *device_status (host) is BTX_OK or BTX_ERR_TIMEOUT. */
 btx_status btx_device_status(const void* workspace, void* stream, int32_t* device_status);
+
+/* Optional stage timing for the calling host thread.  `events` is a host array of n
+ * cudaEvent_t (as void*), or NULL to switch the hook off.  While set, btx_moe_forward records
+ * events[0..4] on its stream: start, after routing+permutation+gather, after GEMM-1 (W1/W3 +
+ * SwiGLU), after GEMM-2 (W2 + gate scatter), after combine; btx_moe_backward records
+ * events[0..7]: start, after the dy gather, after dgrad-2, after dgrad-1, after the W2, W1 and W3
+ * weight gradients, after the router backward.  Entries beyond n, or NULL entries, are skipped. */
+btx_status btx_set_stage_events(void* const* events, int32_t n);
 
 const char* btx_status_string(btx_status s);
 int32_t btx_version(void);

@@ -44,8 +44,9 @@ class MergeItem(C.Structure):
                 ("src", C.POINTER(C.c_void_p)), ("dst", C.c_void_p)]
 
 
-EXPORTS = ["btx_moe_sizes", "btx_moe_forward", "btx_moe_backward", "btx_lb_loss_workspace_size", "btx_lb_loss",
-           "btx_merge_workspace_size", "btx_merge", "btx_device_status", "btx_status_string", "btx_version"]
+EXPORTS = ["btx_moe_sizes", "btx_moe_forward", "btx_moe_backward", "btx_moe_step_host",
+           "btx_lb_loss_workspace_size", "btx_lb_loss", "btx_merge_workspace_size", "btx_merge",
+           "btx_device_status", "btx_set_stage_events", "btx_status_string", "btx_version"]
 
 
 def lib():
@@ -60,6 +61,8 @@ def lib():
                                       sz, vp]
         L.btx_moe_backward.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp,
                                        i32, vp, sz, vp]
+        L.btx_moe_step_host.argtypes = [C.POINTER(MoeDesc)] + [vp] * 14 + [f32] + [vp] * 5 + [i32, vp, vp, sz, vp]
+        L.btx_set_stage_events.argtypes = [C.POINTER(vp), i32]
         L.btx_lb_loss_workspace_size.argtypes = [C.POINTER(MoeDesc), C.POINTER(sz)]
         L.btx_lb_loss.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, sz, vp]
         L.btx_merge_workspace_size.argtypes = [i32, C.c_uint64, C.POINTER(sz)]
@@ -165,6 +168,41 @@ def btx_moe_backward(desc, x, w_router, router_bias, w1, w3, w2, dy, lb_grad_sca
                                _stream(x.device))
     if s != BTX_OK:
         raise BtxError(s, "btx_moe_backward")
+
+
+def btx_moe_step_host(desc, x_host, dy_host, y_host, dx_host, loss_host, x_dev, dy_dev, y_dev, dx_dev, w_router,
+                      router_bias, w1, w3, w2, lb_grad_scale, dw_router, dbias, dw1, dw3, dw2, accumulate, saved,
+                      workspace):
+    """Forward + backward with activations in (pinned) host tensors; see btx.h."""
+    for t in (x_host, dy_host, y_host, dx_host, loss_host):
+        if t.is_cuda or not t.is_contiguous():
+            raise RuntimeError("btx_moe_step_host: host tensors must be contiguous CPU tensors")
+    hp = lambda t: C.c_void_p(t.data_ptr())
+    s = lib().btx_moe_step_host(C.byref(desc), hp(x_host), hp(dy_host), hp(y_host), hp(dx_host), hp(loss_host),
+                                _ptr(x_dev), _ptr(dy_dev), _ptr(y_dev), _ptr(dx_dev), _ptr(w_router),
+                                _ptr(router_bias), _ptr(w1), _ptr(w3), _ptr(w2), float(lb_grad_scale),
+                                _ptr(dw_router), _ptr(dbias), _ptr(dw1), _ptr(dw3), _ptr(dw2), int(accumulate),
+                                _ptr(saved), _ptr(workspace), workspace.numel(), _stream(x_dev.device))
+    if s != BTX_OK:
+        raise BtxError(s, "btx_moe_step_host")
+
+
+_stage_keepalive = None
+
+
+def btx_set_stage_events(events):
+    """events: list of torch.cuda.Event(enable_timing=True) that have been recorded at least once
+    (so that their handles exist), or None to switch the hook off."""
+    global _stage_keepalive
+    if events is None:
+        _stage_keepalive = None
+        s = lib().btx_set_stage_events(None, 0)
+    else:
+        arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+        _stage_keepalive = (arr, events)
+        s = lib().btx_set_stage_events(arr, len(events))
+    if s != BTX_OK:
+        raise BtxError(s, "btx_set_stage_events")
 
 
 def btx_lb_loss_workspace_size(desc):

@@ -95,6 +95,14 @@ static void resolve(const Plan& p, char* saved, char* ws, Buffers* b) {
   b->dg_part = (float*)(ws + p.w_dg_part);  b->dz = (float*)(ws + p.w_dz);  b->dwr_part = (float*)(ws + p.w_dwr_part);
 }
 
+static thread_local void* const* g_stage_events = nullptr;
+static thread_local int g_stage_count = 0;
+
+void mark_stage(int i, cudaStream_t st) {
+  if (g_stage_events != nullptr && i < g_stage_count && g_stage_events[i] != nullptr)
+    cudaEventRecord((cudaEvent_t)g_stage_events[i], st);
+}
+
 static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
 
 static btx_status check_device() {
@@ -141,16 +149,20 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
   Buffers b;
   resolve(pl, sv, ws, &b);
 
+  mark_stage(0, st);
   BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
   BTX_CUDA_OK(launch_router(pl, desc->dtype, desc->routing, desc->lb_alpha, x, w_router, router_bias, nullptr, b, st));
   BTX_CUDA_OK(launch_permute(pl, b, st));
   BTX_CUDA_OK(launch_gather_rows(pl, x, b.xs, b, st));
+  mark_stage(1, st);
   if (desc->dtype == BTX_F32) {
     BTX_CUDA_OK(launch_expert_forward_f32(pl, w1, w3, w2, b, desc->save_for_backward, st));
   } else {
     if ((s = launch_expert_forward_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
   }
+  mark_stage(3, st);
   BTX_CUDA_OK(launch_combine(pl, desc->dtype, b.yp, y, st));
+  mark_stage(4, st);
 
   if (routing) {
     auto out = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
@@ -193,8 +205,10 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
   cudaStream_t st = (cudaStream_t)stream;
   Buffers b;
   resolve(pl, (char*)saved, (char*)workspace, &b);
+  mark_stage(0, st);
   BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
   BTX_CUDA_OK(launch_gather_rows(pl, dy, b.dys, b, st));
+  mark_stage(1, st);
   if (desc->dtype == BTX_F32) {
     BTX_CUDA_OK(launch_expert_backward_f32(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, st));
   } else {
@@ -203,6 +217,45 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
   BTX_CUDA_OK(launch_router_backward(pl, desc->dtype, desc->routing, desc->lb_alpha, lb_grad_scale,
                                      desc->lb_stopgrad_u, 1, x, w_router, b, dx, dw_router, dbias, nullptr,
                                      accumulate, st));
+  mark_stage(7, st);
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_host, const void* dy_host,
+                                        void* y_host, void* dx_host, float* loss_host, void* x_dev, void* dy_dev,
+                                        void* y_dev, void* dx_dev, const void* w_router, const float* router_bias,
+                                        const void* w1, const void* w3, const void* w2, float lb_grad_scale,
+                                        float* dw_router, float* dbias, float* dw1, float* dw3, float* dw2,
+                                        int32_t accumulate, void* saved, void* workspace, size_t workspace_bytes,
+                                        void* stream) {
+  Plan pl;
+  btx_status s = make_plan(desc, &pl, false);
+  if (s != BTX_OK) return s;
+  if (!x_host || !dy_host || !y_host || !dx_host || !loss_host || !x_dev || !dy_dev || !y_dev || !dx_dev || !saved)
+    return BTX_ERR_INVALID_ARG;
+  if (!desc->save_for_backward) return BTX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t act_bytes = (size_t)pl.T * pl.d * pl.esize;
+  BTX_CUDA_OK(cudaMemcpyAsync(x_dev, x_host, act_bytes, cudaMemcpyHostToDevice, st));
+  BTX_CUDA_OK(cudaMemcpyAsync(dy_dev, dy_host, act_bytes, cudaMemcpyHostToDevice, st));
+  btx_routing_out ro;
+  memset(&ro, 0, sizeof(ro));
+  if ((s = btx_moe_forward(desc, x_dev, w_router, router_bias, w1, w3, w2, y_dev, &ro, saved, workspace,
+                           workspace_bytes, stream)) != BTX_OK)
+    return s;
+  if ((s = btx_moe_backward(desc, x_dev, w_router, router_bias, w1, w3, w2, dy_dev, lb_grad_scale, saved, dx_dev,
+                            dw_router, dbias, dw1, dw3, dw2, accumulate, workspace, workspace_bytes, stream)) != BTX_OK)
+    return s;
+  BTX_CUDA_OK(cudaMemcpyAsync(y_host, y_dev, act_bytes, cudaMemcpyDeviceToHost, st));
+  BTX_CUDA_OK(cudaMemcpyAsync(dx_host, dx_dev, act_bytes, cudaMemcpyDeviceToHost, st));
+  BTX_CUDA_OK(cudaMemcpyAsync(loss_host, (const char*)saved + pl.s_loss, 4, cudaMemcpyDeviceToHost, st));
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_set_stage_events(void* const* events, int32_t n) {
+  if (events != nullptr && n < 1) return BTX_ERR_INVALID_ARG;
+  g_stage_events = events;
+  g_stage_count = events ? n : 0;
   return BTX_OK;
 }
 

@@ -51,6 +51,9 @@ struct Buffers {
   float* dg_part;  float* dz;  float* dwr_part;
 };
 
+// Records stage event i of the calling thread's timing hook (no-op when the hook is off).
+void mark_stage(int i, cudaStream_t st);
+
 // ---------------------------------------------------------------------------------------------
 // Launchers (defined in the .cu files).
 // ---------------------------------------------------------------------------------------------

@@ -176,6 +176,7 @@ cudaError_t launch_expert_forward_f32(const Plan& pl, const void* w1, const void
   p.a0 = (const float*)b.xs; p.b0 = (const float*)w1; p.b1 = (const float*)w3;
   p.o0 = (float*)b.act; p.o1 = (float*)b.h1; p.o2 = (float*)b.h3; p.save = save; p.N = pl.F;
   simt_gemm_kernel<S_FWD1><<<dim3((pl.F + TN - 1) / TN, mt), 256, 0, st>>>(p);
+  mark_stage(2, st);
   // GEMM-2: gate-scaled expert rows
   p.a0 = (const float*)b.act; p.b0 = (const float*)w2; p.o0 = b.yp; p.N = pl.d;
   simt_gemm_kernel<S_FWD2><<<dim3((pl.d + TN - 1) / TN, mt), 256, 0, st>>>(p);
@@ -194,17 +195,22 @@ cudaError_t launch_expert_backward_f32(const Plan& pl, const void* w1, const voi
   p.a0 = (const float*)b.dys; p.b0 = (const float*)w2; p.h1 = (const float*)b.h1; p.h3 = (const float*)b.h3;
   p.o0 = (float*)b.dh1; p.o1 = (float*)b.dh3; p.o2 = (float*)b.ga; p.dg_part = b.dg_part; p.N = pl.F;
   simt_gemm_kernel<S_DACT><<<dim3((pl.F + TN - 1) / TN, mt), 256, 0, st>>>(p);
+  mark_stage(2, st);
   // dgrad-1: dXs = dh1 W1 + dh3 W3
   p.a0 = (const float*)b.dh1; p.a1 = (const float*)b.dh3; p.b0 = (const float*)w1; p.b1 = (const float*)w3;
   p.o0 = b.dxp; p.N = pl.d;
   simt_gemm_kernel<S_DX><<<dim3((pl.d + TN - 1) / TN, mt), 256, 0, st>>>(p);
+  mark_stage(3, st);
   // wgrads: contraction over the expert's (padded) token rows
   p.a0 = (const float*)b.dys; p.ldp = pl.d; p.b0 = (const float*)b.ga; p.ldq = pl.F; p.o0 = dw2; p.M = pl.d; p.N = pl.F;
   simt_gemm_kernel<S_WGRAD><<<dim3((pl.F + TN - 1) / TN, (pl.d + TM - 1) / TM, pl.E), 256, 0, st>>>(p);
+  mark_stage(4, st);
   p.a0 = (const float*)b.dh1; p.ldp = pl.F; p.b0 = (const float*)b.xs; p.ldq = pl.d; p.o0 = dw1; p.M = pl.F; p.N = pl.d;
   simt_gemm_kernel<S_WGRAD><<<dim3((pl.d + TN - 1) / TN, (pl.F + TM - 1) / TM, pl.E), 256, 0, st>>>(p);
+  mark_stage(5, st);
   p.a0 = (const float*)b.dh3; p.o0 = dw3;
   simt_gemm_kernel<S_WGRAD><<<dim3((pl.d + TN - 1) / TN, (pl.F + TM - 1) / TM, pl.E), 256, 0, st>>>(p);
+  mark_stage(6, st);
   return cudaGetLastError();
 }
 

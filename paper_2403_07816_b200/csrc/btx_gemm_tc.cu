@@ -538,6 +538,7 @@ btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void
   p.n_tiles = (pl.F + 127) / 128; p.kb_total = (pl.d + BK - 1) / BK; p.N = pl.F;
   p.o0 = (__nv_bfloat16*)b.act; p.o1 = (__nv_bfloat16*)b.h1; p.o2 = (__nv_bfloat16*)b.h3; p.save = save;
   if ((s = launch_tc<G_FWD1>(a, a, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
+  mark_stage(2, st);
   // GEMM-2: gate-scaled expert rows = act W2^T
   if (!make_map(&a, b.act, F, RP, 0, 64, 128) || !make_map(&b0, w2, F, d, E, 64, 256)) return BTX_ERR_CUDA;
   p.n_tiles = (pl.d + BN - 1) / BN; p.kb_total = (pl.F + BK - 1) / BK; p.N = pl.d; p.of = b.yp;
@@ -557,6 +558,7 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   p.h1 = (const __nv_bfloat16*)b.h1; p.h3 = (const __nv_bfloat16*)b.h3;
   p.o0 = (__nv_bfloat16*)b.dh1; p.o1 = (__nv_bfloat16*)b.dh3; p.o2 = (__nv_bfloat16*)b.ga; p.dg_part = b.dg_part;
   if ((s = launch_tc<G_DACT>(a0, a0, b0, b0, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
+  mark_stage(2, st);
   // dgrad-1: dXs = dh1 W1 + dh3 W3 (weights read N-major), scatter to t*k+slot rows
   if (!make_map(&a0, b.dh1, F, RP, 0, 64, 128) || !make_map(&a1, b.dh3, F, RP, 0, 64, 128) ||
       !make_map(&b0, w1, d, F, E, 64, 64) || !make_map(&b1, w3, d, F, E, 64, 64))
@@ -564,18 +566,23 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   p.n_tiles = (pl.d + BN - 1) / BN; p.kb_half = (pl.F + BK - 1) / BK; p.kb_total = 2 * p.kb_half; p.N = pl.d;
   p.of = b.dxp;
   if ((s = launch_tc<G_DX>(a0, a1, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
+  mark_stage(3, st);
   // wgrads: contraction over the expert's padded token rows, both operands MN-major
   p.accumulate = accumulate;
   if (!make_map(&a0, b.dys, d, RP, 0, 64, 64) || !make_map(&b0, b.ga, F, RP, 0, 64, 64)) return BTX_ERR_CUDA;
   p.M = pl.d; p.N = pl.F; p.m_tiles = (pl.d + BM - 1) / BM; p.n_tiles = (pl.F + BN - 1) / BN; p.of = dw2;
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
+  mark_stage(4, st);
   if (!make_map(&a0, b.dh1, F, RP, 0, 64, 64) || !make_map(&a1, b.dh3, F, RP, 0, 64, 64) ||
       !make_map(&b0, b.xs, d, RP, 0, 64, 64))
     return BTX_ERR_CUDA;
   p.M = pl.F; p.N = pl.d; p.m_tiles = (pl.F + BM - 1) / BM; p.n_tiles = (pl.d + BN - 1) / BN; p.of = dw1;
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
+  mark_stage(5, st);
   p.of = dw3;
-  return launch_tc<G_WGRAD>(a1, a1, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st);
+  s = launch_tc<G_WGRAD>(a1, a1, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st);
+  mark_stage(6, st);
+  return s;
 }
 
 }  // namespace btx
