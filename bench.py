@@ -201,6 +201,8 @@ def run_moe(args, workload):
     barrier(world)
     dev = torch.device("cuda", local)
     T, d, F, E, k, seed = WORKLOADS[workload]
+    if args.tokens:
+        T = args.tokens                      # reduced batch for profiler captures
     train = workload == "fwd_bwd"
     layers = 32 if workload == "decode" else 1
     K, W = args.steps, max(args.warmup, 3)
@@ -307,7 +309,7 @@ def run_moe(args, workload):
                             "frac_of_nominal_2250": achieved / 2250.0}
 
     # ---- end to end through the host-buffer entry point (training workload only) ----
-    if train:
+    if train and not args.no_e2e:
         inp = sets[0]
         hx = inp["x"].cpu().pin_memory(); hdy = inp["dy"].cpu().pin_memory()
         hy = torch.empty_like(hx).pin_memory(); hdx = torch.empty_like(hx).pin_memory()
@@ -335,7 +337,7 @@ def run_moe(args, workload):
         line["e2e"] = None
 
     # ---- CPU oracle beside it (rank 0, single GPU only) ----
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and workload != "decode":
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and workload != "decode" and not args.tokens:
         del sets
         torch.cuda.empty_cache()
         n_tok = 128 if train else 256
@@ -434,6 +436,8 @@ def main():
     ap.add_argument("--workload", default="fwd_bwd", choices=["fwd_bwd", "fwd", "decode", "merge"])
     ap.add_argument("--merge-layers", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--tokens", type=int, default=0, help="override T (profiling only; not a bench number)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
