@@ -126,6 +126,24 @@ btx_status btx_lb_loss_workspace_size(const btx_moe_desc* desc, size_t* workspac
 btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits, float* loss, float* u, float* p,
                        float* dlogits, void* workspace, size_t workspace_bytes, void* stream);
 
+/* btx_lb_loss without a caller-supplied workspace (the paper has no counterpart; this is a
+ * packaging variant of the call above).  It is meant for callers that hold no allocator: plug-in
+ * code that is handed tensors by a host framework whose memory pool owns all device memory, or a
+ * training loop that must not pay for the device-wide synchronisation a cudaMalloc implies.  The
+ * scratch lives in a 4 MiB (BTX_LB_NOALLOC_SCRATCH_BYTES) static device array inside the library,
+ * which every GPU that loads the library holds until the process exits.  Same arguments and
+ * results as btx_lb_loss; inputs and outputs are still the caller's.
+ *   - Requests whose btx_lb_loss_workspace_size exceeds the array return BTX_ERR_WORKSPACE and
+ *     launch nothing (4 MiB covers e.g. T = 32768 tokens with E = 4).
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current); make that first call before starting any stream capture.
+ *   - The call allocates and frees nothing.  All calls on one device share the array, which keeps
+ *     whatever the previous call left in it (the call itself clears the part that must start at
+ *     zero): two calls whose kernels may overlap on the GPU, e.g. on different streams, race. */
+#define BTX_LB_NOALLOC_SCRATCH_BYTES (4u << 20)
+btx_status btx_lb_loss_noalloc(const btx_moe_desc* desc, const float* logits, float* loss, float* u, float* p,
+                               float* dlogits, void* stream);
+
 /* MiX merge (Section 3.2): the feed-forward matrices of the N expert LLMs become the experts of
  * one MoE layer (kind FFN: dst[e*numel .. ] = src[e], bit for bit); every other parameter is the
  * uniform mean over the N models (kind AVERAGE: fp32 sum in model order, divided by N, rounded

@@ -45,7 +45,7 @@ class MergeItem(C.Structure):
 
 
 EXPORTS = ["btx_moe_sizes", "btx_moe_forward", "btx_moe_backward", "btx_moe_step_host",
-           "btx_lb_loss_workspace_size", "btx_lb_loss", "btx_merge_workspace_size", "btx_merge",
+           "btx_lb_loss_workspace_size", "btx_lb_loss", "btx_lb_loss_noalloc", "btx_merge_workspace_size", "btx_merge",
            "btx_device_status", "btx_set_stage_events", "btx_status_string", "btx_version"]
 
 
@@ -65,6 +65,7 @@ def lib():
         L.btx_set_stage_events.argtypes = [C.POINTER(vp), i32]
         L.btx_lb_loss_workspace_size.argtypes = [C.POINTER(MoeDesc), C.POINTER(sz)]
         L.btx_lb_loss.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, sz, vp]
+        L.btx_lb_loss_noalloc.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp]
         L.btx_merge_workspace_size.argtypes = [i32, C.c_uint64, C.POINTER(sz)]
         L.btx_merge.argtypes = [i32, i32, C.POINTER(MergeItem), C.c_uint64, vp, sz, vp]
         L.btx_device_status.argtypes = [vp, vp, C.POINTER(i32)]
@@ -218,6 +219,14 @@ def btx_lb_loss(desc, logits, loss, u, p, dlogits, workspace):
                           workspace.numel(), _stream(logits.device))
     if s != BTX_OK:
         raise BtxError(s, "btx_lb_loss")
+
+
+def btx_lb_loss_noalloc(desc, logits, loss, u, p, dlogits):
+    """btx_lb_loss on the library's own static scratch: no workspace argument, nothing allocated."""
+    s = lib().btx_lb_loss_noalloc(C.byref(desc), _ptr(logits), _ptr(loss), _ptr(u), _ptr(p), _ptr(dlogits),
+                                  _stream(logits.device))
+    if s != BTX_OK:
+        raise BtxError(s, "btx_lb_loss_noalloc")
 
 
 def btx_merge_workspace_size(n_models, n_items):

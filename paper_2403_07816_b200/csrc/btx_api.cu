@@ -2,6 +2,7 @@
 // forward and backward passes (see include/btx.h for the contract of every call).
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "btx_common.cuh"
 
@@ -290,6 +291,40 @@ extern "C" btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits,
                                        nullptr, nullptr, b, nullptr, nullptr, nullptr, dlogits, 0, st));
   }
   return BTX_OK;
+}
+
+// Scratch of btx_lb_loss_noalloc.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the device address it resolves to differs per GPU.
+static __device__ __align__(256) unsigned char g_lb_noalloc_scratch[BTX_LB_NOALLOC_SCRATCH_BYTES];
+
+static btx_status lb_noalloc_scratch(void** out) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static void* addr[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return BTX_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return BTX_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(mu);
+  if (addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_lb_noalloc_scratch) != cudaSuccess || ptr == nullptr) return BTX_ERR_CUDA;
+    addr[dev] = ptr;
+  }
+  *out = addr[dev];
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_lb_loss_noalloc(const btx_moe_desc* desc, const float* logits, float* loss, float* u,
+                                          float* p, float* dlogits, void* stream) {
+  size_t need = 0;
+  btx_status s = btx_lb_loss_workspace_size(desc, &need);
+  if (s != BTX_OK) return s;
+  if (need > (size_t)BTX_LB_NOALLOC_SCRATCH_BYTES) return BTX_ERR_WORKSPACE;   // beyond the static array
+  void* scratch = nullptr;
+  if ((s = lb_noalloc_scratch(&scratch)) != BTX_OK) return s;
+  // btx_lb_loss clears the status block at the head of the scratch and overwrites every other
+  // region before reading it, so stale contents of an earlier call are harmless.
+  return btx_lb_loss(desc, logits, loss, u, p, dlogits, scratch, BTX_LB_NOALLOC_SCRATCH_BYTES, stream);
 }
 
 extern "C" btx_status btx_device_status(const void* workspace, void* stream, int32_t* device_status) {
