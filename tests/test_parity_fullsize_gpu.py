@@ -1,0 +1,115 @@
+"""Parity at the benchmark's full sizes (Llama-2-7B-shaped layer: d_model 4096, d_ff 11008, 4 experts),
+in the launch configuration bench.py times.  Routing, counts and the permutation are compared in full
+and bit-exactly (oracle fed the GPU's fp32 logits); floating-point outputs are compared on sampled
+tokens (y, dx) and sampled hidden units (dW1, dW3, dW2), which the oracle computes one by one, plus
+properties that hold at any size (router-gradient rows sum to zero)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import btx_oracle as o
+from paper_2403_07816_b200 import binding as B
+from paper_2403_07816_b200 import synth
+from util import gpu_backward, gpu_forward, np64, rel_err
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+D, F, E = 4096, 11008, 4
+TOL = 1e-2
+ALPHA = 0.01
+
+
+def full_size_case(T, k, seed, routing=B.ROUTE_TOPK, bias=None, backward=True, n_tok=192, n_hidden=24):
+    inp = synth.moe_inputs(T, D, F, E, seed, torch.bfloat16, DEV, with_dy=backward)
+    fwd = gpu_forward(inp, k, routing, ALPHA, bias, save=backward)
+    r = fwd["routing"]
+    kk = E if routing == B.ROUTE_SOFT else k
+    cpu = {n: np64(t) for n, t in inp.items()}
+    b64 = None if bias is None else np64(bias)
+    rng = np.random.default_rng(seed)
+    tok = np.sort(rng.choice(T, size=min(n_tok, T), replace=False))
+
+    # routing: full size, bit-exact on the GPU's logits
+    z_gpu = r.logits.cpu().numpy()
+    assert rel_err(z_gpu, o.router_logits(cpu["x"], cpu["w_router"], b64)) <= TOL
+    z, idx, g, p_tok = o.route(cpu["x"], cpu["w_router"], kk, routing, b64, logits=z_gpu)
+    assert np.array_equal(r.topk_idx.cpu().numpy(), idx)
+    counts, offsets, perm, inv_perm = o.dispatch(idx, E)
+    for name, want in [("counts", counts), ("offsets", offsets), ("perm", perm), ("inv_perm", inv_perm)]:
+        assert np.array_equal(getattr(r, name).cpu().numpy(), want), name
+    assert rel_err(r.gates.cpu().numpy(), g) <= 1e-5 and rel_err(r.probs.cpu().numpy(), p_tok) <= 1e-5
+    loss, u, p = o.lb_loss(o.dense_gates(idx, g, E), p_tok, ALPHA)
+    assert abs(r.lb_loss.item() - loss) <= 1e-5 * loss
+    assert rel_err(r.u.cpu().numpy(), u) <= 1e-5 and rel_err(r.p.cpu().numpy(), p) <= 1e-5
+
+    # y on sampled tokens
+    ref = o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], kk, routing, ALPHA,
+                        router_bias=b64, logits=z_gpu, tokens=tok)
+    y = np64(fwd["y"])
+    assert np.all(np.isfinite(y))
+    e_y = np.max(np.abs(y[tok] - ref["y"])) / np.max(np.abs(ref["y"]))
+    assert e_y <= TOL, f"y {e_y}"
+    if not backward:
+        return counts
+    got = gpu_backward(inp, fwd, 1.0, bias)
+    sl = o.moe_backward_token_slice(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], cpu["dy"], idx, g,
+                                    p_tok, u, p, tok, routing, ALPHA, 1.0, False)
+    dx = np64(got["dx"])
+    assert np.all(np.isfinite(dx))
+    e_dx = np.max(np.abs(dx[tok] - sl["dx"])) / np.max(np.abs(sl["dx"]))
+    assert e_dx <= TOL, f"dx {e_dx}"
+    # weight gradients on sampled hidden units, over all tokens of the expert
+    for e in range(E):
+        J = np.sort(rng.choice(F, size=n_hidden, replace=False))
+        d1, d3, d2 = o.expert_wgrad_hidden_slice(cpu["x"], cpu["w1"], cpu["w3"], cpu["w2"], cpu["dy"], idx, g, e, J)
+        Jt = torch.from_numpy(J).to(DEV)
+        for name, want, have in [("dw1", d1, got["dw1"][e][Jt]), ("dw3", d3, got["dw3"][e][Jt]),
+                                 ("dw2", d2, got["dw2"][e][:, Jt])]:
+            if np.max(np.abs(want)) == 0:
+                assert float(have.abs().max()) == 0.0
+                continue
+            err = rel_err(np64(have), want)
+            assert err <= TOL, f"{name}[{e}] {err}"
+    # properties at full size: every softmax Jacobian is shift invariant
+    dwr = np64(got["dw_router"])
+    assert np.all(np.isfinite(dwr))
+    assert np.max(np.abs(dwr.sum(axis=0))) <= 1e-3 * np.max(np.abs(dwr))
+    assert abs(np64(got["dbias"]).sum()) <= 1e-3 * np.max(np.abs(np64(got["dbias"]))) + 1e-6
+    for n in ("dw1", "dw3", "dw2"):
+        assert bool(torch.isfinite(got[n]).all()), n
+    return counts
+
+
+def test_forward_T4096_seed1():
+    full_size_case(4096, 2, seed=1, backward=False)
+
+
+def test_forward_backward_T16384_seed2():
+    counts = full_size_case(16384, 2, seed=2)
+    assert counts.min() > 0.2 * 32768 and counts.max() < 0.3 * 32768      # roughly uniform loads
+
+
+def test_switch_top1_T16384_seed3():
+    full_size_case(16384, 1, seed=3, routing=B.ROUTE_SWITCH, n_tok=128, n_hidden=16)
+
+
+def test_soft_routing_T16384_seed3():
+    full_size_case(16384, 4, seed=3, routing=B.ROUTE_SOFT, n_tok=96, n_hidden=12)
+
+
+def test_skewed_top2_T16384_seed3():
+    bias = synth.skew_bias(E, DEV)
+    counts = full_size_case(16384, 2, seed=3, bias=bias, n_tok=128, n_hidden=16)
+    assert counts[0] > 0.4 * 32768                                        # expert 0 takes the largest share
+
+
+def test_decode_shaped_T32_two_layers_seed4():
+    for layer in range(2):
+        inp = synth.moe_inputs(32, D, F, E, 4, torch.bfloat16, DEV, layer=layer, with_dy=False)
+        fwd = gpu_forward(inp, 2, save=False)
+        cpu = {n: np64(t) for n, t in inp.items()}
+        z_gpu = fwd["routing"].logits.cpu().numpy()
+        ref = o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], 2, alpha=ALPHA, logits=z_gpu)
+        assert np.array_equal(fwd["routing"].topk_idx.cpu().numpy(), ref["topk_idx"])
+        assert np.array_equal(fwd["routing"].perm.cpu().numpy(), ref["perm"])
+        assert rel_err(np64(fwd["y"]), ref["y"]) <= TOL
