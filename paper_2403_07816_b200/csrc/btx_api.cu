@@ -32,7 +32,7 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   p.esize = desc->dtype == BTX_BF16 ? 2 : 4;
   p.r_pad_max = (int)align_up((size_t)p.R + (size_t)p.E * (kRowTile - 1), kRowTile);
   p.mt_max = p.r_pad_max / kRowTile;
-  p.nt_dact = desc->dtype == BTX_BF16 ? (p.F + 255) / 256 : (p.F + 63) / 64;
+  p.nt_dact = desc->dtype == BTX_BF16 ? 2 * ((p.F + 255) / 256) : (p.F + 63) / 64;   // row-dot partials per row
   p.route_blocks = (p.T + 7) / 8;
   if (p.route_blocks > 148 * 8) p.route_blocks = 148 * 8;
   p.perm_blocks = (p.R + 1023) / 1024;

@@ -10,7 +10,7 @@
 
 namespace btx {
 
-constexpr int kRowTile = 128;        // expert segments of the sorted buffers are padded to this many rows
+constexpr int kRowTile = 256;        // expert segments of the sorted buffers are padded to this many rows
 constexpr int kMaxExperts = 32;
 constexpr int kStatusWords = 64;     // first 256 bytes of every workspace: device status block
 

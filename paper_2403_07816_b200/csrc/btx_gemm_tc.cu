@@ -1,13 +1,21 @@
 // BF16 expert GEMMs on the 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM,
 // operands staged in shared memory by TMA), one persistent warp-specialised kernel template.
 //
-//   warp 0      TMA producer: fills a 4-stage ring of (A 128x64, B 256x64) bf16 tiles
-//   warp 1      allocates TMEM, issues tcgen05.mma (one lane), commits to mbarriers
-//   warps 2-5   epilogue: tcgen05.ld of a 128x256 fp32 accumulator (one row per thread),
-//               fused element-wise work, stores.  Two accumulators (2 x 256 TMEM columns)
-//               let the epilogue of tile i overlap the main loop of tile i+1.
+// Two CTAs on neighbouring SMs form a cluster and work on one 256 x 256 output tile with
+// tcgen05.mma.cta_group::2: each CTA stages its own 128 rows of A and one half (128 of the 256
+// columns) of B, so shared-memory fill and operand-read traffic per SM is two thirds of what a
+// single-CTA 128 x 256 tile needs, and each CTA keeps a 128 x 256 fp32 accumulator in its TMEM.
 //
-// Modes (all grouped by expert through the 128-row padded sorted layout):
+//   warp 0      TMA producer (one lane): fills a 6-stage ring of (A 128x64, B 128x64) bf16 tiles;
+//               both CTAs signal the leader CTA's "full" barrier
+//   warp 1      allocates TMEM; in the leader CTA one lane issues the MMAs for the pair and
+//               commits (multicast) to the barriers of both CTAs
+//   warps 2-9   epilogue: tcgen05.ld of the CTA's accumulator (one row per thread, two warps per
+//               32-row TMEM quarter, each taking half of the columns), fused element-wise work,
+//               stores.  Two accumulators (2 x 256 TMEM columns) let the epilogue of tile i
+//               overlap the main loop of tile i+1.
+//
+// Modes (all grouped by expert through the 256-row padded sorted layout):
 //   FWD1   [h1|h3] = Xs [W1;W3]^T, epilogue a = silu(h1)*h3        (Section 3.2, FF_i)
 //   FWD2   rows   = a W2^T, epilogue gate scale + scatter to t*k+slot rows
 //   DACT   dA'    = dYs W2, epilogue SwiGLU backward, g*a, row-dot <dA', a> (d gate)
@@ -17,7 +25,9 @@
 // operands in WGRAD) are fed as MN-major shared-memory tiles, so nothing is ever transposed.
 //
 // Every mbarrier wait is bounded: after about two seconds it records BTX_ERR_TIMEOUT in the
-// workspace status word, raises a CTA-wide abort flag and the kernel drains and returns.
+// workspace status word, raises a CTA-wide abort flag and the kernel drains and returns.  Both
+// CTAs always meet at a cluster barrier before they exit, so no remote arrival can target a CTA
+// that has already left.
 #include <cuda.h>
 
 #include "btx_common.cuh"
@@ -25,20 +35,23 @@
 namespace btx {
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int BM = 128;                                  // rows per CTA; the pair covers 2*BM = kRowTile
+constexpr int BN = 256, BK = 64, STAGES = 6;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / 2) * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int CHUNK_BYTES = 64 * BK * 2;                 // one 64x64 MN-major box
-constexpr int TC_THREADS = 192;
+constexpr int EPI_WARPS = 8;
+constexpr int TC_THREADS = 64 + EPI_WARPS * 32;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 constexpr int GROUP_N = 8;                               // column tiles per raster group
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+static_assert(2 * BM == kRowTile, "a CTA pair covers one padded row tile");
 
 enum TcMode { G_FWD1 = 0, G_FWD2 = 1, G_DACT = 2, G_DX = 3, G_WGRAD = 4 };
 
 struct TcParams {
   int d, F, E, r_pad_max;
   int n_tiles;                  // column tiles
-  int m_tiles;                  // WGRAD: row tiles per expert
+  int m_tiles;                  // WGRAD: 256-row tiles per expert
   int kb_total;                 // K blocks per tile (grouped modes)
   int kb_half;                  // DX: K blocks of the first operand pair
   int M, N;                     // output rows per expert (WGRAD) / columns
@@ -62,14 +75,31 @@ struct TcParams {
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+// arrive on a barrier that may live in the other CTA of the cluster
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -102,27 +132,35 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// TMA tile loads of one CTA of a pair; the completion bytes go to `bar`, a shared::cluster address
+// that may name the leader CTA's barrier.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// arrive (once the MMAs issued so far have retired) on the barrier at this offset in both CTAs
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)3) : "memory");
 }
-__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accum) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
@@ -170,9 +208,10 @@ __device__ __forceinline__ void unpack8(uint4 q, float* v) {
 
 // ---------------------------------------------------------------------------------------------
 // Tile schedule: the same function is evaluated by the producer, the MMA issuer and the epilogue
+// of both CTAs.  A tile is 256 output rows (128 per CTA) by 256 columns.
 // ---------------------------------------------------------------------------------------------
 struct Tile {
-  int m0;        // first output row (padded sorted row, or row of the weight gradient)
+  int m0;        // first output row of the pair's tile
   int nt;        // column tile index
   int e;         // expert
   int k_base;    // WGRAD: first contraction row
@@ -182,7 +221,7 @@ struct Tile {
 template <int MODE>
 __device__ __forceinline__ int total_tiles(const TcParams& p) {
   if (MODE == G_WGRAD) return p.E * p.m_tiles * p.n_tiles;
-  return (p.pad_offsets[p.E] / BM) * p.n_tiles;
+  return (p.pad_offsets[p.E] / kRowTile) * p.n_tiles;
 }
 
 template <int MODE>
@@ -194,7 +233,7 @@ __device__ __forceinline__ Tile get_tile(const TcParams& p, int t) {
     tl.e = t / (p.m_tiles * p.n_tiles);
     local = t - tl.e * p.m_tiles * p.n_tiles;
   } else {
-    mt_count = p.pad_offsets[p.E] / BM;
+    mt_count = p.pad_offsets[p.E] / kRowTile;
   }
   // raster: groups of GROUP_N column tiles; inside a group rows advance slowest
   const int full = p.n_tiles / GROUP_N;
@@ -204,7 +243,7 @@ __device__ __forceinline__ Tile get_tile(const TcParams& p, int t) {
   else { g = full; rem = local - in_full; width = p.n_tiles - full * GROUP_N; }
   const int mt = rem / width;
   tl.nt = g * GROUP_N + rem - mt * width;
-  tl.m0 = mt * BM;
+  tl.m0 = mt * kRowTile;
   if (MODE == G_WGRAD) {
     tl.k_base = p.pad_offsets[tl.e];
     tl.kb = (p.pad_offsets[tl.e + 1] - tl.k_base) / BK;
@@ -220,7 +259,7 @@ __device__ __forceinline__ Tile get_tile(const TcParams& p, int t) {
 // The kernel
 // ---------------------------------------------------------------------------------------------
 template <int MODE>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
                const TcParams p) {
@@ -228,83 +267,102 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;                        // 1024-byte aligned ring
   uint8_t* ctl = smem_raw + (tiles - raw) + STAGES * STAGE_BYTES;       // barriers behind the ring
-  const uint32_t bar_full = smem_u32(ctl);                              // STAGES x 8 B
-  const uint32_t bar_empty = bar_full + STAGES * 8;
-  const uint32_t bar_tfull = bar_empty + STAGES * 8;                    // 2 x 8 B
-  const uint32_t bar_tempty = bar_tfull + 16;
+  const uint32_t bar_full = smem_u32(ctl);                              // STAGES x 8 B (used in the leader)
+  const uint32_t bar_empty = bar_full + STAGES * 8;                     // STAGES x 8 B (each CTA its own)
+  const uint32_t bar_tfull = bar_empty + STAGES * 8;                    // 2 x 8 B (each CTA its own)
+  const uint32_t bar_tempty = bar_tfull + 16;                           // 2 x 8 B (used in the leader)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + STAGES * 16 + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + STAGES * 16 + 40);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();                              // 0 = leader of the pair
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   constexpr bool A_MN = (MODE == G_WGRAD);
   constexpr bool B_MN = (MODE == G_DACT || MODE == G_DX || MODE == G_WGRAD);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + s * 8, 1); mbar_init(bar_empty + s * 8, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + a * 8, 1); mbar_init(bar_tempty + a * 8, 128); }
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + a * 8, 1); mbar_init(bar_tempty + a * 8, 2 * EPI_WARPS * 32); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();                                     // the peer's barriers exist before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int n_total = total_tiles<MODE>(p);
 
   if (warp == 0) {
-    // ------------------------------- TMA producer -------------------------------
+    // ------------------------------- TMA producer (both CTAs) -------------------------------
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
+      uint32_t uses = 0;                                  // stages filled so far (for the final drain)
       bool ok = true;
-      for (int t = blockIdx.x; t < n_total && ok; t += gridDim.x) {
+      for (int t = pair; t < n_total && ok; t += n_pairs) {
         const Tile tl = get_tile<MODE>(p, t);
+        const int m0 = tl.m0 + (int)rank * BM;            // this CTA's rows
         for (int kb = 0; kb < tl.kb; ++kb) {
           if (!(ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status))) break;
-          const uint32_t full = bar_full + stage * 8;
+          const uint32_t full_local = bar_full + stage * 8;
+          const uint32_t full = map_to_cta(full_local, 0);                 // the leader collects both CTAs' bytes
           const uint32_t sA = tiles + stage * STAGE_BYTES, sB = sA + A_BYTES;
-          mbar_expect_tx(full, STAGE_BYTES);
+          if (rank == 0) mbar_expect_tx(full_local, 2 * STAGE_BYTES);
           if (MODE == G_FWD1) {
-            tma_load_2d(sA, &tmA0, kb * BK, tl.m0, full);
-            tma_load_3d(sB, &tmB0, kb * BK, tl.nt * 128, tl.e, full);
-            tma_load_3d(sB + B_BYTES / 2, &tmB1, kb * BK, tl.nt * 128, tl.e, full);
+            // B tile = [128 rows of W1 | 128 rows of W3]: the leader stages W1, its peer W3
+            tma_load_2d(sA, &tmA0, kb * BK, m0, full);
+            tma_load_3d(sB, rank == 0 ? &tmB0 : &tmB1, kb * BK, tl.nt * 128, tl.e, full);
           } else if (MODE == G_FWD2) {
-            tma_load_2d(sA, &tmA0, kb * BK, tl.m0, full);
-            tma_load_3d(sB, &tmB0, kb * BK, tl.nt * BN, tl.e, full);
+            tma_load_2d(sA, &tmA0, kb * BK, m0, full);
+            tma_load_3d(sB, &tmB0, kb * BK, tl.nt * BN + (int)rank * 128, tl.e, full);
           } else if (MODE == G_DACT) {
-            tma_load_2d(sA, &tmA0, kb * BK, tl.m0, full);
+            tma_load_2d(sA, &tmA0, kb * BK, m0, full);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) tma_load_3d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + j * 64, kb * BK, tl.e, full);
+            for (int j = 0; j < 2; ++j)
+              tma_load_3d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + ((int)rank * 2 + j) * 64, kb * BK, tl.e, full);
           } else if (MODE == G_DX) {
             const bool second = kb >= p.kb_half;
             const int kk = (second ? kb - p.kb_half : kb) * BK;
-            tma_load_2d(sA, second ? &tmA1 : &tmA0, kk, tl.m0, full);
+            tma_load_2d(sA, second ? &tmA1 : &tmA0, kk, m0, full);
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              tma_load_3d(sB + j * CHUNK_BYTES, second ? &tmB1 : &tmB0, tl.nt * BN + j * 64, kk, tl.e, full);
+            for (int j = 0; j < 2; ++j)
+              tma_load_3d(sB + j * CHUNK_BYTES, second ? &tmB1 : &tmB0, tl.nt * BN + ((int)rank * 2 + j) * 64, kk, tl.e,
+                          full);
           } else {
             const int row = tl.k_base + kb * BK;
 #pragma unroll
-            for (int j = 0; j < 2; ++j) tma_load_2d(sA + j * CHUNK_BYTES, &tmA0, tl.m0 + j * 64, row, full);
+            for (int j = 0; j < 2; ++j) tma_load_2d(sA + j * CHUNK_BYTES, &tmA0, m0 + j * 64, row, full);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) tma_load_2d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + j * 64, row, full);
+            for (int j = 0; j < 2; ++j)
+              tma_load_2d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + ((int)rank * 2 + j) * 64, row, full);
           }
+          ++uses;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
+      // Drain: wait until the MMAs that read this CTA's last stages have retired, i.e. until every
+      // commit addressed to this CTA's "empty" barriers has landed.
+      // (a slot that was never filled passes at once)
+      (void)uses;
+      for (int i = 0; i < STAGES && ok; ++i) {
+        ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status);
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
     }
   } else if (warp == 1) {
-    // ------------------------------- MMA issuer -------------------------------
-    if (lane == 0) {
+    // ------------------------------- MMA issuer (leader CTA only) -------------------------------
+    if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
-                                 ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                                 ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) |
+                                 ((uint32_t)((2 * BM) >> 4) << 24);
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < n_total && ok; t += gridDim.x) {
+      for (int t = pair; t < n_total && ok; t += n_pairs) {
         const Tile tl = get_tile<MODE>(p, t);
         if (tl.kb == 0) continue;
         if (!(ok = mbar_wait(bar_tempty + acc * 8, acc_phase ^ 1u, abort_flag, p.status))) break;
@@ -320,24 +378,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             // advance 16 contraction elements: 32 B inside a K-major row, 16 rows (2048 B) MN-major
             const uint64_t ao = (uint64_t)((A_MN ? 2048 : 32) * k16 >> 4);
             const uint64_t bo = (uint64_t)((B_MN ? 2048 : 32) * k16 >> 4);
-            tc_mma(tmem_d, da + ao, db + bo, idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+            tc_mma_pair(tmem_d, da + ao, db + bo, idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
           }
-          tc_commit(bar_empty + stage * 8);              // frees the stage when these MMAs retire
+          tc_commit_pair(bar_empty + stage * 8);         // frees the stage in both CTAs when these MMAs retire
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        tc_commit(bar_tfull + acc * 8);
+        tc_commit_pair(bar_tfull + acc * 8);
         acc ^= 1u;
         if (acc == 0) acc_phase ^= 1u;
       }
     }
   } else {
-    // ------------------------------- epilogue -------------------------------
+    // ------------------------------- epilogue (both CTAs) -------------------------------
     const int q = warp & 3;                               // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;                     // which half of the accumulator columns
     const int row = q * 32 + lane;
+    const uint32_t tempty_leader = map_to_cta(bar_tempty, 0);
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < n_total && ok; t += gridDim.x) {
+    for (int t = pair; t < n_total && ok; t += n_pairs) {
       const Tile tl = get_tile<MODE>(p, t);
       const bool have_acc = tl.kb > 0;
       if (have_acc) {
@@ -345,13 +405,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         tc_fence_after();
       }
       const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
-      const int rp = tl.m0 + row;
+      const int rp = tl.m0 + (int)rank * BM + row;
       float v[32];
 
       if (MODE == G_FWD1) {
         float w[32], a[8];
         const int F = p.F;
-        for (int c = 0; c < 128; c += 32) {
+        for (int c = half * 64; c < half * 64 + 64; c += 32) {
           tc_ld32(taddr + c, v);
           tc_ld32(taddr + 128 + c, w);
           const int col = tl.nt * 128 + c;
@@ -373,7 +433,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         const int flat = p.rowmap[rp];
         const float g = (MODE == G_FWD2 && flat >= 0) ? p.gates[flat] : 1.0f;
         const int N = p.N;
-        for (int c = 0; c < BN; c += 32) {
+        for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
           tc_ld32(taddr + c, v);                          // all lanes take part in the load
           const int col = tl.nt * BN + c;
           if (flat >= 0) {
@@ -390,16 +450,27 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         const float g = flat >= 0 ? p.gates[flat] : 0.f;
         const int F = p.F;
         float rowdot = 0.f;
-        for (int c = 0; c < BN; c += 32) {
-          tc_ld32(taddr + c, v);
+        for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
           const int col = tl.nt * BN + c;
+          // fetch the saved pre-activations of this chunk before touching TMEM: the loads are
+          // independent of the accumulator and would otherwise serialise behind the stores
+          uint4 q1[4], q3[4];
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            if (col + g8 * 8 < F) {
+              const size_t o = (size_t)rp * F + col + g8 * 8;
+              q1[g8] = *reinterpret_cast<const uint4*>(p.h1 + o);
+              q3[g8] = *reinterpret_cast<const uint4*>(p.h3 + o);
+            }
+          }
+          tc_ld32(taddr + c, v);
 #pragma unroll
           for (int g8 = 0; g8 < 4; ++g8) {
             if (col + g8 * 8 < F) {
               const size_t o = (size_t)rp * F + col + g8 * 8;
               float h1[8], h3[8], d1[8], d3[8], ga[8];
-              unpack8(*reinterpret_cast<const uint4*>(p.h1 + o), h1);
-              unpack8(*reinterpret_cast<const uint4*>(p.h3 + o), h3);
+              unpack8(q1[g8], h1);
+              unpack8(q3[g8], h3);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 const float da = v[g8 * 8 + i];
@@ -414,11 +485,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             }
           }
         }
-        p.dg_part[(size_t)tl.nt * p.r_pad_max + rp] = rowdot;
+        p.dg_part[(size_t)(tl.nt * 2 + half) * p.r_pad_max + rp] = rowdot;
       } else {  // WGRAD
         const int N = p.N;
         const bool row_ok = rp < p.M;
-        for (int c = 0; c < BN; c += 32) {
+        for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
           if (have_acc) tc_ld32(taddr + c, v);
           else {
 #pragma unroll
@@ -443,18 +514,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       }
       if (have_acc) {
         tc_fence_before();
-        mbar_arrive(bar_tempty + acc * 8);
+        mbar_arrive_cluster(tempty_leader + acc * 8);     // the leader's MMA issuer waits for both CTAs
         acc ^= 1u;
         if (acc == 0) acc_phase ^= 1u;
       }
     }
   }
 
+  // Nobody leaves before both CTAs are done: remote arrivals and multicast commits must find
+  // their target barriers alive.
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
   }
 }
 
@@ -508,10 +582,10 @@ btx_status launch_tc(const CUtensorMap& a0, const CUtensorMap& a1, const CUtenso
                      const TcParams& p, int max_tiles, cudaStream_t st) {
   if (cudaFuncSetAttribute(tc_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
     return BTX_ERR_CUDA;
-  int grid = sm_count();
-  if (grid > max_tiles) grid = max_tiles;
-  if (grid < 1) grid = 1;
-  tc_gemm_kernel<MODE><<<grid, TC_THREADS, SMEM_BYTES, st>>>(a0, a1, b0, b1, p);
+  int pairs = sm_count() / 2;
+  if (pairs > max_tiles) pairs = max_tiles;
+  if (pairs < 1) pairs = 1;
+  tc_gemm_kernel<MODE><<<2 * pairs, TC_THREADS, SMEM_BYTES, st>>>(a0, a1, b0, b1, p);   // cluster dims are compiled in
   return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
 }
 
@@ -540,7 +614,7 @@ btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void
   if ((s = launch_tc<G_FWD1>(a, a, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(2, st);
   // GEMM-2: gate-scaled expert rows = act W2^T
-  if (!make_map(&a, b.act, F, RP, 0, 64, 128) || !make_map(&b0, w2, F, d, E, 64, 256)) return BTX_ERR_CUDA;
+  if (!make_map(&a, b.act, F, RP, 0, 64, 128) || !make_map(&b0, w2, F, d, E, 64, 128)) return BTX_ERR_CUDA;
   p.n_tiles = (pl.d + BN - 1) / BN; p.kb_total = (pl.F + BK - 1) / BK; p.N = pl.d; p.of = b.yp;
   return launch_tc<G_FWD2>(a, a, b0, b0, p, pl.mt_max * p.n_tiles, st);
 }
@@ -570,13 +644,13 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   // wgrads: contraction over the expert's padded token rows, both operands MN-major
   p.accumulate = accumulate;
   if (!make_map(&a0, b.dys, d, RP, 0, 64, 64) || !make_map(&b0, b.ga, F, RP, 0, 64, 64)) return BTX_ERR_CUDA;
-  p.M = pl.d; p.N = pl.F; p.m_tiles = (pl.d + BM - 1) / BM; p.n_tiles = (pl.F + BN - 1) / BN; p.of = dw2;
+  p.M = pl.d; p.N = pl.F; p.m_tiles = (pl.d + kRowTile - 1) / kRowTile; p.n_tiles = (pl.F + BN - 1) / BN; p.of = dw2;
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(4, st);
   if (!make_map(&a0, b.dh1, F, RP, 0, 64, 64) || !make_map(&a1, b.dh3, F, RP, 0, 64, 64) ||
       !make_map(&b0, b.xs, d, RP, 0, 64, 64))
     return BTX_ERR_CUDA;
-  p.M = pl.F; p.N = pl.d; p.m_tiles = (pl.F + BM - 1) / BM; p.n_tiles = (pl.d + BN - 1) / BN; p.of = dw1;
+  p.M = pl.F; p.N = pl.d; p.m_tiles = (pl.F + kRowTile - 1) / kRowTile; p.n_tiles = (pl.d + BN - 1) / BN; p.of = dw1;
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(5, st);
   p.of = dw3;

@@ -143,19 +143,26 @@ router_kernel(int Tn, int d, int E, int k, int routing, const T* __restrict__ x,
   }
 }
 
-__global__ void lb_finalize_kernel(int Tn, int E, int nblocks, float alpha, const float* __restrict__ route_part,
-                                   float* __restrict__ u, float* __restrict__ p, float* __restrict__ loss) {
+// One warp per (expert, u|p) pair: lanes sum strided block partials in double, then a fixed-order
+// shuffle tree, so the result does not depend on scheduling.
+__global__ void __launch_bounds__(256)
+lb_finalize_kernel(int Tn, int E, int nblocks, float alpha, const float* __restrict__ route_part,
+                   float* __restrict__ u, float* __restrict__ p, float* __restrict__ loss) {
   __shared__ double su[kMaxExperts], sp[kMaxExperts];
-  int tid = threadIdx.x;
-  if (tid < 2 * E) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int pair = warp; pair < 2 * E; pair += 8) {
     double s = 0.0;
-    for (int b = 0; b < nblocks; ++b) s += (double)route_part[(size_t)b * 2 * E + tid];
+    for (int b = lane; b < nblocks; b += 32) s += (double)route_part[(size_t)b * 2 * E + pair];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     s /= (double)Tn;
-    if (tid & 1) { sp[tid >> 1] = s; p[tid >> 1] = (float)s; }
-    else { su[tid >> 1] = s; u[tid >> 1] = (float)s; }
+    if (lane == 0) {
+      if (pair & 1) { sp[pair >> 1] = s; p[pair >> 1] = (float)s; }
+      else { su[pair >> 1] = s; u[pair >> 1] = (float)s; }
+    }
   }
   __syncthreads();
-  if (tid == 0) {
+  if (threadIdx.x == 0) {
     double acc = 0.0;
     for (int e = 0; e < E; ++e) acc += su[e] * sp[e];
     loss[0] = (float)((double)alpha * (double)E * acc);
@@ -432,7 +439,7 @@ cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, c
         pl.T, pl.d, pl.E, pl.k, routing, (const float*)x, (const float*)w_router, bias, given_logits, b.logits,
         b.topk, b.gates, b.probs, b.route_part);
   }
-  lb_finalize_kernel<<<1, 64, 0, st>>>(pl.T, pl.E, pl.route_blocks, alpha, b.route_part, b.u, b.p, b.loss);
+  lb_finalize_kernel<<<1, 256, 0, st>>>(pl.T, pl.E, pl.route_blocks, alpha, b.route_part, b.u, b.p, b.loss);
   return cudaGetLastError();
 }
 
