@@ -97,17 +97,21 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// arrive on a barrier that may live in the other CTA of the cluster
+// Arrive on a barrier that may live in the other CTA of the cluster.  Relaxed: the arrival only
+// hands a drained TMEM accumulator back (ordered by tcgen05.fence::before_thread_sync); it must not
+// wait for this thread's outstanding global stores the way a releasing arrival would.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// One poll of the barrier.  The hint lets the hardware park the thread (up to about 10 us) until
+// the phase completes instead of spinning on shared memory.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(10000u) : "memory");
   return ok != 0;
 }
 __device__ __forceinline__ unsigned long long global_ns() {
@@ -121,7 +125,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 0u) {
+    if ((it & 15u) == 0u) {
       if (*abort_flag) return false;
       if (global_ns() - t0 > kWaitLimitNs) {
         *abort_flag = 1;
@@ -190,6 +194,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
   dsc |= 2ull << 61;                                      // 128-byte swizzle
   return dsc;
 }
+
+// SwiGLU pieces for the BF16 epilogues: sigmoid from one ex2 and one reciprocal approximation
+// (relative error about 2^-21, far below bf16 rounding).
+__device__ __forceinline__ float fast_sigmoid(float v) { return __frcp_rn(1.0f + __expf(-v)); }
+__device__ __forceinline__ float fast_swiglu(float h1, float h3) { return h1 * fast_sigmoid(h1) * h3; }
 
 __device__ __forceinline__ uint4 pack8(const float* v) {
   __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
@@ -419,7 +428,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           for (int g8 = 0; g8 < 4; ++g8) {
             if (col + g8 * 8 < F) {
 #pragma unroll
-              for (int i = 0; i < 8; ++i) a[i] = swiglu_f32(v[g8 * 8 + i], w[g8 * 8 + i]);
+              for (int i = 0; i < 8; ++i) a[i] = fast_swiglu(v[g8 * 8 + i], w[g8 * 8 + i]);
               const size_t o = (size_t)rp * F + col + g8 * 8;
               *reinterpret_cast<uint4*>(p.o0 + o) = pack8(a);
               if (p.save) {
@@ -474,8 +483,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 const float da = v[g8 * 8 + i];
-                const float a = swiglu_f32(h1[i], h3[i]);
-                swiglu_bwd_f32(h1[i], h3[i], g * da, d1[i], d3[i]);
+                const float sg = fast_sigmoid(h1[i]);
+                const float hs = h1[i] * sg;                    // silu(h1)
+                const float a = hs * h3[i];
+                const float gda = g * da;
+                d1[i] = gda * h3[i] * sg * (1.0f + h1[i] * (1.0f - sg));
+                d3[i] = gda * hs;
                 ga[i] = g * a;
                 rowdot = fmaf(da, a, rowdot);
               }
