@@ -12,7 +12,8 @@
 //               commits (multicast) to the barriers of both CTAs
 //   warps 2-9   epilogue: tcgen05.ld of the CTA's accumulator (one row per thread, two warps per
 //               32-row TMEM quarter, each taking half of the columns), fused element-wise work,
-//               stores.  Two accumulators (2 x 256 TMEM columns) let the epilogue of tile i
+//               stores staged through shared memory so that global memory sees whole lines.
+//               Two accumulators (2 x 256 TMEM columns) let the epilogue of tile i
 //               overlap the main loop of tile i+1.
 //
 // Modes (all grouped by expert through the 256-row padded sorted layout):
@@ -41,7 +42,8 @@ constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / 2) * BK * 2, STAGE_BYTES = 
 constexpr int CHUNK_BYTES = 64 * BK * 2;                 // one 64x64 MN-major box
 constexpr int EPI_WARPS = 8;
 constexpr int TC_THREADS = 64 + EPI_WARPS * 32;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int STAGING_BYTES = 4096;                      // per epilogue warp: 32 rows x 128 B
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + EPI_WARPS * STAGING_BYTES;
 constexpr int GROUP_N = 8;                               // column tiles per raster group
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 static_assert(2 * BM == kRowTile, "a CTA pair covers one padded row tile");
@@ -212,6 +214,44 @@ __device__ __forceinline__ void unpack8(uint4 q, float* v) {
   for (int i = 0; i < 4; ++i) {
     float2 f = __bfloat1622float2(h[i]);
     v[2 * i] = f.x; v[2 * i + 1] = f.y;
+  }
+}
+
+// Staging block addressing (bytes).  Rows of 64 B (32 bf16) or 128 B (32 fp32); the 16-byte piece
+// index is XOR-swizzled with the row so that both the row-wise accesses (lane = row) and the
+// line-wise accesses (8 or 4 rows per instruction) are free of bank conflicts.
+__device__ __forceinline__ uint32_t sw64(int r, int j) { return (uint32_t)(r * 64 + ((j ^ ((r >> 1) & 3)) << 4)); }
+__device__ __forceinline__ uint32_t sw128(int r, int j) { return (uint32_t)(r * 128 + ((j ^ (r & 7)) << 4)); }
+
+// lane = row: put this lane's 32 values into the block
+__device__ __forceinline__ void stage_row_bf16(uint8_t* buf, int lane, const float* v) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(buf + sw64(lane, j)) = pack8(v + j * 8);
+}
+__device__ __forceinline__ void stage_row_f32(uint8_t* buf, int lane, const float* v) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    *reinterpret_cast<float4*>(buf + sw128(lane, j)) = make_float4(v[j * 4], v[j * 4 + 1], v[j * 4 + 2], v[j * 4 + 3]);
+}
+__device__ __forceinline__ void unstage_row_bf16(const uint8_t* buf, int lane, float* v) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) unpack8(*reinterpret_cast<const uint4*>(buf + sw64(lane, j)), v + j * 8);
+}
+// 32 x 32 bf16 block <-> global rows of `ld` elements starting at g; cv = valid columns (multiple of 8)
+__device__ __forceinline__ void flush_bf16(const uint8_t* buf, int lane, __nv_bfloat16* g, size_t ld, int cv) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = i * 8 + (lane >> 2), j = lane & 3;
+    if (j * 8 < cv) *reinterpret_cast<uint4*>(g + (size_t)r * ld + j * 8) = *reinterpret_cast<const uint4*>(buf + sw64(r, j));
+  }
+}
+__device__ __forceinline__ void fetch_bf16(uint8_t* buf, int lane, const __nv_bfloat16* g, size_t ld, int cv) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = i * 8 + (lane >> 2), j = lane & 3;
+    uint4 x = make_uint4(0, 0, 0, 0);
+    if (j * 8 < cv) x = *reinterpret_cast<const uint4*>(g + (size_t)r * ld + j * 8);
+    *reinterpret_cast<uint4*>(buf + sw64(r, j)) = x;
   }
 }
 
@@ -404,6 +444,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     const int half = (warp - 2) >> 2;                     // which half of the accumulator columns
     const int row = q * 32 + lane;
     const uint32_t tempty_leader = map_to_cta(bar_tempty, 0);
+    uint8_t* stg = ctl + 256 + (warp - 2) * STAGING_BYTES;   // this warp's staging block
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     for (int t = pair; t < n_total && ok; t += n_pairs) {
@@ -417,25 +458,34 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       const int rp = tl.m0 + (int)rank * BM + row;
       float v[32];
 
+      // Each lane owns one accumulator row, but global memory wants whole lines: every 32-column
+      // chunk goes through this warp's 4 KB staging block in shared memory so that one store (or
+      // load) instruction of the warp covers 8 rows x 64 B (bf16) or 4 rows x 128 B (fp32).
+      const int row0 = tl.m0 + (int)rank * BM + q * 32;   // first row of this warp's 32-row block
+
       if (MODE == G_FWD1) {
-        float w[32], a[8];
+        float w[32], a[32];
         const int F = p.F;
         for (int c = half * 64; c < half * 64 + 64; c += 32) {
+          const int col = tl.nt * 128 + c;
+          const int cv = min(32, F - col);
+          if (cv <= 0) break;
           tc_ld32(taddr + c, v);
           tc_ld32(taddr + 128 + c, w);
-          const int col = tl.nt * 128 + c;
 #pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            if (col + g8 * 8 < F) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) a[i] = fast_swiglu(v[g8 * 8 + i], w[g8 * 8 + i]);
-              const size_t o = (size_t)rp * F + col + g8 * 8;
-              *reinterpret_cast<uint4*>(p.o0 + o) = pack8(a);
-              if (p.save) {
-                *reinterpret_cast<uint4*>(p.o1 + o) = pack8(v + g8 * 8);
-                *reinterpret_cast<uint4*>(p.o2 + o) = pack8(w + g8 * 8);
-              }
-            }
+          for (int i = 0; i < 32; ++i) a[i] = fast_swiglu(v[i], w[i]);
+          const size_t gofs = (size_t)row0 * F + col;
+          stage_row_bf16(stg, lane, a);
+          if (p.save) stage_row_bf16(stg + 2048, lane, v);
+          __syncwarp();
+          flush_bf16(stg, lane, p.o0 + gofs, F, cv);
+          if (p.save) flush_bf16(stg + 2048, lane, p.o1 + gofs, F, cv);
+          __syncwarp();
+          if (p.save) {
+            stage_row_bf16(stg, lane, w);
+            __syncwarp();
+            flush_bf16(stg, lane, p.o2 + gofs, F, cv);
+            __syncwarp();
           }
         }
       } else if (MODE == G_FWD2 || MODE == G_DX) {
@@ -443,16 +493,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         const float g = (MODE == G_FWD2 && flat >= 0) ? p.gates[flat] : 1.0f;
         const int N = p.N;
         for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
-          tc_ld32(taddr + c, v);                          // all lanes take part in the load
           const int col = tl.nt * BN + c;
-          if (flat >= 0) {
-            float* o = p.of + (size_t)flat * N + col;
+          const int cv = min(32, N - col);
+          if (cv <= 0) break;
+          tc_ld32(taddr + c, v);
 #pragma unroll
-            for (int g4 = 0; g4 < 8; ++g4)
-              if (col + g4 * 4 < N)
-                *reinterpret_cast<float4*>(o + g4 * 4) =
-                    make_float4(g * v[g4 * 4], g * v[g4 * 4 + 1], g * v[g4 * 4 + 2], g * v[g4 * 4 + 3]);
+          for (int i = 0; i < 32; ++i) v[i] *= g;
+          stage_row_f32(stg, lane, v);
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 4 + (lane >> 3), j = lane & 7;
+            const int rflat = __shfl_sync(0xffffffffu, flat, r);
+            if (rflat >= 0 && j * 4 < cv)
+              *reinterpret_cast<uint4*>(p.of + (size_t)rflat * N + col + j * 4) =
+                  *reinterpret_cast<const uint4*>(stg + sw128(r, j));
           }
+          __syncwarp();
         }
       } else if (MODE == G_DACT) {
         const int flat = p.rowmap[rp];
@@ -461,68 +518,69 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         float rowdot = 0.f;
         for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
           const int col = tl.nt * BN + c;
-          // fetch the saved pre-activations of this chunk before touching TMEM: the loads are
-          // independent of the accumulator and would otherwise serialise behind the stores
-          uint4 q1[4], q3[4];
-#pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            if (col + g8 * 8 < F) {
-              const size_t o = (size_t)rp * F + col + g8 * 8;
-              q1[g8] = *reinterpret_cast<const uint4*>(p.h1 + o);
-              q3[g8] = *reinterpret_cast<const uint4*>(p.h3 + o);
-            }
-          }
+          const int cv = min(32, F - col);
+          if (cv <= 0) break;
+          const size_t gofs = (size_t)row0 * F + col;
+          // saved pre-activations of the 32x32 block: coalesced loads into the staging block
+          fetch_bf16(stg, lane, p.h1 + gofs, F, cv);
+          fetch_bf16(stg + 2048, lane, p.h3 + gofs, F, cv);
           tc_ld32(taddr + c, v);
+          __syncwarp();
+          float h1[32], h3[32];
+          unstage_row_bf16(stg, lane, h1);
+          unstage_row_bf16(stg + 2048, lane, h3);
+          __syncwarp();
 #pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            if (col + g8 * 8 < F) {
-              const size_t o = (size_t)rp * F + col + g8 * 8;
-              float h1[8], h3[8], d1[8], d3[8], ga[8];
-              unpack8(q1[g8], h1);
-              unpack8(q3[g8], h3);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const float da = v[g8 * 8 + i];
-                const float sg = fast_sigmoid(h1[i]);
-                const float hs = h1[i] * sg;                    // silu(h1)
-                const float a = hs * h3[i];
-                const float gda = g * da;
-                d1[i] = gda * h3[i] * sg * (1.0f + h1[i] * (1.0f - sg));
-                d3[i] = gda * hs;
-                ga[i] = g * a;
-                rowdot = fmaf(da, a, rowdot);
-              }
-              *reinterpret_cast<uint4*>(p.o0 + o) = pack8(d1);
-              *reinterpret_cast<uint4*>(p.o1 + o) = pack8(d3);
-              *reinterpret_cast<uint4*>(p.o2 + o) = pack8(ga);
-            }
+          for (int i = 0; i < 32; ++i) {
+            const float da = v[i];
+            const float sg = fast_sigmoid(h1[i]);
+            const float hs = h1[i] * sg;                      // silu(h1)
+            const float a = hs * h3[i];
+            const float gda = g * da;
+            rowdot = (i < cv) ? fmaf(da, a, rowdot) : rowdot;
+            v[i] = g * a;                                     // g*a, reuses the accumulator registers
+            h3[i] = gda * h3[i] * sg * (1.0f + h1[i] * (1.0f - sg));   // dh1
+            h1[i] = gda * hs;                                 // dh3
           }
+          stage_row_bf16(stg, lane, h3);
+          stage_row_bf16(stg + 2048, lane, h1);
+          __syncwarp();
+          flush_bf16(stg, lane, p.o0 + gofs, F, cv);
+          flush_bf16(stg + 2048, lane, p.o1 + gofs, F, cv);
+          __syncwarp();
+          stage_row_bf16(stg, lane, v);
+          __syncwarp();
+          flush_bf16(stg, lane, p.o2 + gofs, F, cv);
+          __syncwarp();
         }
         p.dg_part[(size_t)(tl.nt * 2 + half) * p.r_pad_max + rp] = rowdot;
       } else {  // WGRAD
         const int N = p.N;
-        const bool row_ok = rp < p.M;
         for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
+          const int col = tl.nt * BN + c;
+          const int cv = min(32, N - col);
+          if (cv <= 0) break;
           if (have_acc) tc_ld32(taddr + c, v);
           else {
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = 0.f;
           }
-          const int col = tl.nt * BN + c;
-          if (row_ok) {
-            float* o = p.of + ((size_t)tl.e * p.M + rp) * N + col;
+          stage_row_f32(stg, lane, v);
+          __syncwarp();
 #pragma unroll
-            for (int g4 = 0; g4 < 8; ++g4) {
-              if (col + g4 * 4 < N) {
-                float4 r = make_float4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
-                if (p.accumulate) {
-                  const float4 old = *reinterpret_cast<const float4*>(o + g4 * 4);
-                  r.x += old.x; r.y += old.y; r.z += old.z; r.w += old.w;
-                }
-                *reinterpret_cast<float4*>(o + g4 * 4) = r;
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 4 + (lane >> 3), j = lane & 7;
+            if (row0 + r < p.M && j * 4 < cv) {
+              float* o = p.of + ((size_t)tl.e * p.M + row0 + r) * N + col + j * 4;
+              float4 x4 = *reinterpret_cast<const float4*>(stg + sw128(r, j));
+              if (p.accumulate) {
+                const float4 old = *reinterpret_cast<const float4*>(o);
+                x4.x += old.x; x4.y += old.y; x4.z += old.z; x4.w += old.w;
               }
+              *reinterpret_cast<float4*>(o) = x4;
             }
           }
+          __syncwarp();
         }
       }
       if (have_acc) {
