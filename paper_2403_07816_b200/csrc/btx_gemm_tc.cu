@@ -12,9 +12,8 @@
 //               commits (multicast) to the barriers of both CTAs
 //   warps 2-9   epilogue: tcgen05.ld of the CTA's accumulator (one row per thread, two warps per
 //               32-row TMEM quarter, each taking half of the columns), fused element-wise work,
-//               stores staged through shared memory so that global memory sees whole lines.
-//               Two accumulators (2 x 256 TMEM columns) let the epilogue of tile i
-//               overlap the main loop of tile i+1.
+//               32-byte-per-lane global stores.  Two accumulators (2 x 256 TMEM columns) let the
+//               epilogue of tile i overlap the main loop of tile i+1.
 //
 // Modes (all grouped by expert through the 256-row padded sorted layout):
 //   FWD1   [h1|h3] = Xs [W1;W3]^T, epilogue a = silu(h1)*h3        (Section 3.2, FF_i)
@@ -42,8 +41,7 @@ constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / 2) * BK * 2, STAGE_BYTES = 
 constexpr int CHUNK_BYTES = 64 * BK * 2;                 // one 64x64 MN-major box
 constexpr int EPI_WARPS = 8;
 constexpr int TC_THREADS = 64 + EPI_WARPS * 32;
-constexpr int STAGING_BYTES = 4096;                      // per epilogue warp: 32 rows x 128 B
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + EPI_WARPS * STAGING_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 constexpr int GROUP_N = 8;                               // column tiles per raster group
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 static_assert(2 * BM == kRowTile, "a CTA pair covers one padded row tile");
@@ -69,6 +67,7 @@ struct TcParams {
   float* of;
   float* dg_part;
   int save, accumulate;
+  int wide;                     // all epilogue rows start on 32-byte boundaries
   int32_t* status;
 };
 
@@ -202,6 +201,28 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
 __device__ __forceinline__ float fast_sigmoid(float v) { return __frcp_rn(1.0f + __expf(-v)); }
 __device__ __forceinline__ float fast_swiglu(float h1, float h3) { return h1 * fast_sigmoid(h1) * h3; }
 
+// Epilogue global accesses move 32 bytes per lane (a whole DRAM sector) whenever the row pitch and
+// base allow it: half-sector (16-byte) writes from 32 different rows per instruction cost far more
+// in the memory pipeline, and in power, than their byte count suggests.
+__device__ __forceinline__ void st32(void* p, uint4 a, uint4 b, bool wide, bool second = true) {
+  if (wide) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w),
+                 "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+  } else {
+    reinterpret_cast<uint4*>(p)[0] = a;
+    if (second) reinterpret_cast<uint4*>(p)[1] = b;
+  }
+}
+__device__ __forceinline__ void ld32(const void* p, uint4& a, uint4& b, bool wide, bool second = true) {
+  if (wide) {
+    asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w),
+                 "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p));
+  } else {
+    a = reinterpret_cast<const uint4*>(p)[0];
+    b = second ? reinterpret_cast<const uint4*>(p)[1] : make_uint4(0, 0, 0, 0);
+  }
+}
+__device__ __forceinline__ uint4 f4(const float* v) { return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])); }
 __device__ __forceinline__ uint4 pack8(const float* v) {
   __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
   __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), e = __floats2bfloat162_rn(v[6], v[7]);
@@ -214,44 +235,6 @@ __device__ __forceinline__ void unpack8(uint4 q, float* v) {
   for (int i = 0; i < 4; ++i) {
     float2 f = __bfloat1622float2(h[i]);
     v[2 * i] = f.x; v[2 * i + 1] = f.y;
-  }
-}
-
-// Staging block addressing (bytes).  Rows of 64 B (32 bf16) or 128 B (32 fp32); the 16-byte piece
-// index is XOR-swizzled with the row so that both the row-wise accesses (lane = row) and the
-// line-wise accesses (8 or 4 rows per instruction) are free of bank conflicts.
-__device__ __forceinline__ uint32_t sw64(int r, int j) { return (uint32_t)(r * 64 + ((j ^ ((r >> 1) & 3)) << 4)); }
-__device__ __forceinline__ uint32_t sw128(int r, int j) { return (uint32_t)(r * 128 + ((j ^ (r & 7)) << 4)); }
-
-// lane = row: put this lane's 32 values into the block
-__device__ __forceinline__ void stage_row_bf16(uint8_t* buf, int lane, const float* v) {
-#pragma unroll
-  for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(buf + sw64(lane, j)) = pack8(v + j * 8);
-}
-__device__ __forceinline__ void stage_row_f32(uint8_t* buf, int lane, const float* v) {
-#pragma unroll
-  for (int j = 0; j < 8; ++j)
-    *reinterpret_cast<float4*>(buf + sw128(lane, j)) = make_float4(v[j * 4], v[j * 4 + 1], v[j * 4 + 2], v[j * 4 + 3]);
-}
-__device__ __forceinline__ void unstage_row_bf16(const uint8_t* buf, int lane, float* v) {
-#pragma unroll
-  for (int j = 0; j < 4; ++j) unpack8(*reinterpret_cast<const uint4*>(buf + sw64(lane, j)), v + j * 8);
-}
-// 32 x 32 bf16 block <-> global rows of `ld` elements starting at g; cv = valid columns (multiple of 8)
-__device__ __forceinline__ void flush_bf16(const uint8_t* buf, int lane, __nv_bfloat16* g, size_t ld, int cv) {
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = i * 8 + (lane >> 2), j = lane & 3;
-    if (j * 8 < cv) *reinterpret_cast<uint4*>(g + (size_t)r * ld + j * 8) = *reinterpret_cast<const uint4*>(buf + sw64(r, j));
-  }
-}
-__device__ __forceinline__ void fetch_bf16(uint8_t* buf, int lane, const __nv_bfloat16* g, size_t ld, int cv) {
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = i * 8 + (lane >> 2), j = lane & 3;
-    uint4 x = make_uint4(0, 0, 0, 0);
-    if (j * 8 < cv) x = *reinterpret_cast<const uint4*>(g + (size_t)r * ld + j * 8);
-    *reinterpret_cast<uint4*>(buf + sw64(r, j)) = x;
   }
 }
 
@@ -443,8 +426,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     const int q = warp & 3;                               // TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;                     // which half of the accumulator columns
     const int row = q * 32 + lane;
+    const bool wide = p.wide != 0;                        // 32-byte accesses allowed for this launch
     const uint32_t tempty_leader = map_to_cta(bar_tempty, 0);
-    uint8_t* stg = ctl + 256 + (warp - 2) * STAGING_BYTES;   // this warp's staging block
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     for (int t = pair; t < n_total && ok; t += n_pairs) {
@@ -458,34 +441,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       const int rp = tl.m0 + (int)rank * BM + row;
       float v[32];
 
-      // Each lane owns one accumulator row, but global memory wants whole lines: every 32-column
-      // chunk goes through this warp's 4 KB staging block in shared memory so that one store (or
-      // load) instruction of the warp covers 8 rows x 64 B (bf16) or 4 rows x 128 B (fp32).
-      const int row0 = tl.m0 + (int)rank * BM + q * 32;   // first row of this warp's 32-row block
-
       if (MODE == G_FWD1) {
-        float w[32], a[32];
+        float w[32];
         const int F = p.F;
         for (int c = half * 64; c < half * 64 + 64; c += 32) {
-          const int col = tl.nt * 128 + c;
-          const int cv = min(32, F - col);
-          if (cv <= 0) break;
           tc_ld32(taddr + c, v);
           tc_ld32(taddr + 128 + c, w);
+          const int col = tl.nt * 128 + c;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) a[i] = fast_swiglu(v[i], w[i]);
-          const size_t gofs = (size_t)row0 * F + col;
-          stage_row_bf16(stg, lane, a);
-          if (p.save) stage_row_bf16(stg + 2048, lane, v);
-          __syncwarp();
-          flush_bf16(stg, lane, p.o0 + gofs, F, cv);
-          if (p.save) flush_bf16(stg + 2048, lane, p.o1 + gofs, F, cv);
-          __syncwarp();
-          if (p.save) {
-            stage_row_bf16(stg, lane, w);
-            __syncwarp();
-            flush_bf16(stg, lane, p.o2 + gofs, F, cv);
-            __syncwarp();
+          for (int g16 = 0; g16 < 2; ++g16) {
+            if (col + g16 * 16 < F) {
+              float a16[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i) a16[i] = fast_swiglu(v[g16 * 16 + i], w[g16 * 16 + i]);
+              const size_t o = (size_t)rp * F + col + g16 * 16;
+              st32(p.o0 + o, pack8(a16), pack8(a16 + 8), wide, col + g16 * 16 + 8 < F);
+              if (p.save) {
+                st32(p.o1 + o, pack8(v + g16 * 16), pack8(v + g16 * 16 + 8), wide, col + g16 * 16 + 8 < F);
+                st32(p.o2 + o, pack8(w + g16 * 16), pack8(w + g16 * 16 + 8), wide, col + g16 * 16 + 8 < F);
+              }
+            }
           }
         }
       } else if (MODE == G_FWD2 || MODE == G_DX) {
@@ -493,23 +468,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         const float g = (MODE == G_FWD2 && flat >= 0) ? p.gates[flat] : 1.0f;
         const int N = p.N;
         for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
-          const int col = tl.nt * BN + c;
-          const int cv = min(32, N - col);
-          if (cv <= 0) break;
           tc_ld32(taddr + c, v);
+          const int col = tl.nt * BN + c;
+          if (flat >= 0) {
+            float* o = p.of + (size_t)flat * N + col;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] *= g;
-          stage_row_f32(stg, lane, v);
-          __syncwarp();
+            for (int g8 = 0; g8 < 4; ++g8)
+              if (col + g8 * 8 < N) {
+                float t8[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int r = i * 4 + (lane >> 3), j = lane & 7;
-            const int rflat = __shfl_sync(0xffffffffu, flat, r);
-            if (rflat >= 0 && j * 4 < cv)
-              *reinterpret_cast<uint4*>(p.of + (size_t)rflat * N + col + j * 4) =
-                  *reinterpret_cast<const uint4*>(stg + sw128(r, j));
+                for (int i = 0; i < 8; ++i) t8[i] = g * v[g8 * 8 + i];
+                st32(o + g8 * 8, f4(t8), f4(t8 + 4), wide);
+              }
           }
-          __syncwarp();
         }
       } else if (MODE == G_DACT) {
         const int flat = p.rowmap[rp];
@@ -518,69 +489,69 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         float rowdot = 0.f;
         for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
           const int col = tl.nt * BN + c;
-          const int cv = min(32, F - col);
-          if (cv <= 0) break;
-          const size_t gofs = (size_t)row0 * F + col;
-          // saved pre-activations of the 32x32 block: coalesced loads into the staging block
-          fetch_bf16(stg, lane, p.h1 + gofs, F, cv);
-          fetch_bf16(stg + 2048, lane, p.h3 + gofs, F, cv);
-          tc_ld32(taddr + c, v);
-          __syncwarp();
-          float h1[32], h3[32];
-          unstage_row_bf16(stg, lane, h1);
-          unstage_row_bf16(stg + 2048, lane, h3);
-          __syncwarp();
+          uint4 q1[4], q3[4];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float da = v[i];
-            const float sg = fast_sigmoid(h1[i]);
-            const float hs = h1[i] * sg;                      // silu(h1)
-            const float a = hs * h3[i];
-            const float gda = g * da;
-            rowdot = (i < cv) ? fmaf(da, a, rowdot) : rowdot;
-            v[i] = g * a;                                     // g*a, reuses the accumulator registers
-            h3[i] = gda * h3[i] * sg * (1.0f + h1[i] * (1.0f - sg));   // dh1
-            h1[i] = gda * hs;                                 // dh3
+          for (int g16 = 0; g16 < 2; ++g16) {
+            if (col + g16 * 16 < F) {
+              const size_t o = (size_t)rp * F + col + g16 * 16;
+              ld32(p.h1 + o, q1[2 * g16], q1[2 * g16 + 1], wide, col + g16 * 16 + 8 < F);
+              ld32(p.h3 + o, q3[2 * g16], q3[2 * g16 + 1], wide, col + g16 * 16 + 8 < F);
+            }
           }
-          stage_row_bf16(stg, lane, h3);
-          stage_row_bf16(stg + 2048, lane, h1);
-          __syncwarp();
-          flush_bf16(stg, lane, p.o0 + gofs, F, cv);
-          flush_bf16(stg + 2048, lane, p.o1 + gofs, F, cv);
-          __syncwarp();
-          stage_row_bf16(stg, lane, v);
-          __syncwarp();
-          flush_bf16(stg, lane, p.o2 + gofs, F, cv);
-          __syncwarp();
+          tc_ld32(taddr + c, v);
+#pragma unroll
+          for (int g16 = 0; g16 < 2; ++g16) {
+            if (col + g16 * 16 < F) {
+              const size_t o = (size_t)rp * F + col + g16 * 16;
+              float h1[16], h3[16], d1[16], d3[16], ga[16];
+              unpack8(q1[2 * g16], h1); unpack8(q1[2 * g16 + 1], h1 + 8);
+              unpack8(q3[2 * g16], h3); unpack8(q3[2 * g16 + 1], h3 + 8);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const float da = v[g16 * 16 + i];
+                const float sg = fast_sigmoid(h1[i]);
+                const float hs = h1[i] * sg;
+                const float a = hs * h3[i];
+                const float gda = g * da;
+                d1[i] = gda * h3[i] * sg * (1.0f + h1[i] * (1.0f - sg));
+                d3[i] = gda * hs;
+                ga[i] = g * a;
+                rowdot = fmaf(da, a, rowdot);
+              }
+              st32(p.o0 + o, pack8(d1), pack8(d1 + 8), wide, col + g16 * 16 + 8 < F);
+              st32(p.o1 + o, pack8(d3), pack8(d3 + 8), wide, col + g16 * 16 + 8 < F);
+              st32(p.o2 + o, pack8(ga), pack8(ga + 8), wide, col + g16 * 16 + 8 < F);
+            }
+          }
         }
         p.dg_part[(size_t)(tl.nt * 2 + half) * p.r_pad_max + rp] = rowdot;
       } else {  // WGRAD
         const int N = p.N;
+        const bool row_ok = rp < p.M;
         for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
-          const int col = tl.nt * BN + c;
-          const int cv = min(32, N - col);
-          if (cv <= 0) break;
           if (have_acc) tc_ld32(taddr + c, v);
           else {
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = 0.f;
           }
-          stage_row_f32(stg, lane, v);
-          __syncwarp();
+          const int col = tl.nt * BN + c;
+          if (row_ok) {
+            float* o = p.of + ((size_t)tl.e * p.M + rp) * N + col;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int r = i * 4 + (lane >> 3), j = lane & 7;
-            if (row0 + r < p.M && j * 4 < cv) {
-              float* o = p.of + ((size_t)tl.e * p.M + row0 + r) * N + col + j * 4;
-              float4 x4 = *reinterpret_cast<const float4*>(stg + sw128(r, j));
-              if (p.accumulate) {
-                const float4 old = *reinterpret_cast<const float4*>(o);
-                x4.x += old.x; x4.y += old.y; x4.z += old.z; x4.w += old.w;
+            for (int g8 = 0; g8 < 4; ++g8) {
+              if (col + g8 * 8 < N) {
+                float t8[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) t8[i] = v[g8 * 8 + i];
+                if (p.accumulate) {
+                  uint4 a, b; ld32(o + g8 * 8, a, b, wide);
+                  t8[0] += __uint_as_float(a.x); t8[1] += __uint_as_float(a.y); t8[2] += __uint_as_float(a.z); t8[3] += __uint_as_float(a.w);
+                  t8[4] += __uint_as_float(b.x); t8[5] += __uint_as_float(b.y); t8[6] += __uint_as_float(b.z); t8[7] += __uint_as_float(b.w);
+                }
+                st32(o + g8 * 8, f4(t8), f4(t8 + 4), wide);
               }
-              *reinterpret_cast<float4*>(o) = x4;
             }
           }
-          __syncwarp();
         }
       }
       if (have_acc) {
@@ -660,6 +631,8 @@ btx_status launch_tc(const CUtensorMap& a0, const CUtensorMap& a1, const CUtenso
   return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
 }
 
+bool aligned32(const void* p) { return ((uintptr_t)p & 31) == 0; }
+
 TcParams base_params(const Plan& pl, const Buffers& b) {
   TcParams p = {};
   p.d = pl.d; p.F = pl.F; p.E = pl.E; p.r_pad_max = pl.r_pad_max;
@@ -682,11 +655,14 @@ btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void
   TcParams p = base_params(pl, b);
   p.n_tiles = (pl.F + 127) / 128; p.kb_total = (pl.d + BK - 1) / BK; p.N = pl.F;
   p.o0 = (__nv_bfloat16*)b.act; p.o1 = (__nv_bfloat16*)b.h1; p.o2 = (__nv_bfloat16*)b.h3; p.save = save;
+  const bool f_pitch32 = pl.F % 16 == 0;                  // bf16 rows of F elements start on 32-byte boundaries
+  p.wide = f_pitch32 && aligned32(b.act) && aligned32(b.h1) && aligned32(b.h3);
   if ((s = launch_tc<G_FWD1>(a, a, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(2, st);
   // GEMM-2: gate-scaled expert rows = act W2^T
   if (!make_map(&a, b.act, F, RP, 0, 64, 128) || !make_map(&b0, w2, F, d, E, 64, 128)) return BTX_ERR_CUDA;
   p.n_tiles = (pl.d + BN - 1) / BN; p.kb_total = (pl.F + BK - 1) / BK; p.N = pl.d; p.of = b.yp;
+  p.wide = aligned32(b.yp);                               // fp32 rows of d (a multiple of 8) elements
   return launch_tc<G_FWD2>(a, a, b0, b0, p, pl.mt_max * p.n_tiles, st);
 }
 
@@ -702,6 +678,7 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   p.n_tiles = (pl.F + BN - 1) / BN; p.kb_total = (pl.d + BK - 1) / BK; p.N = pl.F;
   p.h1 = (const __nv_bfloat16*)b.h1; p.h3 = (const __nv_bfloat16*)b.h3;
   p.o0 = (__nv_bfloat16*)b.dh1; p.o1 = (__nv_bfloat16*)b.dh3; p.o2 = (__nv_bfloat16*)b.ga; p.dg_part = b.dg_part;
+  p.wide = pl.F % 16 == 0 && aligned32(b.h1) && aligned32(b.h3) && aligned32(b.dh1) && aligned32(b.dh3) && aligned32(b.ga);
   if ((s = launch_tc<G_DACT>(a0, a0, b0, b0, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(2, st);
   // dgrad-1: dXs = dh1 W1 + dh3 W3 (weights read N-major), scatter to t*k+slot rows
@@ -709,22 +686,24 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
       !make_map(&b0, w1, d, F, E, 64, 64) || !make_map(&b1, w3, d, F, E, 64, 64))
     return BTX_ERR_CUDA;
   p.n_tiles = (pl.d + BN - 1) / BN; p.kb_half = (pl.F + BK - 1) / BK; p.kb_total = 2 * p.kb_half; p.N = pl.d;
-  p.of = b.dxp;
+  p.of = b.dxp; p.wide = aligned32(b.dxp);
   if ((s = launch_tc<G_DX>(a0, a1, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(3, st);
   // wgrads: contraction over the expert's padded token rows, both operands MN-major
   p.accumulate = accumulate;
   if (!make_map(&a0, b.dys, d, RP, 0, 64, 64) || !make_map(&b0, b.ga, F, RP, 0, 64, 64)) return BTX_ERR_CUDA;
   p.M = pl.d; p.N = pl.F; p.m_tiles = (pl.d + kRowTile - 1) / kRowTile; p.n_tiles = (pl.F + BN - 1) / BN; p.of = dw2;
+  p.wide = aligned32(dw2);
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(4, st);
   if (!make_map(&a0, b.dh1, F, RP, 0, 64, 64) || !make_map(&a1, b.dh3, F, RP, 0, 64, 64) ||
       !make_map(&b0, b.xs, d, RP, 0, 64, 64))
     return BTX_ERR_CUDA;
   p.M = pl.F; p.N = pl.d; p.m_tiles = (pl.F + kRowTile - 1) / kRowTile; p.n_tiles = (pl.d + BN - 1) / BN; p.of = dw1;
+  p.wide = aligned32(dw1);
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(5, st);
-  p.of = dw3;
+  p.of = dw3; p.wide = aligned32(dw3);
   s = launch_tc<G_WGRAD>(a1, a1, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st);
   mark_stage(6, st);
   return s;
