@@ -282,6 +282,16 @@ def run_moe(args, workload):
                     roofline={"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                               "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["_source"],
                               "kernel": "tc_gemm_kernel (all launches of the step)"})
+        # per-layer stage times from one extra, untimed pass
+        evs = [new_events(5) for _ in sets]
+        for inp, ev in zip(sets, evs):
+            B.btx_set_stage_events(ev)
+            B.btx_moe_forward(desc, inp["x"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], y, None, None, ws)
+        B.btx_set_stage_events(None)
+        torch.cuda.synchronize()
+        names_f = ["route_permute_gather", "gemm1_swiglu", "gemm2_scatter", "combine"]
+        line["stages_ms"] = {"fwd." + nme: round(statistics.mean(ev[i].elapsed_time(ev[i + 1]) for ev in evs), 4)
+                             for i, nme in enumerate(names_f)}
     else:
         tokens_s = T / (ms * 1e-3) * world
         line.update(metric="moe_ffn_%s_tokens_per_s" % workload, value=tokens_s, unit="tokens/s",

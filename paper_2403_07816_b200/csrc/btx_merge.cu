@@ -1,6 +1,7 @@
 // MiX merge (Section 3.2): feed-forward matrices are copied into the stacked expert tensor,
 // every other parameter is averaged over the N models.  One persistent, bandwidth-bound kernel
-// walks a table of work items in 16 KB chunks with 128-bit streaming loads and stores.
+// walks a table of work items in 64 KB chunks with 128-bit streaming loads and stores, four
+// vectors per thread in flight from every source.
 #include <vector>
 
 #include "btx_common.cuh"
@@ -9,7 +10,7 @@ namespace btx {
 namespace {
 
 constexpr int kMaxModels = 16;
-constexpr int kChunkVecs = 1024;          // 16-byte vectors per chunk
+constexpr int kChunkVecs = 4096;          // 16-byte vectors per chunk (64 KB of output)
 constexpr int kMergeThreads = 256;
 
 struct DevItem {
@@ -86,9 +87,50 @@ merge_kernel(const DevItem* __restrict__ items, const uint64_t* __restrict__ chu
     const uint64_t v1 = min(nvec, v0 + (uint64_t)kChunkVecs);
     const int ns = it.nsrc;
     uint4* dst = reinterpret_cast<uint4*>(it.dst);
+    constexpr int U = 4;                                    // vectors per thread per round
     if (ns == 1) {
       const uint4* s = reinterpret_cast<const uint4*>(it.src[0]);
-      for (uint64_t v = v0 + threadIdx.x; v < v1; v += kMergeThreads) st_stream(dst + v, ld_stream(s + v));
+      uint64_t v = v0 + threadIdx.x;
+      for (; v + (U - 1) * kMergeThreads < v1; v += U * kMergeThreads) {
+        uint4 x[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) x[u] = ld_stream(s + v + u * kMergeThreads);
+#pragma unroll
+        for (int u = 0; u < U; ++u) st_stream(dst + v + u * kMergeThreads, x[u]);
+      }
+      for (; v < v1; v += kMergeThreads) st_stream(dst + v, ld_stream(s + v));
+    } else if (ns == 4) {
+      // the common case (four expert LLMs): all 16 loads of a round are issued before any use
+      const uint4* s0 = reinterpret_cast<const uint4*>(it.src[0]);
+      const uint4* s1 = reinterpret_cast<const uint4*>(it.src[1]);
+      const uint4* s2 = reinterpret_cast<const uint4*>(it.src[2]);
+      const uint4* s3 = reinterpret_cast<const uint4*>(it.src[3]);
+      uint64_t v = v0 + threadIdx.x;
+      for (; v + (U - 1) * kMergeThreads < v1; v += U * kMergeThreads) {
+        uint4 x[U][4];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const uint64_t w = v + u * kMergeThreads;
+          x[u][0] = ld_stream(s0 + w); x[u][1] = ld_stream(s1 + w); x[u][2] = ld_stream(s2 + w); x[u][3] = ld_stream(s3 + w);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          float acc[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+#pragma unroll
+          for (int m = 0; m < 4; ++m) Elem<T>::add(acc, x[u][m]);    // model order 0..3
+          st_stream(dst + v + u * kMergeThreads, Elem<T>::pack(acc, 4.0f));
+        }
+      }
+      for (; v < v1; v += kMergeThreads) {
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+        Elem<T>::add(acc, ld_stream(s0 + v)); Elem<T>::add(acc, ld_stream(s1 + v));
+        Elem<T>::add(acc, ld_stream(s2 + v)); Elem<T>::add(acc, ld_stream(s3 + v));
+        st_stream(dst + v, Elem<T>::pack(acc, 4.0f));
+      }
     } else {
       for (uint64_t v = v0 + threadIdx.x; v < v1; v += kMergeThreads) {
         float acc[8];
