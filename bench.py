@@ -204,7 +204,7 @@ def run_moe(args, workload):
     if args.tokens:
         T = args.tokens                      # reduced batch for profiler captures
     train = workload == "fwd_bwd"
-    layers = 32 if workload == "decode" else 1
+    layers = (args.layers or 32) if workload == "decode" else 1
     K, W = args.steps, max(args.warmup, 3)
     peaks = load_peaks()
 
@@ -267,7 +267,8 @@ def run_moe(args, workload):
 
     R = T * k
     flops_step = (18 if train else 6) * R * d * F * layers
-    launches_per_step = (9 + (10 if train else 0)) * layers
+    fwd_launches = 5 if T * k <= 1024 else 9        # small batches route and permute in one launch
+    launches_per_step = (fwd_launches + (10 if train else 0)) * layers
     line = {
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "clocks": clocks,
@@ -447,6 +448,7 @@ def main():
     ap.add_argument("--merge-layers", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="decode: number of layers (profiling only)")
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling only; not a bench number)")
     args = ap.parse_args()
     if args.impl == "reference":

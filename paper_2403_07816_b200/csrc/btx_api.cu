@@ -152,8 +152,14 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
 
   mark_stage(0, st);
   BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
-  BTX_CUDA_OK(launch_router(pl, desc->dtype, desc->routing, desc->lb_alpha, x, w_router, router_bias, nullptr, b, st));
-  BTX_CUDA_OK(launch_permute(pl, b, st));
+  if (route_permute_small_fits(pl)) {
+    BTX_CUDA_OK(launch_route_permute_small(pl, desc->dtype, desc->routing, desc->lb_alpha, x, w_router, router_bias, b,
+                                           st));
+  } else {
+    BTX_CUDA_OK(launch_router(pl, desc->dtype, desc->routing, desc->lb_alpha, x, w_router, router_bias, nullptr, b,
+                              st));
+    BTX_CUDA_OK(launch_permute(pl, b, st));
+  }
   BTX_CUDA_OK(launch_gather_rows(pl, x, b.xs, b, st));
   mark_stage(1, st);
   if (desc->dtype == BTX_F32) {

@@ -60,6 +60,10 @@ void mark_stage(int i, cudaStream_t st);
 cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, const void* x, const void* w_router,
                           const float* bias, const float* given_logits, const Buffers& b, cudaStream_t st);
 cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st);
+// Router + loss + permutation in one single-block launch, for batches with T*k <= 1024.
+bool route_permute_small_fits(const Plan& pl);
+cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, float alpha, const void* x,
+                                       const void* w_router, const float* bias, const Buffers& b, cudaStream_t st);
 cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st);
 cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, void* y, cudaStream_t st);
 cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float alpha, float lb_scale,

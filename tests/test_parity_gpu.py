@@ -39,7 +39,8 @@ def test_tiny_config_forward_backward(dtype):
 
 @pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 @pytest.mark.parametrize("T,d,F,E,k", [(37, 64, 72, 5, 3), (1, 128, 128, 4, 2), (300, 136, 264, 8, 2),
-                                        (129, 64, 64, 1, 1), (515, 192, 328, 3, 1)])
+                                        (129, 64, 64, 1, 1), (515, 192, 328, 3, 1),
+                                        (700, 64, 72, 4, 2)])      # T*k > 1024: multi-block routing kernels
 def test_ragged_shapes(dtype, T, d, F, E, k):
     run_case(T, d, F, E, k, dtype, seed=11, alpha=0.05, lb_scale=0.7)
 
