@@ -54,7 +54,7 @@ struct TcParams {
   int m_tiles;                  // WGRAD: 256-row tiles per expert
   int kb_total;                 // K blocks per tile (grouped modes)
   int kb_half;                  // DX: K blocks of the first operand pair
-  int M, N;                     // output rows per expert (WGRAD) / columns
+  int M, N;                     // WGRAD: gradient columns (lane side) and rows; other modes: N = output columns
   const int32_t* tile_expert;
   const int32_t* pad_offsets;
   const int32_t* rowmap;
@@ -525,30 +525,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           }
         }
         p.dg_part[(size_t)(tl.nt * 2 + half) * p.r_pad_max + rp] = rowdot;
-      } else {  // WGRAD
-        const int N = p.N;
-        const bool row_ok = rp < p.M;
+      } else {  // WGRAD, stored transposed: lane = column of the gradient, TMEM column = its row
+        const int ncols = p.M, nrows = p.N;                // memory shape of one expert's gradient: [nrows][ncols]
+        const bool lane_ok = rp < ncols;
         for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
+          const int r0 = tl.nt * BN + c;
+          if (r0 >= nrows) break;
           if (have_acc) tc_ld32(taddr + c, v);
           else {
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = 0.f;
           }
-          const int col = tl.nt * BN + c;
-          if (row_ok) {
-            float* o = p.of + ((size_t)tl.e * p.M + rp) * N + col;
+          if (lane_ok) {
+            float* o = p.of + ((size_t)tl.e * nrows + r0) * ncols + rp;
 #pragma unroll
-            for (int g8 = 0; g8 < 4; ++g8) {
-              if (col + g8 * 8 < N) {
-                float t8[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) t8[i] = v[g8 * 8 + i];
-                if (p.accumulate) {
-                  uint4 a, b; ld32(o + g8 * 8, a, b, wide);
-                  t8[0] += __uint_as_float(a.x); t8[1] += __uint_as_float(a.y); t8[2] += __uint_as_float(a.z); t8[3] += __uint_as_float(a.w);
-                  t8[4] += __uint_as_float(b.x); t8[5] += __uint_as_float(b.y); t8[6] += __uint_as_float(b.z); t8[7] += __uint_as_float(b.w);
-                }
-                st32(o + g8 * 8, f4(t8), f4(t8 + 4), wide);
+            for (int i = 0; i < 32; ++i) {
+              if (r0 + i < nrows) {                        // one 128-byte line per warp instruction
+                float x = v[i];
+                if (p.accumulate) x += o[(size_t)i * ncols];
+                o[(size_t)i * ncols] = x;
               }
             }
           }
@@ -689,22 +684,22 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   p.of = b.dxp; p.wide = aligned32(b.dxp);
   if ((s = launch_tc<G_DX>(a0, a1, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(3, st);
-  // wgrads: contraction over the expert's padded token rows, both operands MN-major
+  // wgrads: contraction over the expert's padded token rows, both operands MN-major.  The operand
+  // indexed by the gradient's contiguous (column) index goes on the M side, so that the 32 lanes of
+  // an epilogue warp write 32 neighbouring columns of one gradient row.
   p.accumulate = accumulate;
-  if (!make_map(&a0, b.dys, d, RP, 0, 64, 64) || !make_map(&b0, b.ga, F, RP, 0, 64, 64)) return BTX_ERR_CUDA;
-  p.M = pl.d; p.N = pl.F; p.m_tiles = (pl.d + kRowTile - 1) / kRowTile; p.n_tiles = (pl.F + BN - 1) / BN; p.of = dw2;
-  p.wide = aligned32(dw2);
+  if (!make_map(&a0, b.ga, F, RP, 0, 64, 64) || !make_map(&b0, b.dys, d, RP, 0, 64, 64)) return BTX_ERR_CUDA;
+  p.M = pl.F; p.N = pl.d; p.m_tiles = (pl.F + kRowTile - 1) / kRowTile; p.n_tiles = (pl.d + BN - 1) / BN; p.of = dw2;
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(4, st);
-  if (!make_map(&a0, b.dh1, F, RP, 0, 64, 64) || !make_map(&a1, b.dh3, F, RP, 0, 64, 64) ||
-      !make_map(&b0, b.xs, d, RP, 0, 64, 64))
+  if (!make_map(&a0, b.xs, d, RP, 0, 64, 64) || !make_map(&b0, b.dh1, F, RP, 0, 64, 64) ||
+      !make_map(&b1, b.dh3, F, RP, 0, 64, 64))
     return BTX_ERR_CUDA;
-  p.M = pl.F; p.N = pl.d; p.m_tiles = (pl.F + kRowTile - 1) / kRowTile; p.n_tiles = (pl.d + BN - 1) / BN; p.of = dw1;
-  p.wide = aligned32(dw1);
+  p.M = pl.d; p.N = pl.F; p.m_tiles = (pl.d + kRowTile - 1) / kRowTile; p.n_tiles = (pl.F + BN - 1) / BN; p.of = dw1;
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
   mark_stage(5, st);
-  p.of = dw3; p.wide = aligned32(dw3);
-  s = launch_tc<G_WGRAD>(a1, a1, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st);
+  p.of = dw3;
+  s = launch_tc<G_WGRAD>(a0, a0, b1, b1, p, pl.E * p.m_tiles * p.n_tiles, st);
   mark_stage(6, st);
   return s;
 }
