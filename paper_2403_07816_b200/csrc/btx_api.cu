@@ -37,6 +37,12 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   if (p.route_blocks > 148 * 8) p.route_blocks = 148 * 8;
   p.perm_blocks = (p.R + 1023) / 1024;
   p.wr_chunks = (p.T + 127) / 128;
+  p.small = !routing_only && desc->dtype == BTX_BF16 && route_permute_small_fits(p);
+  if (p.small) {
+    const int chunks = p.E < p.R ? p.E : p.R;             // typical: every expert holds one token chunk
+    p.dec_s1 = pick_decode_splits(2 * chunks * ((p.F + 255) / 256), (p.d + 63) / 64);
+    p.dec_s2 = pick_decode_splits(chunks * ((p.d + 255) / 256), (p.F + 63) / 64);
+  }
 
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
@@ -73,6 +79,10 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   p.w_ga = take(rp * p.F * p.esize);
   p.w_dxp = take((size_t)p.R * p.d * 4);
   if (o < fwd_end) o = fwd_end;
+  if (p.small) {
+    const size_t n1 = (size_t)2 * p.dec_s1 * p.R * p.F, n2 = (size_t)p.dec_s2 * p.R * p.d;
+    p.w_part = take((n1 > n2 ? n1 : n2) * 4);
+  }
   // a forward that keeps nothing for backward parks its "saved" state here
   p.w_saved_fallback = take(p.saved_bytes);
   p.workspace_bytes = o;
@@ -93,6 +103,7 @@ static void resolve(const Plan& p, char* saved, char* ws, Buffers* b) {
   b->act = ws + p.w_act;  b->yp = (float*)(ws + p.w_yp);
   b->dys = ws + p.w_dys;  b->dh1 = ws + p.w_dh1;  b->dh3 = ws + p.w_dh3;  b->ga = ws + p.w_ga;
   b->dxp = (float*)(ws + p.w_dxp);
+  b->part = (float*)(ws + p.w_part);
   b->dg_part = (float*)(ws + p.w_dg_part);  b->dz = (float*)(ws + p.w_dz);  b->dwr_part = (float*)(ws + p.w_dwr_part);
 }
 
@@ -162,13 +173,19 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
   }
   BTX_CUDA_OK(launch_gather_rows(pl, x, b.xs, b, st));
   mark_stage(1, st);
+  const float* expert_rows = b.yp;
+  int splits = 1;
   if (desc->dtype == BTX_F32) {
     BTX_CUDA_OK(launch_expert_forward_f32(pl, w1, w3, w2, b, desc->save_for_backward, st));
+  } else if (pl.small) {
+    if ((s = launch_expert_forward_small_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
+    expert_rows = b.part;
+    splits = pl.dec_s2;
   } else {
     if ((s = launch_expert_forward_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
   }
   mark_stage(3, st);
-  BTX_CUDA_OK(launch_combine(pl, desc->dtype, b.yp, y, st));
+  BTX_CUDA_OK(launch_combine(pl, desc->dtype, expert_rows, splits, y, st));
   mark_stage(4, st);
 
   if (routing) {

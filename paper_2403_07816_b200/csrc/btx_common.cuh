@@ -26,12 +26,14 @@ struct Plan {
   int route_blocks;                  // blocks of the router kernel (partial sums for u, p)
   int perm_blocks;                   // blocks of the permutation kernels
   int wr_chunks;                     // token chunks of the router-weight gradient
+  int small;                         // BF16 batch with T*k <= 1024: weight-streaming forward kernels
+  int dec_s1, dec_s2;                // their contraction splits (pass 1: W1/W3, pass 2: W2)
   // saved
   size_t s_topk, s_gates, s_probs, s_logits, s_u, s_p, s_loss, s_counts, s_offsets, s_pad_offsets,
       s_tile_expert, s_rowmap, s_flat2row, s_perm, s_inv_perm, s_xs, s_h1, s_h3, saved_bytes;
   // workspace
   size_t w_status, w_route_part, w_perm_counts, w_perm_base, w_act, w_yp, w_dys, w_dh1, w_dh3, w_ga,
-      w_dxp, w_dg_part, w_dz, w_dwr_part, w_saved_fallback, workspace_bytes;
+      w_dxp, w_dg_part, w_dz, w_dwr_part, w_part, w_saved_fallback, workspace_bytes;
 };
 
 // routing_only: plan for btx_lb_loss (no expert buffers)
@@ -49,6 +51,7 @@ struct Buffers {
   int32_t* status;    float* route_part;  int32_t* perm_counts;  int32_t* perm_base;
   void* act;  float* yp;  void* dys;  void* dh1;  void* dh3;  void* ga;  float* dxp;
   float* dg_part;  float* dz;  float* dwr_part;
+  float* part;        // split partial products of the small-batch forward
 };
 
 // Records stage event i of the calling thread's timing hook (no-op when the hook is off).
@@ -65,7 +68,8 @@ bool route_permute_small_fits(const Plan& pl);
 cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, float alpha, const void* x,
                                        const void* w_router, const float* bias, const Buffers& b, cudaStream_t st);
 cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st);
-cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, void* y, cudaStream_t st);
+// y[t] = sum over slots and over `splits` partial copies ([split][R][d]) of the expert rows
+cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, cudaStream_t st);
 cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float alpha, float lb_scale,
                                    int stopgrad_u, int have_dg, const void* x, const void* w_router, const Buffers& b,
                                    void* dx, float* dw_router, float* dbias, float* dlogits_out, int accumulate,
@@ -79,6 +83,9 @@ cudaError_t launch_expert_backward_f32(const Plan& pl, const void* w1, const voi
                                        cudaStream_t st);
 btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                       const Buffers& b, int save, cudaStream_t st);
+int pick_decode_splits(int base_tiles, int kb_total);
+btx_status launch_expert_forward_small_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
+                                            const Buffers& b, int save, cudaStream_t st);
 btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                        const Buffers& b, float* dw1, float* dw3, float* dw2, int accumulate,
                                        cudaStream_t st);

@@ -1,0 +1,284 @@
+// Weight-streaming expert GEMMs for small batches (T*k <= 1024, the decode-shaped case), BF16.
+//
+// With a few tokens per expert the layer is bound by reading the expert weights once from HBM.
+// The weights therefore take the M side of the tensor-core tile (256 weight rows per CTA pair,
+// tcgen05.mma.cta_group::2) and a narrow chunk of 64 token rows takes the N side, so an MMA costs
+// 32 cycles instead of 128 and the tensor pipe never limits the stream.  The contraction is split
+// into S parts per tile so that the number of work items is a multiple of the CTA pairs; every
+// item writes its fp32 partial product for the valid tokens only, addressed [split][t*k+slot][row]:
+// a lane owns a weight row, so the 32 lanes of a warp write one 128-byte line per token.
+//
+//   pass 1   partial h1, h3 = W1_e x, W3_e x   -> swiglu_fixup_kernel sums the parts, a = silu(h1)*h3
+//   pass 2   partial gate * W2_e a             -> combine kernel sums parts and slots into y
+//
+// Same warp roles, barriers and bounded waits as the training-shaped kernel: warp 0 TMA producer
+// (9 stages of 128x64 weights + 32x64 tokens per CTA), warp 1 MMA issuer in the leader CTA,
+// warps 2-9 epilogue.
+#include "btx_tc_ptx.cuh"
+
+namespace btx {
+namespace {
+
+using namespace tcx;
+
+constexpr int WM = 128;                                  // weight rows per CTA (256 per pair)
+constexpr int TOK = 64;                                  // token rows per chunk (MMA N)
+constexpr int D_STAGES = 9;
+constexpr int DA_BYTES = WM * BK * 2, DB_BYTES = (TOK / 2) * BK * 2, D_STAGE_BYTES = DA_BYTES + DB_BYTES;
+constexpr int D_EPI_WARPS = 8;
+constexpr int D_THREADS = 64 + D_EPI_WARPS * 32;
+constexpr int D_MAX_CHUNKS = 192;                        // (1024 + 32 * 255) / 64 rounded up
+constexpr int D_SMEM_BYTES = D_STAGES * D_STAGE_BYTES + 1024 + 256 + (D_MAX_CHUNKS + 2) * 4;
+
+struct SwapParams {
+  int W;                        // weight rows per expert (F in pass 1, d in pass 2)
+  int E, S, n_w, m_tiles, kb_total;
+  const int32_t* pad_offsets;
+  const int32_t* tile_expert;
+  const int32_t* rowmap;
+  const float* gates;           // non-null: scale every token column by its gate
+  float* out0;                  // [S][R][W]
+  float* out1;                  // second weight matrix (pass 1: W3)
+  size_t split_stride;          // R * W
+  int32_t* status;
+};
+
+struct DTile { int which, chunk, mt, e, kb0, kb1, s; };
+
+__device__ __forceinline__ DTile d_tile(const SwapParams& p, const int* chunks, int n_valid, int t) {
+  DTile tl;
+  tl.s = t % p.S; t /= p.S;
+  tl.mt = t % p.m_tiles; t /= p.m_tiles;
+  const int ci = t % n_valid;
+  tl.which = t / n_valid;
+  tl.chunk = chunks[ci];
+  tl.e = p.tile_expert[(tl.chunk * TOK) / kRowTile];
+  tl.kb0 = (int)((long long)tl.s * p.kb_total / p.S);
+  tl.kb1 = (int)((long long)(tl.s + 1) * p.kb_total / p.S);
+  return tl;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(D_THREADS, 1)
+tc_swapk_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+                const __grid_constant__ CUtensorMap tmX, const SwapParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t ring = (raw + 1023u) & ~1023u;
+  uint8_t* ctl = smem_raw + (ring - raw) + D_STAGES * D_STAGE_BYTES;
+  const uint32_t bar_full = smem_u32(ctl);
+  const uint32_t bar_empty = bar_full + D_STAGES * 8;
+  const uint32_t bar_tfull = bar_empty + D_STAGES * 8;
+  const uint32_t bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + D_STAGES * 16 + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + D_STAGES * 16 + 40);
+  int* chunks = reinterpret_cast<int*>(ctl + 256);        // [0] = count, [1..] = chunk ids that hold tokens
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < D_STAGES; ++s) { mbar_init(bar_full + s * 8, 1); mbar_init(bar_empty + s * 8, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + a * 8, 1); mbar_init(bar_tempty + a * 8, 2 * D_EPI_WARPS * 32); }
+    *abort_flag = 0;
+    // expert segments start with their real rows, so a chunk holds tokens iff its first row does
+    int n = 0;
+    const int all = p.pad_offsets[p.E] / TOK;
+    for (int c = 0; c < all && n < D_MAX_CHUNKS; ++c)
+      if (p.rowmap[c * TOK] >= 0) chunks[1 + n++] = c;
+    chunks[0] = n;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int n_valid = chunks[0];
+  const int n_total = p.n_w * n_valid * p.m_tiles * p.S;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int t = pair; t < n_total && ok; t += n_pairs) {
+        const DTile tl = d_tile(p, chunks + 1, n_valid, t);
+        for (int kb = tl.kb0; kb < tl.kb1; ++kb) {
+          if (!(ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status))) break;
+          const uint32_t full_local = bar_full + stage * 8;
+          const uint32_t full = map_to_cta(full_local, 0);
+          const uint32_t sA = ring + stage * D_STAGE_BYTES, sB = sA + DA_BYTES;
+          if (rank == 0) mbar_expect_tx(full_local, 2 * D_STAGE_BYTES);
+          tma_load_3d(sA, tl.which ? &tmW1 : &tmW0, kb * BK, tl.mt * 2 * WM + (int)rank * WM, tl.e, full);
+          tma_load_2d(sB, &tmX, kb * BK, tl.chunk * TOK + (int)rank * (TOK / 2), full);
+          if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      for (int i = 0; i < D_STAGES && ok; ++i) {          // drain: all commits to this CTA have landed
+        ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status);
+        if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TOK >> 3) << 17) |
+                                 ((uint32_t)((2 * WM) >> 4) << 24);
+      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+      bool ok = true;
+      for (int t = pair; t < n_total && ok; t += n_pairs) {
+        const DTile tl = d_tile(p, chunks + 1, n_valid, t);
+        if (tl.kb1 <= tl.kb0) continue;
+        if (!(ok = mbar_wait(bar_tempty + acc * 8, acc_phase ^ 1u, abort_flag, p.status))) break;
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + acc * 256;
+        for (int kb = tl.kb0; kb < tl.kb1; ++kb) {
+          if (!(ok = mbar_wait(bar_full + stage * 8, phase, abort_flag, p.status))) break;
+          tc_fence_after();
+          const uint32_t sA = ring + stage * D_STAGE_BYTES, sB = sA + DA_BYTES;
+          const uint64_t da = smem_desc(sA, false), db = smem_desc(sB, false);
+#pragma unroll
+          for (int k16 = 0; k16 < BK / 16; ++k16)
+            tc_mma_pair(tmem_d, da + (uint64_t)(2 * k16), db + (uint64_t)(2 * k16), idesc,
+                        (kb > tl.kb0 || k16 > 0) ? 1u : 0u);
+          tc_commit_pair(bar_empty + stage * 8);
+          if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit_pair(bar_tfull + acc * 8);
+        acc ^= 1u;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    const int q = warp & 3, half = (warp - 2) >> 2;
+    const uint32_t tempty_leader = map_to_cta(bar_tempty, 0);
+    uint32_t acc = 0, acc_phase = 0;
+    bool ok = true;
+    for (int t = pair; t < n_total && ok; t += n_pairs) {
+      const DTile tl = d_tile(p, chunks + 1, n_valid, t);
+      if (tl.kb1 <= tl.kb0) continue;
+      // token of this lane's column: lane i of the warp looks up column half*32 + i
+      const int my_flat = p.rowmap[tl.chunk * TOK + half * 32 + lane];
+      const float my_gate = (p.gates != nullptr && my_flat >= 0) ? p.gates[my_flat] : 1.0f;
+      if (!(ok = mbar_wait(bar_tfull + acc * 8, acc_phase, abort_flag, p.status))) break;
+      tc_fence_after();
+      float v[32];
+      tc_ld32(tmem_base + acc * 256 + half * 32 + ((uint32_t)(q * 32) << 16), v);
+      tc_fence_before();
+      mbar_arrive_cluster(tempty_leader + acc * 8);
+      acc ^= 1u;
+      if (acc == 0) acc_phase ^= 1u;
+      const int wrow = tl.mt * 2 * WM + (int)rank * WM + q * 32 + lane;
+      float* out = (tl.which ? p.out1 : p.out0) + (size_t)tl.s * p.split_stride + wrow;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int flat = __shfl_sync(0xffffffffu, my_flat, i);
+        const float g = __shfl_sync(0xffffffffu, my_gate, i);
+        if (flat >= 0 && wrow < p.W) out[(size_t)flat * p.W] = g * v[i];
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+  }
+}
+
+// act[row][f] = silu(sum_s P1) * (sum_s P3) for the rows that hold tokens; h1/h3 are kept as well
+// when the forward saves for backward.  One block row per assignment, four columns per thread.
+__global__ void __launch_bounds__(256)
+swiglu_fixup_kernel(int F, int S, size_t split_stride, const float* __restrict__ p1, const float* __restrict__ p3,
+                    const int32_t* __restrict__ flat2row, __nv_bfloat16* __restrict__ act,
+                    __nv_bfloat16* __restrict__ h1s, __nv_bfloat16* __restrict__ h3s) {
+  const int flat = blockIdx.y;
+  const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (f >= F) return;
+  const size_t src = (size_t)flat * F + f;
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+  for (int s = 0; s < S; ++s) {
+    const float4 x = *reinterpret_cast<const float4*>(p1 + s * split_stride + src);
+    const float4 y = *reinterpret_cast<const float4*>(p3 + s * split_stride + src);
+    a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w;
+    b.x += y.x; b.y += y.y; b.z += y.z; b.w += y.w;
+  }
+  auto pack4 = [](float x0, float x1, float x2, float x3) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(x0, x1), hi = __floats2bfloat162_rn(x2, x3);
+    return make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+  };
+  const size_t dst = (size_t)flat2row[flat] * F + f;
+  *reinterpret_cast<uint2*>(act + dst) =
+      pack4(fast_swiglu(a.x, b.x), fast_swiglu(a.y, b.y), fast_swiglu(a.z, b.z), fast_swiglu(a.w, b.w));
+  if (h1s != nullptr) {
+    *reinterpret_cast<uint2*>(h1s + dst) = pack4(a.x, a.y, a.z, a.w);
+    *reinterpret_cast<uint2*>(h3s + dst) = pack4(b.x, b.y, b.z, b.w);
+  }
+}
+
+btx_status launch_swapk(const CUtensorMap& w0, const CUtensorMap& w1, const CUtensorMap& x, const SwapParams& p,
+                        cudaStream_t st) {
+  if (cudaFuncSetAttribute(tc_swapk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, D_SMEM_BYTES) != cudaSuccess)
+    return BTX_ERR_CUDA;
+  int pairs = sm_count() / 2;
+  if (pairs < 1) pairs = 1;
+  tc_swapk_kernel<<<2 * pairs, D_THREADS, D_SMEM_BYTES, st>>>(w0, w1, x, p);
+  return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
+}
+
+}  // namespace
+
+// Number of contraction splits that makes base_tiles * S fill whole rounds of the CTA pairs.
+int pick_decode_splits(int base_tiles, int kb_total) {
+  const int pairs = 74;                                   // 148 SMs; only a balance heuristic
+  int best = 1;
+  double best_eff = 0.0;
+  for (int S = 1; S <= 8 && S <= kb_total; ++S) {
+    const int tiles = base_tiles * S;
+    const double eff = (double)tiles / (double)(((tiles + pairs - 1) / pairs) * pairs);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best = S; }
+    if (eff >= 0.96) return S;
+  }
+  return best;
+}
+
+btx_status launch_expert_forward_small_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
+                                            const Buffers& b, int save, cudaStream_t st) {
+  const uint64_t d = pl.d, F = pl.F, E = pl.E, RP = pl.r_pad_max;
+  CUtensorMap m0, m1, mx;
+  btx_status s;
+  SwapParams p = {};
+  p.E = pl.E; p.pad_offsets = b.pad_offsets; p.tile_expert = b.tile_expert; p.rowmap = b.rowmap; p.status = b.status;
+  if (save) {   // backward reads whole padded tiles of h1/h3: rows without a token must be finite
+    if (cudaMemsetAsync(b.h1, 0, (size_t)RP * F * 2, st) != cudaSuccess ||
+        cudaMemsetAsync(b.h3, 0, (size_t)RP * F * 2, st) != cudaSuccess)
+      return BTX_ERR_CUDA;
+  }
+  // pass 1: partial h1, h3
+  if (!make_map(&m0, w1, d, F, E, 64, WM) || !make_map(&m1, w3, d, F, E, 64, WM) || !make_map(&mx, b.xs, d, RP, 0, 64, TOK / 2))
+    return BTX_ERR_CUDA;
+  p.W = pl.F; p.n_w = 2; p.m_tiles = (pl.F + 2 * WM - 1) / (2 * WM); p.kb_total = (pl.d + BK - 1) / BK; p.S = pl.dec_s1;
+  p.split_stride = (size_t)pl.R * pl.F;
+  p.out0 = b.part; p.out1 = b.part + (size_t)pl.dec_s1 * p.split_stride; p.gates = nullptr;
+  if ((s = launch_swapk(m0, m1, mx, p, st)) != BTX_OK) return s;
+  swiglu_fixup_kernel<<<dim3((pl.F / 4 + 255) / 256, pl.R), 256, 0, st>>>(
+      pl.F, pl.dec_s1, p.split_stride, p.out0, p.out1, b.flat2row, (__nv_bfloat16*)b.act,
+      save ? (__nv_bfloat16*)b.h1 : nullptr, save ? (__nv_bfloat16*)b.h3 : nullptr);
+  if (cudaGetLastError() != cudaSuccess) return BTX_ERR_CUDA;
+  mark_stage(2, st);
+  // pass 2: partial gate-scaled expert rows
+  if (!make_map(&m0, w2, F, d, E, 64, WM) || !make_map(&mx, b.act, F, RP, 0, 64, TOK / 2)) return BTX_ERR_CUDA;
+  p.W = pl.d; p.n_w = 1; p.m_tiles = (pl.d + 2 * WM - 1) / (2 * WM); p.kb_total = (pl.F + BK - 1) / BK; p.S = pl.dec_s2;
+  p.split_stride = (size_t)pl.R * pl.d;
+  p.out0 = b.part; p.out1 = b.part; p.gates = b.gates;
+  return launch_swapk(m0, m0, mx, p, st);
+}
+
+}  // namespace btx

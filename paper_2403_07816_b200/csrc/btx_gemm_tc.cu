@@ -28,22 +28,20 @@
 // workspace status word, raises a CTA-wide abort flag and the kernel drains and returns.  Both
 // CTAs always meet at a cluster barrier before they exit, so no remote arrival can target a CTA
 // that has already left.
-#include <cuda.h>
-
-#include "btx_common.cuh"
+#include "btx_tc_ptx.cuh"
 
 namespace btx {
 namespace {
 
+using namespace tcx;
+
 constexpr int BM = 128;                                  // rows per CTA; the pair covers 2*BM = kRowTile
-constexpr int BN = 256, BK = 64, STAGES = 6;
+constexpr int BN = 256, STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / 2) * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int CHUNK_BYTES = 64 * BK * 2;                 // one 64x64 MN-major box
 constexpr int EPI_WARPS = 8;
 constexpr int TC_THREADS = 64 + EPI_WARPS * 32;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 constexpr int GROUP_N = 8;                               // column tiles per raster group
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 static_assert(2 * BM == kRowTile, "a CTA pair covers one padded row tile");
 
 enum TcMode { G_FWD1 = 0, G_FWD2 = 1, G_DACT = 2, G_DX = 3, G_WGRAD = 4 };
@@ -70,173 +68,6 @@ struct TcParams {
   int wide;                     // all epilogue rows start on 32-byte boundaries
   int32_t* status;
 };
-
-// ---------------------------------------------------------------------------------------------
-// PTX wrappers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Arrive on a barrier that may live in the other CTA of the cluster.  Relaxed: the arrival only
-// hands a drained TMEM accumulator back (ordered by tcgen05.fence::before_thread_sync); it must not
-// wait for this thread's outstanding global stores the way a releasing arrival would.
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// One poll of the barrier.  The hint lets the hardware park the thread (up to about 10 us) until
-// the phase completes instead of spinning on shared memory.
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity), "r"(10000u) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out of time).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  unsigned long long t0 = global_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 15u) == 0u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        atomicExch(status, (int32_t)BTX_ERR_TIMEOUT);
-        return false;
-      }
-    }
-  }
-}
-
-// TMA tile loads of one CTA of a pair; the completion bytes go to `bar`, a shared::cluster address
-// that may name the leader CTA's barrier.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// arrive (once the MMAs issued so far have retired) on the barrier at this offset in both CTAs
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-      ::"r"(bar), "h"((uint16_t)3) : "memory");
-}
-__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accum) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle.  K-major: rows of 128 B, 8-row groups
-// 1024 B apart (stride offset).  MN-major: 64-element (128 B) runs along M/N, 8 contraction rows
-// per 1024 B group (stride offset), next 64-element run 8192 B further (leading offset).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
-  uint64_t dsc = (uint64_t)((addr & 0x3FFFFu) >> 4);
-  dsc |= (uint64_t)((mn_major ? CHUNK_BYTES : 16) >> 4) << 16;
-  dsc |= (uint64_t)(1024 >> 4) << 32;
-  dsc |= 1ull << 46;                                      // descriptor version of this architecture
-  dsc |= 2ull << 61;                                      // 128-byte swizzle
-  return dsc;
-}
-
-// SwiGLU pieces for the BF16 epilogues: sigmoid from one ex2 and one reciprocal approximation
-// (relative error about 2^-21, far below bf16 rounding).
-__device__ __forceinline__ float fast_sigmoid(float v) { return __frcp_rn(1.0f + __expf(-v)); }
-__device__ __forceinline__ float fast_swiglu(float h1, float h3) { return h1 * fast_sigmoid(h1) * h3; }
-
-// Epilogue global accesses move 32 bytes per lane (a whole DRAM sector) whenever the row pitch and
-// base allow it: half-sector (16-byte) writes from 32 different rows per instruction cost far more
-// in the memory pipeline, and in power, than their byte count suggests.
-__device__ __forceinline__ void st32(void* p, uint4 a, uint4 b, bool wide, bool second = true) {
-  if (wide) {
-    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w),
-                 "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
-  } else {
-    reinterpret_cast<uint4*>(p)[0] = a;
-    if (second) reinterpret_cast<uint4*>(p)[1] = b;
-  }
-}
-__device__ __forceinline__ void ld32(const void* p, uint4& a, uint4& b, bool wide, bool second = true) {
-  if (wide) {
-    asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w),
-                 "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p));
-  } else {
-    a = reinterpret_cast<const uint4*>(p)[0];
-    b = second ? reinterpret_cast<const uint4*>(p)[1] : make_uint4(0, 0, 0, 0);
-  }
-}
-__device__ __forceinline__ uint4 f4(const float* v) { return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])); }
-__device__ __forceinline__ uint4 pack8(const float* v) {
-  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
-  __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), e = __floats2bfloat162_rn(v[6], v[7]);
-  return make_uint4(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b),
-                    *reinterpret_cast<uint32_t*>(&c), *reinterpret_cast<uint32_t*>(&e));
-}
-__device__ __forceinline__ void unpack8(uint4 q, float* v) {
-  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&q);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float2 f = __bfloat1622float2(h[i]);
-    v[2 * i] = f.x; v[2 * i + 1] = f.y;
-  }
-}
 
 // ---------------------------------------------------------------------------------------------
 // Tile schedule: the same function is evaluated by the producer, the MMA issuer and the epilogue
@@ -572,47 +403,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 // ---------------------------------------------------------------------------------------------
 // Host side: tensor maps and launches
 // ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn == nullptr) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)sym;
-  }
-  return fn;
-}
-
-// bf16 tensor [rows, cols] (2D) or [E, rows, cols] (3D), cols contiguous; box = (box_cols, box_rows[, 1])
-bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t experts, uint32_t box_cols,
-              uint32_t box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[3] = {cols, rows, experts};
-  cuuint64_t strides[2] = {cols * 2, cols * rows * 2};
-  cuuint32_t box[3] = {box_cols, box_rows, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  const cuuint32_t rank = experts > 0 ? 3 : 2;
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
-}
 
 template <int MODE>
 btx_status launch_tc(const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0, const CUtensorMap& b1,
@@ -625,8 +415,6 @@ btx_status launch_tc(const CUtensorMap& a0, const CUtensorMap& a1, const CUtenso
   tc_gemm_kernel<MODE><<<2 * pairs, TC_THREADS, SMEM_BYTES, st>>>(a0, a1, b0, b1, p);   // cluster dims are compiled in
   return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
 }
-
-bool aligned32(const void* p) { return ((uintptr_t)p & 31) == 0; }
 
 TcParams base_params(const Plan& pl, const Buffers& b) {
   TcParams p = {};

@@ -389,19 +389,22 @@ template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16*
   *reinterpret_cast<uint2*>(p) = q;
 }
 
-// y[t, :] = sum_slot rows[t*k + slot, :]   (+ sum_e dz[t,e] * wr[e, :] when dz != nullptr)
+// y[t, :] = sum_slot sum_split rows[split][t*k + slot, :]   (+ sum_e dz[t,e] * wr[e, :] when dz != nullptr)
 template <typename T>
 __global__ void __launch_bounds__(256)
-combine_kernel(int Tn, int d, int k, int E, const float* __restrict__ rows, const float* __restrict__ dz,
+combine_kernel(int Tn, int d, int k, int E, int splits, const float* __restrict__ rows, const float* __restrict__ dz,
                const T* __restrict__ wr, T* __restrict__ y) {
+  const size_t split_stride = (size_t)Tn * k * d;
   const int vecs = d >> 2;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)Tn * vecs;
        i += (size_t)gridDim.x * blockDim.x) {
     int t = (int)(i / vecs), c = (int)(i % vecs) * 4;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < k; ++s) {
-      float4 v = *reinterpret_cast<const float4*>(rows + ((size_t)t * k + s) * d + c);
-      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      for (int sp = 0; sp < splits; ++sp) {
+        float4 v = *reinterpret_cast<const float4*>(rows + sp * split_stride + ((size_t)t * k + s) * d + c);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
     }
     if (dz != nullptr) {
       for (int e = 0; e < E; ++e) {
@@ -578,14 +581,14 @@ cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted
   return cudaGetLastError();
 }
 
-cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, void* y, cudaStream_t st) {
+cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, cudaStream_t st) {
   size_t n = (size_t)pl.T * (pl.d / 4);
   int blocks = (int)min((n + 255) / 256, (size_t)148 * 32);
   if (dtype == BTX_BF16)
-    combine_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, rows, nullptr, nullptr,
+    combine_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr,
                                                           (__nv_bfloat16*)y);
   else
-    combine_kernel<float><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, rows, nullptr, nullptr, (float*)y);
+    combine_kernel<float><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr, (float*)y);
   return cudaGetLastError();
 }
 
@@ -604,12 +607,12 @@ cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float
   if (dtype == BTX_BF16) {
     router_dw_partial_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(pl.T, pl.d, pl.E, (const __nv_bfloat16*)x, b.dz,
                                                                   b.dwr_part, bias_part);
-    combine_kernel<__nv_bfloat16><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, b.dxp, b.dz,
+    combine_kernel<__nv_bfloat16><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, 1, b.dxp, b.dz,
                                                            (const __nv_bfloat16*)w_router, (__nv_bfloat16*)dx);
   } else {
     router_dw_partial_kernel<float><<<grid, 256, 0, st>>>(pl.T, pl.d, pl.E, (const float*)x, b.dz, b.dwr_part,
                                                           bias_part);
-    combine_kernel<float><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, b.dxp, b.dz, (const float*)w_router,
+    combine_kernel<float><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, 1, b.dxp, b.dz, (const float*)w_router,
                                                    (float*)dx);
   }
   router_dw_reduce_kernel<<<(pl.E * pl.d + 255) / 256, 256, 0, st>>>(pl.d, pl.E, pl.wr_chunks, b.dwr_part, bias_part,
