@@ -45,6 +45,53 @@ template <> struct Vec<__nv_bfloat16> {
 // ---------------------------------------------------------------------------------------------
 // Router
 // ---------------------------------------------------------------------------------------------
+// Selection, gates and softmax for one token from the logits z[0..E) in shared memory (all lanes of
+// the calling warp take part).  On return lane e (< E) holds the dense gate and probability of expert e.
+__device__ __forceinline__ void route_select(int t, int E, int k, int routing, const float* z, int lane,
+                                             float* __restrict__ logits, int32_t* __restrict__ topk,
+                                             float* __restrict__ gates, float* __restrict__ probs, float& my_g,
+                                             float& my_p) {
+  uint32_t taken = 0;
+  int sel[kMaxExperts];
+  int first = 0;
+  // repeated arg-max: strict '>' keeps the lower index on ties
+  for (int j = 0; j < k; ++j) {
+    int best = -1;
+    float zb = 0.f;
+    for (int e = 0; e < E; ++e) {
+      if ((taken >> e) & 1u) continue;
+      float ze = z[e];
+      if (best < 0 || ze > zb) { best = e; zb = ze; }
+    }
+    taken |= 1u << best;
+    sel[j] = best;
+    if (j == 0) first = best;
+  }
+  const float zmax = z[first];
+  float psum = 0.f;
+  for (int e = 0; e < E; ++e) psum += expf(z[e] - zmax);
+  my_p = (lane < E) ? expf(z[lane] - zmax) / psum : 0.f;
+  my_g = 0.f;
+  if (routing == BTX_ROUTE_SWITCH) {
+    float g0 = expf(z[first] - zmax) / psum;
+    if (lane == first) my_g = g0;
+    if (lane == 0) { topk[t] = first; gates[t] = g0; }
+  } else {
+    float gsum = 0.f;
+    for (int j = 0; j < k; ++j) gsum += expf(z[sel[j]] - zmax);
+    for (int j = 0; j < k; ++j) {
+      float gj = expf(z[sel[j]] - zmax) / gsum;
+      if (sel[j] == lane) my_g = gj;
+      if (lane == 0) { topk[(size_t)t * k + j] = sel[j]; gates[(size_t)t * k + j] = gj; }
+    }
+  }
+  if (lane < E) {
+    probs[(size_t)t * E + lane] = my_p;
+    logits[(size_t)t * E + lane] = z[lane];
+  }
+  __syncwarp();
+}
+
 // Routing of one token by one warp: logits (or the given ones), top-k by repeated arg-max with
 // ties to the lower index, gates, full softmax.  `z` is this warp's shared scratch of kMaxExperts
 // floats.  On return lane e (< E) holds the dense gate and the probability of expert e.
@@ -88,46 +135,7 @@ __device__ __forceinline__ void route_token(int t, int d, int E, int k, int rout
     }
   }
   __syncwarp();
-  // Every lane runs the same selection on the shared logits; lane 0 writes the results.
-  uint32_t taken = 0;
-  int sel[kMaxExperts];
-  int first = 0;
-  // repeated arg-max: strict '>' keeps the lower index on ties
-  for (int j = 0; j < k; ++j) {
-    int best = -1;
-    float zb = 0.f;
-    for (int e = 0; e < E; ++e) {
-      if ((taken >> e) & 1u) continue;
-      float ze = z[e];
-      if (best < 0 || ze > zb) { best = e; zb = ze; }
-    }
-    taken |= 1u << best;
-    sel[j] = best;
-    if (j == 0) first = best;
-  }
-  const float zmax = z[first];
-  float psum = 0.f;
-  for (int e = 0; e < E; ++e) psum += expf(z[e] - zmax);
-  my_p = (lane < E) ? expf(z[lane] - zmax) / psum : 0.f;
-  my_g = 0.f;
-  if (routing == BTX_ROUTE_SWITCH) {
-    float g0 = expf(z[first] - zmax) / psum;
-    if (lane == first) my_g = g0;
-    if (lane == 0) { topk[t] = first; gates[t] = g0; }
-  } else {
-    float gsum = 0.f;
-    for (int j = 0; j < k; ++j) gsum += expf(z[sel[j]] - zmax);
-    for (int j = 0; j < k; ++j) {
-      float gj = expf(z[sel[j]] - zmax) / gsum;
-      if (sel[j] == lane) my_g = gj;
-      if (lane == 0) { topk[(size_t)t * k + j] = sel[j]; gates[(size_t)t * k + j] = gj; }
-    }
-  }
-  if (lane < E) {
-    probs[(size_t)t * E + lane] = my_p;
-    logits[(size_t)t * E + lane] = z[lane];
-  }
-  __syncwarp();
+  route_select(t, E, k, routing, z, lane, logits, topk, gates, probs, my_g, my_p);
 }
 
 template <typename T>
@@ -276,56 +284,106 @@ perm_scatter_kernel(int R, int E, int nblocks, const int32_t* __restrict__ topk,
 }
 
 // ---------------------------------------------------------------------------------------------
-// Small batches (R = T*k <= 1024, e.g. decoding): router, loss and permutation in ONE block, so the
-// step costs one launch instead of six.  Same results as the kernels above; the batch means are
-// summed per warp and then over the 32 warps in warp order.
+// Small batches (R = T*k <= 1024, e.g. decoding): router, loss and permutation in ONE launch
+// instead of six.  (The workspace status block is zeroed at the start of every forward call; its
+// word 8 is the ticket counter.)
 // ---------------------------------------------------------------------------------------------
-constexpr int kSmallThreads = 1024;
+constexpr int kSmallThreads = 256;
 constexpr int kSmallMaxR = 1024;
 
+// One block per token computes its logits (eight warps share the row) and routes it; the block that
+// finishes last (a ticket counter in the workspace status block) then forms u, p, the loss and the
+// permutation.  Every sum runs in a fixed order, so results do not depend on which block is last.
 template <typename T>
 __global__ void __launch_bounds__(kSmallThreads)
 route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha, int mt_max, int r_pad_max,
                            const T* __restrict__ x, const T* __restrict__ wr, const float* __restrict__ bias,
-                           float* __restrict__ logits, int32_t* __restrict__ topk, float* __restrict__ gates,
-                           float* __restrict__ probs, float* __restrict__ u, float* __restrict__ p,
-                           float* __restrict__ loss, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
-                           int32_t* __restrict__ pad_offsets, int32_t* __restrict__ tile_expert,
-                           int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
-                           int32_t* __restrict__ flat2row) {
+                           float* logits, int32_t* topk, float* gates, float* probs, float* __restrict__ u,
+                           float* __restrict__ p, float* __restrict__ loss, int32_t* __restrict__ counts,
+                           int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
+                           int32_t* __restrict__ tile_expert, int32_t* __restrict__ perm,
+                           int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
+                           int32_t* __restrict__ flat2row, int32_t* ticket) {
   constexpr int NW = kSmallThreads / 32;
-  __shared__ float zs[NW][kMaxExperts];
-  __shared__ float red[NW][kMaxExperts][2];
+  constexpr int VN = Vec<T>::N;
+  __shared__ float part[NW][kMaxExperts];
+  __shared__ float z[kMaxExperts];
   __shared__ double su[kMaxExperts], sp[kMaxExperts];
+  __shared__ int hist[kMaxExperts + 1], running[kMaxExperts + 1], soff[kMaxExperts + 1], spad[kMaxExperts + 1];
   __shared__ int wcnt[NW][kMaxExperts + 1];
-  __shared__ int soff[kMaxExperts + 1], spad[kMaxExperts + 1];
+  __shared__ int is_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x;
   const int R = Tn * k;
 
-  float u_acc = 0.f, p_acc = 0.f;
-  for (int t = warp; t < Tn; t += NW) {
+  const T* xr = x + (size_t)t * d;
+  for (int eb = 0; eb < E; eb += 8) {
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+#pragma unroll 2
+    for (int c = (warp * 32 + lane) * VN; c < d; c += NW * 32 * VN) {
+      float xv[VN];
+      Vec<T>::load(xr + c, xv);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (eb + j < E) {
+          float wv[VN];
+          Vec<T>::load(wr + (size_t)(eb + j) * d + c, wv);
+#pragma unroll
+          for (int v = 0; v < VN; ++v) acc[j] = fmaf(xv[v], wv[v], acc[j]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      float a = acc[j];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+      if (lane == 0 && eb + j < E) part[warp][eb + j] = a;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < E) {
+    float a = 0.f;
+    for (int w = 0; w < NW; ++w) a += part[w][threadIdx.x];
+    z[threadIdx.x] = a + (bias ? bias[threadIdx.x] : 0.f);
+  }
+  __syncthreads();
+  if (warp == 0) {
     float my_g, my_p;
-    route_token<T>(t, d, E, k, routing, x, wr, bias, nullptr, zs[warp], lane, logits, topk, gates, probs, my_g, my_p);
-    u_acc += my_g;
-    p_acc += my_p;
+    route_select(t, E, k, routing, z, lane, logits, topk, gates, probs, my_g, my_p);
   }
-  if (lane < E) { red[warp][lane][0] = u_acc; red[warp][lane][1] = p_acc; }
-  for (int j = threadIdx.x; j < NW * (kMaxExperts + 1); j += kSmallThreads) (&wcnt[0][0])[j] = 0;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+
+  // ---- last block: batch means, loss ----
+  for (int e = warp; e < E; e += NW) {
+    double du = 0.0, dp = 0.0;
+    for (int tt = lane; tt < Tn; tt += 32) {
+      dp += (double)__ldcg(probs + (size_t)tt * E + e);
+      for (int sl = 0; sl < k; ++sl)
+        if (__ldcg(topk + (size_t)tt * k + sl) == e) du += (double)__ldcg(gates + (size_t)tt * k + sl);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      du += __shfl_xor_sync(0xffffffffu, du, o);
+      dp += __shfl_xor_sync(0xffffffffu, dp, o);
+    }
+    if (lane == 0) {
+      du /= (double)Tn; dp /= (double)Tn;
+      su[e] = du; sp[e] = dp; u[e] = (float)du; p[e] = (float)dp;
+    }
+  }
+  // ---- permutation: histogram, scan, stable scatter in rounds of one block ----
+  if (threadIdx.x <= kMaxExperts) hist[threadIdx.x] = 0;
   for (int j = threadIdx.x; j < r_pad_max; j += kSmallThreads) rowmap[j] = -1;
-  __syncthreads();                                   // also orders the topk writes before the reads below
-  if (threadIdx.x < 2 * E) {
-    const int e = threadIdx.x >> 1, which = threadIdx.x & 1;
-    double s = 0.0;
-    for (int w = 0; w < NW; ++w) s += (double)red[w][e][which];
-    s /= (double)Tn;
-    if (which) { sp[e] = s; p[e] = (float)s; } else { su[e] = s; u[e] = (float)s; }
-  }
-  // stable counting sort of the R assignments by expert
-  const int i = threadIdx.x;
-  const int e = (i < R) ? topk[i] : E;               // E = dummy bucket for idle lanes
-  const unsigned same = __match_any_sync(0xffffffffu, e);
-  const int rank = __popc(same & ((1u << lane) - 1u));
-  if (rank == 0) wcnt[warp][e] = __popc(same);
+  __syncthreads();
+  for (int i = threadIdx.x; i < R; i += kSmallThreads) atomicAdd(&hist[__ldcg(topk + i)], 1);
   __syncthreads();
   if (threadIdx.x == 0) {
     double acc = 0.0;
@@ -333,28 +391,44 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
     loss[0] = (float)((double)alpha * (double)E * acc);
     int o = 0, po = 0;
     for (int q = 0; q < E; ++q) {
-      int c = 0;
-      for (int w = 0; w < NW; ++w) c += wcnt[w][q];
-      counts[q] = c; offsets[q] = o; pad_offsets[q] = po; soff[q] = o; spad[q] = po;
+      const int c = hist[q];
+      counts[q] = c; offsets[q] = o; pad_offsets[q] = po; soff[q] = o; spad[q] = po; running[q] = 0;
       o += c;
       po += (c + kRowTile - 1) / kRowTile * kRowTile;
     }
     offsets[E] = o; pad_offsets[E] = po; soff[E] = o; spad[E] = po;
   }
   __syncthreads();
-  if (i < R) {
-    int before = 0;
-    for (int w = 0; w < warp; ++w) before += wcnt[w][e];
-    const int within = before + rank;
-    const int r = soff[e] + within, rp = spad[e] + within;
-    perm[r] = i; inv_perm[i] = r; rowmap[rp] = i; flat2row[i] = rp;
-  }
   for (int mt = threadIdx.x; mt < mt_max; mt += kSmallThreads) {
     const int row = mt * kRowTile;
     int ex = -1;
     for (int q = 0; q < E; ++q)
       if (row >= spad[q] && row < spad[q + 1]) ex = q;
     tile_expert[mt] = ex;
+  }
+  for (int r0 = 0; r0 < R; r0 += kSmallThreads) {
+    for (int j = threadIdx.x; j < NW * (kMaxExperts + 1); j += kSmallThreads) (&wcnt[0][0])[j] = 0;
+    __syncthreads();
+    const int i = r0 + threadIdx.x;
+    const int e = (i < R) ? __ldcg(topk + i) : E;       // E = dummy bucket for idle lanes
+    const unsigned same = __match_any_sync(0xffffffffu, e);
+    const int rank = __popc(same & ((1u << lane) - 1u));
+    if (rank == 0) wcnt[warp][e] = __popc(same);
+    __syncthreads();
+    if (i < R) {
+      int before = 0;
+      for (int w = 0; w < warp; ++w) before += wcnt[w][e];
+      const int within = running[e] + before + rank;
+      const int r = soff[e] + within, rp = spad[e] + within;
+      perm[r] = i; inv_perm[i] = r; rowmap[rp] = i; flat2row[i] = rp;
+    }
+    __syncthreads();
+    if (threadIdx.x < E) {
+      int sum = 0;
+      for (int w = 0; w < NW; ++w) sum += wcnt[w][threadIdx.x];
+      running[threadIdx.x] += sum;
+    }
+    __syncthreads();
   }
 }
 
@@ -549,15 +623,15 @@ bool route_permute_small_fits(const Plan& pl) { return pl.R <= kSmallMaxR; }
 cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, float alpha, const void* x,
                                        const void* w_router, const float* bias, const Buffers& b, cudaStream_t st) {
   if (dtype == BTX_BF16)
-    route_permute_small_kernel<__nv_bfloat16><<<1, kSmallThreads, 0, st>>>(
+    route_permute_small_kernel<__nv_bfloat16><<<pl.T, kSmallThreads, 0, st>>>(
         pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, (const __nv_bfloat16*)x,
         (const __nv_bfloat16*)w_router, bias, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets,
-        b.pad_offsets, b.tile_expert, b.perm, b.inv_perm, b.rowmap, b.flat2row);
+        b.pad_offsets, b.tile_expert, b.perm, b.inv_perm, b.rowmap, b.flat2row, b.status + 8);
   else
-    route_permute_small_kernel<float><<<1, kSmallThreads, 0, st>>>(
+    route_permute_small_kernel<float><<<pl.T, kSmallThreads, 0, st>>>(
         pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, (const float*)x, (const float*)w_router, bias,
         b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets, b.pad_offsets, b.tile_expert, b.perm,
-        b.inv_perm, b.rowmap, b.flat2row);
+        b.inv_perm, b.rowmap, b.flat2row, b.status + 8);
   return cudaGetLastError();
 }
 
