@@ -179,7 +179,8 @@ def barrier(world):
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    torch.cuda.synchronize()
+    if torch.cuda.is_available():
+        torch.cuda.synchronize()
 
 
 def max_over_ranks(value, world, device):
@@ -190,6 +191,13 @@ def max_over_ranks(value, world, device):
     t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def aggregate_throughput(units_per_rank, ms_local, world, device):
+    """Whole-job units/s of N independent replicas: every rank processed `units_per_rank` in its own
+    `ms_local`; the job took the slowest rank's time."""
+    ms = max_over_ranks(ms_local, world, device)
+    return units_per_rank * world / (ms * 1e-3), ms
 
 
 def run_moe(args, workload):

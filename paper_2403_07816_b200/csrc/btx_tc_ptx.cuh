@@ -199,7 +199,7 @@ inline EncodeTiledFn encode_fn() {
 
 // bf16 tensor [rows, cols] (2D) or [E, rows, cols] (3D), cols contiguous; box = (box_cols, box_rows[, 1])
 inline bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t experts, uint32_t box_cols,
-              uint32_t box_rows) {
+              uint32_t box_rows, CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {cols, rows, experts};
@@ -208,7 +208,7 @@ inline bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t r
   cuuint32_t estr[3] = {1, 1, 1};
   const cuuint32_t rank = experts > 0 ? 3 : 2;
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
