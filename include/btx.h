@@ -53,6 +53,8 @@ typedef struct {
   float   lb_alpha;           /* alpha of the load-balancing loss (Section 3.3; 0.01 in 4.1.1) */
   int32_t lb_stopgrad_u;      /* 0: differentiate L_LB through u and p as printed; 1: u const  */
   int32_t save_for_backward;  /* forward fills `saved` so that btx_moe_backward can run        */
+  int32_t skip_wgrad;         /* backward: experts frozen (the paper's freeze ablation, Section */
+                              /* 4.3.1): no dW1/dW3/dW2, only dx and the router gradients       */
 } btx_moe_desc;
 
 /* Optional routing outputs of btx_moe_forward; any member may be NULL.  All device pointers.
@@ -94,7 +96,8 @@ btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, const void* 
  * Sections 1 and 3.2; the loss is added to the training loss with weight 1, Section 3.3).
  * `saved` is the buffer the forward call filled with the same desc and inputs.
  * Outputs: dx[T,d] (dtype); dw_router[E,d], dbias[E] (may be NULL), dw1,dw3[E,F,d], dw2[E,d,F],
- * all fp32.  accumulate = 0 overwrites the weight gradients, 1 adds to them. */
+ * all fp32.  accumulate = 0 overwrites the weight gradients, 1 adds to them.  With desc.skip_wgrad
+ * the three expert gradients are not computed and dw1, dw3, dw2 may be NULL. */
 btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void* w_router,
                             const float* router_bias, const void* w1, const void* w3, const void* w2,
                             const void* dy, float lb_grad_scale, const void* saved,

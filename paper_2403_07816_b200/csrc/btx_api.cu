@@ -216,9 +216,10 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
   Plan pl;
   btx_status s = make_plan(desc, &pl, false);
   if (s != BTX_OK) return s;
-  if (!x || !w_router || !w1 || !w3 || !w2 || !dy || !saved || !dx || !dw_router || !dw1 || !dw3 || !dw2 ||
-      !workspace)
+  const int skip_wgrad = desc->skip_wgrad != 0;
+  if (!x || !w_router || !w1 || !w3 || !w2 || !dy || !saved || !dx || !dw_router || !workspace)
     return BTX_ERR_INVALID_ARG;
+  if (!skip_wgrad && (!dw1 || !dw3 || !dw2)) return BTX_ERR_INVALID_ARG;
   if (misaligned(x) || misaligned(w_router) || misaligned(w1) || misaligned(w3) || misaligned(w2) ||
       misaligned(dy) || misaligned(saved) || misaligned(dx) || misaligned(dw_router) || misaligned(dw1) ||
       misaligned(dw3) || misaligned(dw2) || misaligned(workspace))
@@ -234,9 +235,10 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
   BTX_CUDA_OK(launch_gather_rows(pl, dy, b.dys, b, st));
   mark_stage(1, st);
   if (desc->dtype == BTX_F32) {
-    BTX_CUDA_OK(launch_expert_backward_f32(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, st));
+    BTX_CUDA_OK(launch_expert_backward_f32(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, skip_wgrad, st));
   } else {
-    if ((s = launch_expert_backward_bf16(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, st)) != BTX_OK) return s;
+    if ((s = launch_expert_backward_bf16(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, skip_wgrad, st)) != BTX_OK)
+      return s;
   }
   BTX_CUDA_OK(launch_router_backward(pl, desc->dtype, desc->routing, desc->lb_alpha, lb_grad_scale,
                                      desc->lb_stopgrad_u, 1, x, w_router, b, dx, dw_router, dbias, nullptr,

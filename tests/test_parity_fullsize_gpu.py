@@ -19,7 +19,7 @@ TOL = 1e-2
 ALPHA = 0.01
 
 
-def full_size_case(T, k, seed, routing=B.ROUTE_TOPK, bias=None, backward=True, n_tok=192, n_hidden=24):
+def full_size_case(T, k, seed, routing=B.ROUTE_TOPK, bias=None, backward=True, n_tok=192, n_hidden=24, F=F, E=E):
     inp = synth.moe_inputs(T, D, F, E, seed, torch.bfloat16, DEV, with_dy=backward)
     fwd = gpu_forward(inp, k, routing, ALPHA, bias, save=backward)
     r = fwd["routing"]
@@ -101,6 +101,13 @@ def test_skewed_top2_T16384_seed3():
     bias = synth.skew_bias(E, DEV)
     counts = full_size_case(16384, 2, seed=3, bias=bias, n_tok=128, n_hidden=16)
     assert counts[0] > 0.4 * 32768                                        # expert 0 takes the largest share
+
+
+def test_split_expert_shapes_E8():
+    # "Splitting experts" (Section 3.3): each FFN cut into two chunks of d_ff/2 gives 8 modules;
+    # the paper trains top-4 of 8; top-2 of 8 exercises sparser loads
+    full_size_case(4096, 4, seed=5, F=5504, E=8, n_tok=96, n_hidden=12)
+    full_size_case(4096, 2, seed=6, F=5504, E=8, n_tok=96, n_hidden=12)
 
 
 def test_decode_shaped_T32_two_layers_seed4():

@@ -95,6 +95,18 @@ def test_tied_logits_go_to_lower_index_and_identical_experts(dtype):
     assert rel_err(np64(fwd["y"]), dense) <= TOL[dtype]
 
 
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
+def test_frozen_experts_skip_weight_gradients(dtype):
+    # the paper's freeze ablation: only dx and the router gradients are produced
+    for T in (96, 700):                                   # small-batch and multi-block routing paths
+        inp = synth.moe_inputs(T, 64, 72, 4, 12, dtype, DEV)
+        fwd = gpu_forward(inp, 2, alpha=0.05, skip_wgrad=True)
+        cpu, b64, z_gpu, _ = check_forward(inp, fwd, 2, B.ROUTE_TOPK, 0.05, None, TOL[dtype])
+        got = gpu_backward(inp, fwd)
+        assert got["dw1"] is None
+        check_backward(cpu, b64, z_gpu, got, 2, B.ROUTE_TOPK, 0.05, 1.0, False, TOL[dtype])
+
+
 def test_results_are_deterministic_across_runs():
     inp = synth.moe_inputs(256, 256, 688, 4, 0, torch.float32, DEV)
     a = gpu_forward(inp, 2)

@@ -20,11 +20,11 @@ def rel_err(got, ref):
     return float(np.max(np.abs(got - ref)) / denom)
 
 
-def gpu_forward(inp, k, routing=B.ROUTE_TOPK, alpha=0.01, bias=None, save=True, stopgrad_u=False):
+def gpu_forward(inp, k, routing=B.ROUTE_TOPK, alpha=0.01, bias=None, save=True, stopgrad_u=False, skip_wgrad=False):
     x = inp["x"]
     T, d = x.shape
     E, F, _ = inp["w1"].shape
-    desc = B.make_desc(T, d, F, E, k, x.dtype, routing, alpha, stopgrad_u, save)
+    desc = B.make_desc(T, d, F, E, k, x.dtype, routing, alpha, stopgrad_u, save, skip_wgrad)
     ws, saved = B.alloc_buffers(desc, x.device)
     ws.fill_(0x7F)           # poison: results must not depend on scratch contents
     saved.fill_(0x7F)
@@ -42,7 +42,11 @@ def gpu_backward(inp, fwd, lb_scale=1.0, bias=None, accumulate=False, init=None)
     dev = x.device
     mk = (lambda *s: torch.full(s, init, dtype=torch.float32, device=dev)) if init is not None else \
          (lambda *s: torch.empty(s, dtype=torch.float32, device=dev))
-    out = dict(dx=torch.empty_like(x), dw_router=mk(E, d), dbias=mk(E), dw1=mk(E, F, d), dw3=mk(E, F, d), dw2=mk(E, d, F))
+    out = dict(dx=torch.empty_like(x), dw_router=mk(E, d), dbias=mk(E))
+    if desc.skip_wgrad:
+        out.update(dw1=None, dw3=None, dw2=None)
+    else:
+        out.update(dw1=mk(E, F, d), dw3=mk(E, F, d), dw2=mk(E, d, F))
     fwd["ws"].fill_(0x7F)
     B.btx_moe_backward(desc, x, inp["w_router"], bias, inp["w1"], inp["w3"], inp["w2"], inp["dy"], lb_scale,
                        fwd["saved"], out["dx"], out["dw_router"], out["dbias"], out["dw1"], out["dw3"], out["dw2"],
@@ -84,6 +88,8 @@ def check_backward(cpu, b64, z_gpu, got, k, routing, alpha, lb_scale, stopgrad_u
                          lb_scale, stopgrad_u, router_bias=b64, logits=z_gpu)
     errs = {}
     for name in ("dx", "dw_router", "dbias", "dw1", "dw3", "dw2"):
+        if got[name] is None:
+            continue
         want = ref[name] if base is None or name == "dx" else ref[name] + base
         errs[name] = rel_err(np64(got[name]), want)
     bad = {n: e for n, e in errs.items() if e > tol}
