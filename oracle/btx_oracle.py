@@ -15,7 +15,7 @@ What each part follows (paper = arXiv 2403.07816):
                                                           Llama-2 seed, Section 4.1): SwiGLU
                                                           W2 (silu(W1 x) * W3 x), no biases
   * load-balancing loss ................................ Section 3.3, the L_LB equation
-  * Switch / soft routing .............................. Section 3.3, "Routing method"
+  * Switch / soft / Sample Top-1 routing ............... Section 3.3, "Routing method"
   * merge (stack FFNs, average the rest) ............... Section 3.2, the two paragraphs after
                                                           the routing formula
   * backward ........................................... derivatives of the above (MoE finetuning,
@@ -40,6 +40,7 @@ import numpy as np
 ROUTE_TOPK = 0
 ROUTE_SWITCH = 1
 ROUTE_SOFT = 2
+ROUTE_SAMPLE1 = 3
 
 _F64 = np.float64
 
@@ -188,13 +189,32 @@ def swiglu_ffn(x, w1, w3, w2, return_hidden=False):
 # MoE forward
 # --------------------------------------------------------------------------------------
 
-def route(x, w_router, k, routing=ROUTE_TOPK, router_bias=None, logits=None):
-    """Steps 1-4: logits (or the caller's fp32 logits), selection, gates, full softmax."""
+def route(x, w_router, k, routing=ROUTE_TOPK, router_bias=None, logits=None, noise=None, tau=1.0):
+    """Steps 1-4: logits (or the caller's fp32 logits), selection, gates, full softmax.
+
+    ROUTE_SAMPLE1 (Section 3.3, "Sample Top-1"): with Gumbel noise G (an input) the soft sample is
+    SoftMax((z + G) / tau); only its largest entry is kept as the gate of that one expert.  tau = 0
+    is the inference rule, hard sampling: the expert arg-max(z + G) with gate 1.  For this mode the
+    returned probabilities are those of the perturbed logits (the quantity the gate is taken from).
+    """
     z = router_logits(x, w_router, router_bias) if logits is None else _f64(logits)
     E = z.shape[1]
     kk = E if routing == ROUTE_SOFT else k
-    if routing == ROUTE_SWITCH and kk != 1:
-        raise ValueError("Switch routing needs k = 1")
+    if routing in (ROUTE_SWITCH, ROUTE_SAMPLE1) and kk != 1:
+        raise ValueError("Switch and Sample Top-1 routing need k = 1")
+    if routing == ROUTE_SAMPLE1:
+        if noise is None:
+            raise ValueError("Sample Top-1 routing needs the Gumbel noise")
+        zp = z + _f64(noise)
+        idx = top_k_select(zp, 1)
+        if tau > 0:
+            zp = zp / float(tau)
+            p = full_softmax(zp)
+            g = np.take_along_axis(p, idx.astype(np.int64), axis=1)
+        else:
+            p = full_softmax(zp)
+            g = np.ones((z.shape[0], 1), dtype=_F64)
+        return z, idx, g, p
     idx = top_k_select(z, kk)
     g = gate_values(z, idx, routing)
     p = full_softmax(z)
@@ -202,7 +222,7 @@ def route(x, w_router, k, routing=ROUTE_TOPK, router_bias=None, logits=None):
 
 
 def moe_forward(x, w_router, w1, w3, w2, k, routing=ROUTE_TOPK, alpha=0.01,
-                router_bias=None, logits=None, tokens=None):
+                router_bias=None, logits=None, tokens=None, noise=None, tau=1.0):
     """FF_MoE(x) = sum_i g_i(W_l x) FF_i(x), skipping experts whose gate is zero.
 
     w1, w3: [E, F, d]; w2: [E, d, F].  `logits` (optional, [T, E]) replaces W_l x so that the
@@ -213,7 +233,7 @@ def moe_forward(x, w_router, w1, w3, w2, k, routing=ROUTE_TOPK, alpha=0.01,
     x = _f64(x)
     T, d = x.shape
     E = np.asarray(w1).shape[0]
-    z, idx, g, p_tok = route(x, w_router, k, routing, router_bias, logits)
+    z, idx, g, p_tok = route(x, w_router, k, routing, router_bias, logits, noise, tau)
     gd = dense_gates(idx, g, E)
     loss, u, p = lb_loss(gd, p_tok, alpha)
     counts, offsets, perm, inv_perm = dispatch(idx, E)
@@ -278,13 +298,15 @@ def router_backward_dz(idx, gates, probs, dgate, u, alpha, lb_grad_scale, routin
 
 
 def moe_backward(x, w_router, w1, w3, w2, dy, k, routing=ROUTE_TOPK, alpha=0.01,
-                 lb_grad_scale=1.0, lb_stopgrad_u=False, router_bias=None, logits=None):
+                 lb_grad_scale=1.0, lb_stopgrad_u=False, router_bias=None, logits=None, noise=None, tau=1.0):
     """Gradients of  <Y, dY> + lb_grad_scale * L_LB  w.r.t. x, W_l, bias, W1, W3, W2 (all tokens)."""
     x = _f64(x)
     dy = _f64(dy)
     T, d = x.shape
     E, F, _ = np.asarray(w1).shape
-    z, idx, g, p_tok = route(x, w_router, k, routing, router_bias, logits)
+    z, idx, g, p_tok = route(x, w_router, k, routing, router_bias, logits, noise, tau)
+    if routing == ROUTE_SAMPLE1 and alpha != 0:
+        raise ValueError("Sample Top-1 routing is defined here without the load-balancing loss (alpha = 0)")
     kk = idx.shape[1]
     gd = dense_gates(idx, g, E)
     _, u, p = lb_loss(gd, p_tok, alpha)
@@ -316,7 +338,13 @@ def moe_backward(x, w_router, w1, w3, w2, dy, k, routing=ROUTE_TOPK, alpha=0.01,
     if not lb_stopgrad_u:
         # L_LB through u: d L_LB / d g[t,i] = alpha E p_i / T
         dgate += lb_grad_scale * alpha * E / T * p[idx.astype(np.int64)]
-    dz = router_backward_dz(idx, g, p_tok, dgate, u, alpha, lb_grad_scale, routing)
+    if routing == ROUTE_SAMPLE1:
+        # gate = SoftMax((z+G)/tau)[arg-max]: the Switch Jacobian in the perturbed logits, times 1/tau;
+        # hard sampling (tau = 0) has a constant gate, hence no router gradient
+        dz = (router_backward_dz(idx, g, p_tok, dgate, u, 0.0, 0.0, ROUTE_SWITCH) / float(tau)) if tau > 0 \
+            else np.zeros((T, E), dtype=_F64)
+    else:
+        dz = router_backward_dz(idx, g, p_tok, dgate, u, alpha, lb_grad_scale, routing)
     dw_router = dz.T @ x
     dbias = dz.sum(axis=0)
     dx += dz @ _f64(w_router)

@@ -395,3 +395,70 @@ def test_table4_active_parameter_counts():
     ffn = sum(int(np.prod(s)) for n, s in shapes if ".ffn." in n)
     other = sum(int(np.prod(s)) for n, s in shapes if ".ffn." not in n)
     assert ffn == 4_328_521_728 and other == 2_409_893_888
+
+
+# ---- Sample Top-1 routing (Gumbel softmax, keep the largest entry) ----------------------------
+
+def test_sample_top1_reduces_to_switch_without_noise():
+    x, wr, w1, w3, w2, dy = small_problem(21, scale_r=1.5)
+    zero = np.zeros((x.shape[0], 4))
+    a = o.moe_forward(x, wr, w1, w3, w2, k=1, routing=o.ROUTE_SWITCH, alpha=0.0)
+    b = o.moe_forward(x, wr, w1, w3, w2, k=1, routing=o.ROUTE_SAMPLE1, alpha=0.0, noise=zero, tau=1.0)
+    assert (a["topk_idx"] == b["topk_idx"]).all()
+    np.testing.assert_allclose(a["y"], b["y"], rtol=1e-13)
+    ga = o.moe_backward(x, wr, w1, w3, w2, dy, k=1, routing=o.ROUTE_SWITCH, alpha=0.0)
+    gb = o.moe_backward(x, wr, w1, w3, w2, dy, k=1, routing=o.ROUTE_SAMPLE1, alpha=0.0, noise=zero, tau=1.0)
+    np.testing.assert_allclose(ga["dw_router"], gb["dw_router"], rtol=1e-12, atol=1e-14)
+
+
+def test_sample_top1_selection_and_temperature_limits():
+    r = RNG(22)
+    x, wr, w1, w3, w2, _ = small_problem(22)
+    noise = -np.log(-np.log(r.uniform(size=(x.shape[0], 4))))
+    z = o.router_logits(x, wr)
+    out = o.moe_forward(x, wr, w1, w3, w2, k=1, routing=o.ROUTE_SAMPLE1, alpha=0.0, noise=noise, tau=0.7)
+    assert (out["topk_idx"][:, 0] == np.argmax(z + noise, axis=1)).all()
+    soft = np.exp((z + noise) / 0.7); soft /= soft.sum(1, keepdims=True)
+    np.testing.assert_allclose(out["gates"][:, 0], soft.max(axis=1), rtol=1e-13)   # the kept entry of the soft sample
+    np.testing.assert_allclose(out["logits"], z, rtol=1e-14)                        # reported logits are unperturbed
+    sharp = o.moe_forward(x, wr, w1, w3, w2, k=1, routing=o.ROUTE_SAMPLE1, alpha=0.0, noise=noise, tau=1e-3)
+    np.testing.assert_allclose(sharp["gates"], 1.0, atol=1e-6)                      # annealed: a sharp distribution
+    hard = o.moe_forward(x, wr, w1, w3, w2, k=1, routing=o.ROUTE_SAMPLE1, alpha=0.0, noise=noise, tau=0.0)
+    assert (hard["gates"] == 1.0).all() and (hard["topk_idx"] == out["topk_idx"]).all()
+    e = hard["topk_idx"][:, 0]
+    want = np.stack([o.swiglu_ffn(x[t:t + 1], w1[e[t]], w3[e[t]], w2[e[t]])[0] for t in range(x.shape[0])])
+    np.testing.assert_allclose(hard["y"], want, rtol=1e-12, atol=1e-13)
+
+
+def test_hard_sampling_follows_the_softmax_distribution():
+    # Gumbel-max: arg-max(z + G) is a draw from SoftMax(z)
+    r = RNG(23)
+    z = np.tile(np.array([[1.0, 0.0, -0.5, 2.0]]), (40000, 1))
+    noise = -np.log(-np.log(r.uniform(size=z.shape)))
+    _, idx, _, _ = o.route(None, None, 1, o.ROUTE_SAMPLE1, logits=z, noise=noise, tau=0.0)
+    freq = np.bincount(idx[:, 0], minlength=4) / z.shape[0]
+    np.testing.assert_allclose(freq, o.full_softmax(z[:1])[0], atol=0.01)
+
+
+def test_sample_top1_gradients_against_finite_differences():
+    x, wr, w1, w3, w2, G = small_problem(24, T=10, d=6, F=7, E=4, scale_r=1.5)
+    r = RNG(25)
+    noise = -np.log(-np.log(r.uniform(size=(10, 4))))
+    tau = 0.8
+    zs = np.sort(o.router_logits(x, wr) + noise, axis=1)
+    assert np.min(np.diff(zs, axis=1)) > 1e-3
+    g = o.moe_backward(x, wr, w1, w3, w2, G, k=1, routing=o.ROUTE_SAMPLE1, alpha=0.0, noise=noise, tau=tau)
+    f = lambda: float(np.sum(o.moe_forward(x, wr, w1, w3, w2, k=1, routing=o.ROUTE_SAMPLE1, alpha=0.0,
+                                           noise=noise, tau=tau)["y"] * G))
+    h = 1e-6
+    for arr, name in ((x, "dx"), (wr, "dw_router"), (w2, "dw2"), (w1, "dw1")):
+        for _ in range(6):
+            pos = tuple(int(r.integers(0, s)) for s in arr.shape)
+            old = arr[pos]
+            arr[pos] = old + h; lp = f()
+            arr[pos] = old - h; lm = f()
+            arr[pos] = old
+            fd = (lp - lm) / (2 * h)
+            assert abs(fd - g[name][pos]) <= 2e-6 * max(1.0, abs(fd)), (name, pos, fd, g[name][pos])
+    hard = o.moe_backward(x, wr, w1, w3, w2, G, k=1, routing=o.ROUTE_SAMPLE1, alpha=0.0, noise=noise, tau=0.0)
+    assert np.all(hard["dw_router"] == 0.0)
