@@ -43,8 +43,13 @@ typedef enum { BTX_F32 = 0, BTX_BF16 = 1 } btx_dtype;
  *   TOPK   g = softmax over the k largest logits, zero elsewhere (the paper's default, k = 2).
  *   SWITCH k = 1; the gate is the full-softmax probability of the arg-max expert.
  *   SOFT   g = softmax over all E experts (every expert active); desc.k is ignored.
+ *   SAMPLE1 "Sample Top-1": with the caller's Gumbel noise G[T,E] the soft sample is
+ *          SoftMax((W_l x + G) / desc.gumbel_tau); only its largest entry is kept as the gate of that
+ *          one expert (k = 1).  gumbel_tau = 0 is hard sampling, the paper's inference rule: expert
+ *          arg-max(W_l x + G) with gate 1 and no router gradient.  Defined here without the
+ *          load-balancing loss (lb_alpha must be 0); `probs` then holds the perturbed softmax.
  * Ties between equal logits go to the lower expert index; slot 0 holds the largest logit. */
-typedef enum { BTX_ROUTE_TOPK = 0, BTX_ROUTE_SWITCH = 1, BTX_ROUTE_SOFT = 2 } btx_routing;
+typedef enum { BTX_ROUTE_TOPK = 0, BTX_ROUTE_SWITCH = 1, BTX_ROUTE_SOFT = 2, BTX_ROUTE_SAMPLE1 = 3 } btx_routing;
 
 typedef struct {
   int32_t T, d_model, d_ff, E, k;
@@ -55,6 +60,7 @@ typedef struct {
   int32_t save_for_backward;  /* forward fills `saved` so that btx_moe_backward can run        */
   int32_t skip_wgrad;         /* backward: experts frozen (the paper's freeze ablation, Section */
                               /* 4.3.1): no dW1/dW3/dW2, only dx and the router gradients       */
+  float   gumbel_tau;         /* SAMPLE1 only: temperature of the Gumbel softmax; 0 = hard      */
 } btx_moe_desc;
 
 /* Optional routing outputs of btx_moe_forward; any member may be NULL.  All device pointers.
@@ -85,10 +91,12 @@ btx_status btx_moe_sizes(const btx_moe_desc* desc, size_t* workspace_bytes, size
 /* FF_MoE(x) = sum_i g_i(W_l x) FF_i(x)  (Section 3.2), FF_i(x) = W2_i (silu(W1_i x) * W3_i x),
  * evaluated only for the selected experts, plus the load-balancing loss of Section 3.3.
  *   x[T,d]; w_router[E,d] (W_l); router_bias[E] fp32 or NULL (the paper has no bias);
+ *   router_noise[T,E] fp32 Gumbel noise, required for BTX_ROUTE_SAMPLE1 and ignored otherwise;
  *   w1,w3[E,F,d]; w2[E,d,F]; y[T,d] out.  `routing` may be NULL.  `saved` may be NULL when
  *   desc.save_for_backward == 0.  d and F must be multiples of 8 in BF16 mode, of 4 in F32. */
 btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, const void* w_router,
-                           const float* router_bias, const void* w1, const void* w3, const void* w2,
+                           const float* router_bias, const float* router_noise,
+                           const void* w1, const void* w3, const void* w2,
                            void* y, const btx_routing_out* routing, void* saved,
                            void* workspace, size_t workspace_bytes, void* stream);
 
@@ -99,7 +107,8 @@ btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, const void* 
  * all fp32.  accumulate = 0 overwrites the weight gradients, 1 adds to them.  With desc.skip_wgrad
  * the three expert gradients are not computed and dw1, dw3, dw2 may be NULL. */
 btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void* w_router,
-                            const float* router_bias, const void* w1, const void* w3, const void* w2,
+                            const float* router_bias, const float* router_noise,
+                            const void* w1, const void* w3, const void* w2,
                             const void* dy, float lb_grad_scale, const void* saved,
                             void* dx, float* dw_router, float* dbias,
                             float* dw1, float* dw3, float* dw2, int32_t accumulate,
@@ -115,7 +124,7 @@ btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void*
 btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_host, const void* dy_host,
                              void* y_host, void* dx_host, float* loss_host,
                              void* x_dev, void* dy_dev, void* y_dev, void* dx_dev,
-                             const void* w_router, const float* router_bias,
+                             const void* w_router, const float* router_bias, const float* router_noise,
                              const void* w1, const void* w3, const void* w2, float lb_grad_scale,
                              float* dw_router, float* dbias, float* dw1, float* dw3, float* dw2,
                              int32_t accumulate, void* saved, void* workspace, size_t workspace_bytes,

@@ -14,7 +14,7 @@ import torch
 
 BTX_OK = 0
 BTX_F32, BTX_BF16 = 0, 1
-ROUTE_TOPK, ROUTE_SWITCH, ROUTE_SOFT = 0, 1, 2
+ROUTE_TOPK, ROUTE_SWITCH, ROUTE_SOFT, ROUTE_SAMPLE1 = 0, 1, 2, 3
 PARAM_AVERAGE, PARAM_FFN = 0, 1
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbtx.so")
@@ -31,7 +31,8 @@ class BtxError(RuntimeError):
 class MoeDesc(C.Structure):
     _fields_ = [("T", C.c_int32), ("d_model", C.c_int32), ("d_ff", C.c_int32), ("E", C.c_int32), ("k", C.c_int32),
                 ("dtype", C.c_int32), ("routing", C.c_int32), ("lb_alpha", C.c_float),
-                ("lb_stopgrad_u", C.c_int32), ("save_for_backward", C.c_int32), ("skip_wgrad", C.c_int32)]
+                ("lb_stopgrad_u", C.c_int32), ("save_for_backward", C.c_int32), ("skip_wgrad", C.c_int32),
+                ("gumbel_tau", C.c_float)]
 
 
 class RoutingOut(C.Structure):
@@ -57,11 +58,11 @@ def lib():
         L = C.CDLL(LIB_PATH)
         vp, i32, f32, sz = C.c_void_p, C.c_int32, C.c_float, C.c_size_t
         L.btx_moe_sizes.argtypes = [C.POINTER(MoeDesc), C.POINTER(sz), C.POINTER(sz)]
-        L.btx_moe_forward.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, C.POINTER(RoutingOut), vp, vp,
+        L.btx_moe_forward.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, vp, C.POINTER(RoutingOut), vp, vp,
                                       sz, vp]
-        L.btx_moe_backward.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp,
-                                       i32, vp, sz, vp]
-        L.btx_moe_step_host.argtypes = [C.POINTER(MoeDesc)] + [vp] * 14 + [f32] + [vp] * 5 + [i32, vp, vp, sz, vp]
+        L.btx_moe_backward.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp, vp,
+                                       vp, i32, vp, sz, vp]
+        L.btx_moe_step_host.argtypes = [C.POINTER(MoeDesc)] + [vp] * 15 + [f32] + [vp] * 5 + [i32, vp, vp, sz, vp]
         L.btx_set_stage_events.argtypes = [C.POINTER(vp), i32]
         L.btx_lb_loss_workspace_size.argtypes = [C.POINTER(MoeDesc), C.POINTER(sz)]
         L.btx_lb_loss.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, sz, vp]
@@ -102,10 +103,10 @@ def _stream(device):
 
 
 def make_desc(T, d_model, d_ff, E, k, dtype, routing=ROUTE_TOPK, lb_alpha=0.01, lb_stopgrad_u=False,
-              save_for_backward=False, skip_wgrad=False) -> MoeDesc:
+              save_for_backward=False, skip_wgrad=False, gumbel_tau=0.0) -> MoeDesc:
     code = _dtype_code(dtype) if isinstance(dtype, torch.dtype) else int(dtype)
     return MoeDesc(T, d_model, d_ff, E, k, code, routing, lb_alpha, int(lb_stopgrad_u), int(save_for_backward),
-                   int(skip_wgrad))
+                   int(skip_wgrad), float(gumbel_tau))
 
 
 def btx_moe_sizes(desc: MoeDesc):
@@ -153,9 +154,10 @@ def alloc_buffers(desc: MoeDesc, device):
             torch.empty(max(sv, 16), dtype=torch.uint8, device=device))
 
 
-def btx_moe_forward(desc, x, w_router, router_bias, w1, w3, w2, y, routing, saved, workspace):
+def btx_moe_forward(desc, x, w_router, router_bias, w1, w3, w2, y, routing, saved, workspace, router_noise=None):
     ro = routing.as_struct() if routing is not None else None
-    s = lib().btx_moe_forward(C.byref(desc), _ptr(x), _ptr(w_router), _ptr(router_bias), _ptr(w1), _ptr(w3), _ptr(w2),
+    s = lib().btx_moe_forward(C.byref(desc), _ptr(x), _ptr(w_router), _ptr(router_bias), _ptr(router_noise), _ptr(w1),
+                              _ptr(w3), _ptr(w2),
                               _ptr(y), C.byref(ro) if ro is not None else None, _ptr(saved), _ptr(workspace),
                               workspace.numel(), _stream(x.device))
     if s != BTX_OK:
@@ -163,8 +165,9 @@ def btx_moe_forward(desc, x, w_router, router_bias, w1, w3, w2, y, routing, save
 
 
 def btx_moe_backward(desc, x, w_router, router_bias, w1, w3, w2, dy, lb_grad_scale, saved, dx, dw_router, dbias,
-                     dw1, dw3, dw2, accumulate, workspace):
-    s = lib().btx_moe_backward(C.byref(desc), _ptr(x), _ptr(w_router), _ptr(router_bias), _ptr(w1), _ptr(w3), _ptr(w2),
+                     dw1, dw3, dw2, accumulate, workspace, router_noise=None):
+    s = lib().btx_moe_backward(C.byref(desc), _ptr(x), _ptr(w_router), _ptr(router_bias), _ptr(router_noise), _ptr(w1),
+                               _ptr(w3), _ptr(w2),
                                _ptr(dy), float(lb_grad_scale), _ptr(saved), _ptr(dx), _ptr(dw_router), _ptr(dbias),
                                _ptr(dw1), _ptr(dw3), _ptr(dw2), int(accumulate), _ptr(workspace), workspace.numel(),
                                _stream(x.device))
@@ -174,7 +177,7 @@ def btx_moe_backward(desc, x, w_router, router_bias, w1, w3, w2, dy, lb_grad_sca
 
 def btx_moe_step_host(desc, x_host, dy_host, y_host, dx_host, loss_host, x_dev, dy_dev, y_dev, dx_dev, w_router,
                       router_bias, w1, w3, w2, lb_grad_scale, dw_router, dbias, dw1, dw3, dw2, accumulate, saved,
-                      workspace):
+                      workspace, router_noise=None):
     """Forward + backward with activations in (pinned) host tensors; see btx.h."""
     for t in (x_host, dy_host, y_host, dx_host, loss_host):
         if t.is_cuda or not t.is_contiguous():
@@ -182,7 +185,8 @@ def btx_moe_step_host(desc, x_host, dy_host, y_host, dx_host, loss_host, x_dev, 
     hp = lambda t: C.c_void_p(t.data_ptr())
     s = lib().btx_moe_step_host(C.byref(desc), hp(x_host), hp(dy_host), hp(y_host), hp(dx_host), hp(loss_host),
                                 _ptr(x_dev), _ptr(dy_dev), _ptr(y_dev), _ptr(dx_dev), _ptr(w_router),
-                                _ptr(router_bias), _ptr(w1), _ptr(w3), _ptr(w2), float(lb_grad_scale),
+                                _ptr(router_bias), _ptr(router_noise), _ptr(w1), _ptr(w3), _ptr(w2),
+                                float(lb_grad_scale),
                                 _ptr(dw_router), _ptr(dbias), _ptr(dw1), _ptr(dw3), _ptr(dw2), int(accumulate),
                                 _ptr(saved), _ptr(workspace), workspace.numel(), _stream(x_dev.device))
     if s != BTX_OK:

@@ -15,10 +15,11 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   if (desc->T < 1 || desc->E < 1) return BTX_ERR_INVALID_ARG;
   if (!routing_only && (desc->d_model < 1 || desc->d_ff < 1)) return BTX_ERR_INVALID_ARG;
   if (desc->dtype != BTX_F32 && desc->dtype != BTX_BF16) return BTX_ERR_INVALID_ARG;
-  if (desc->routing < BTX_ROUTE_TOPK || desc->routing > BTX_ROUTE_SOFT) return BTX_ERR_INVALID_ARG;
+  if (desc->routing < BTX_ROUTE_TOPK || desc->routing > BTX_ROUTE_SAMPLE1) return BTX_ERR_INVALID_ARG;
   int k = desc->routing == BTX_ROUTE_SOFT ? desc->E : desc->k;
   if (k < 1 || k > desc->E) return BTX_ERR_INVALID_ARG;
-  if (desc->routing == BTX_ROUTE_SWITCH && k != 1) return BTX_ERR_INVALID_ARG;
+  if ((desc->routing == BTX_ROUTE_SWITCH || desc->routing == BTX_ROUTE_SAMPLE1) && k != 1) return BTX_ERR_INVALID_ARG;
+  if (desc->routing == BTX_ROUTE_SAMPLE1 && (desc->gumbel_tau < 0.f || desc->lb_alpha != 0.f)) return BTX_ERR_UNSUPPORTED;
   if (desc->E > kMaxExperts) return BTX_ERR_UNSUPPORTED;
   const int gran = desc->dtype == BTX_BF16 ? 8 : 4;         // rows must be whole 16-byte vectors
   if (!routing_only && (desc->d_model % gran || desc->d_ff % gran)) return BTX_ERR_UNSUPPORTED;
@@ -115,6 +116,15 @@ void mark_stage(int i, cudaStream_t st) {
     cudaEventRecord((cudaEvent_t)g_stage_events[i], st);
 }
 
+// Sample Top-1 is Switch routing (soft sample) or top-1 with gate 1 (hard sample) on the logits
+// perturbed by the Gumbel noise and divided by the temperature.
+struct EffectiveRouting { int routing; float inv_tau; };
+static EffectiveRouting effective_routing(const btx_moe_desc* desc) {
+  if (desc->routing != BTX_ROUTE_SAMPLE1) return {desc->routing, 1.0f};
+  if (desc->gumbel_tau > 0.f) return {BTX_ROUTE_SWITCH, 1.0f / desc->gumbel_tau};
+  return {BTX_ROUTE_TOPK, 1.0f};
+}
+
 static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
 
 static btx_status check_device() {
@@ -141,7 +151,8 @@ extern "C" btx_status btx_moe_sizes(const btx_moe_desc* desc, size_t* workspace_
 }
 
 extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, const void* w_router,
-                                      const float* router_bias, const void* w1, const void* w3, const void* w2,
+                                      const float* router_bias, const float* router_noise, const void* w1,
+                                      const void* w3, const void* w2,
                                       void* y, const btx_routing_out* routing, void* saved, void* workspace,
                                       size_t workspace_bytes, void* stream) {
   Plan pl;
@@ -149,6 +160,9 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
   if (s != BTX_OK) return s;
   if (!x || !w_router || !w1 || !w3 || !w2 || !y || !workspace) return BTX_ERR_INVALID_ARG;
   if (desc->save_for_backward && !saved) return BTX_ERR_INVALID_ARG;
+  if (desc->routing == BTX_ROUTE_SAMPLE1 && !router_noise) return BTX_ERR_INVALID_ARG;
+  const EffectiveRouting er = effective_routing(desc);
+  const float* noise = desc->routing == BTX_ROUTE_SAMPLE1 ? router_noise : nullptr;
   if (misaligned(x) || misaligned(w_router) || misaligned(w1) || misaligned(w3) || misaligned(w2) || misaligned(y) ||
       misaligned(workspace) || misaligned(saved))
     return BTX_ERR_INVALID_ARG;
@@ -164,11 +178,11 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
   mark_stage(0, st);
   BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
   if (route_permute_small_fits(pl)) {
-    BTX_CUDA_OK(launch_route_permute_small(pl, desc->dtype, desc->routing, desc->lb_alpha, x, w_router, router_bias, b,
-                                           st));
+    BTX_CUDA_OK(launch_route_permute_small(pl, desc->dtype, er.routing, desc->lb_alpha, x, w_router, router_bias, noise,
+                                           er.inv_tau, b, st));
   } else {
-    BTX_CUDA_OK(launch_router(pl, desc->dtype, desc->routing, desc->lb_alpha, x, w_router, router_bias, nullptr, b,
-                              st));
+    BTX_CUDA_OK(launch_router(pl, desc->dtype, er.routing, desc->lb_alpha, x, w_router, router_bias, nullptr, noise,
+                              er.inv_tau, b, st));
     BTX_CUDA_OK(launch_permute(pl, b, st));
   }
   BTX_CUDA_OK(launch_gather_rows(pl, x, b.xs, b, st));
@@ -208,11 +222,13 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
 }
 
 extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void* w_router,
-                                       const float* router_bias, const void* w1, const void* w3, const void* w2,
+                                       const float* router_bias, const float* router_noise, const void* w1,
+                                       const void* w3, const void* w2,
                                        const void* dy, float lb_grad_scale, const void* saved, void* dx,
                                        float* dw_router, float* dbias, float* dw1, float* dw3, float* dw2,
                                        int32_t accumulate, void* workspace, size_t workspace_bytes, void* stream) {
   (void)router_bias;   // the bias only shifts the logits; its gradient needs dz alone
+  (void)router_noise;  // likewise: the forward saved the perturbed probabilities
   Plan pl;
   btx_status s = make_plan(desc, &pl, false);
   if (s != BTX_OK) return s;
@@ -240,9 +256,10 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
     if ((s = launch_expert_backward_bf16(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, skip_wgrad, st)) != BTX_OK)
       return s;
   }
-  BTX_CUDA_OK(launch_router_backward(pl, desc->dtype, desc->routing, desc->lb_alpha, lb_grad_scale,
+  const EffectiveRouting er = effective_routing(desc);
+  BTX_CUDA_OK(launch_router_backward(pl, desc->dtype, er.routing, desc->lb_alpha, lb_grad_scale,
                                      desc->lb_stopgrad_u, 1, x, w_router, b, dx, dw_router, dbias, nullptr,
-                                     accumulate, st));
+                                     accumulate, er.inv_tau, st));
   mark_stage(7, st);
   return BTX_OK;
 }
@@ -250,7 +267,7 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
 extern "C" btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_host, const void* dy_host,
                                         void* y_host, void* dx_host, float* loss_host, void* x_dev, void* dy_dev,
                                         void* y_dev, void* dx_dev, const void* w_router, const float* router_bias,
-                                        const void* w1, const void* w3, const void* w2, float lb_grad_scale,
+                                        const float* router_noise, const void* w1, const void* w3, const void* w2, float lb_grad_scale,
                                         float* dw_router, float* dbias, float* dw1, float* dw3, float* dw2,
                                         int32_t accumulate, void* saved, void* workspace, size_t workspace_bytes,
                                         void* stream) {
@@ -266,10 +283,11 @@ extern "C" btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_
   BTX_CUDA_OK(cudaMemcpyAsync(dy_dev, dy_host, act_bytes, cudaMemcpyHostToDevice, st));
   btx_routing_out ro;
   memset(&ro, 0, sizeof(ro));
-  if ((s = btx_moe_forward(desc, x_dev, w_router, router_bias, w1, w3, w2, y_dev, &ro, saved, workspace,
+  if ((s = btx_moe_forward(desc, x_dev, w_router, router_bias, router_noise, w1, w3, w2, y_dev, &ro, saved, workspace,
                            workspace_bytes, stream)) != BTX_OK)
     return s;
-  if ((s = btx_moe_backward(desc, x_dev, w_router, router_bias, w1, w3, w2, dy_dev, lb_grad_scale, saved, dx_dev,
+  if ((s = btx_moe_backward(desc, x_dev, w_router, router_bias, router_noise, w1, w3, w2, dy_dev, lb_grad_scale, saved,
+                            dx_dev,
                             dw_router, dbias, dw1, dw3, dw2, accumulate, workspace, workspace_bytes, stream)) != BTX_OK)
     return s;
   BTX_CUDA_OK(cudaMemcpyAsync(y_host, y_dev, act_bytes, cudaMemcpyDeviceToHost, st));
@@ -307,13 +325,15 @@ extern "C" btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits,
   Buffers b;
   resolve(pl, ws + pl.w_saved_fallback, ws, &b);
   BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
-  BTX_CUDA_OK(launch_router(pl, BTX_F32, desc->routing, desc->lb_alpha, nullptr, nullptr, nullptr, logits, b, st));
+  if (desc->routing == BTX_ROUTE_SAMPLE1) return BTX_ERR_UNSUPPORTED;
+  BTX_CUDA_OK(launch_router(pl, BTX_F32, desc->routing, desc->lb_alpha, nullptr, nullptr, nullptr, logits, nullptr, 1.0f,
+                            b, st));
   BTX_CUDA_OK(cudaMemcpyAsync(loss, b.loss, 4, cudaMemcpyDeviceToDevice, st));
   BTX_CUDA_OK(cudaMemcpyAsync(u, b.u, pl.E * 4, cudaMemcpyDeviceToDevice, st));
   BTX_CUDA_OK(cudaMemcpyAsync(p, b.p, pl.E * 4, cudaMemcpyDeviceToDevice, st));
   if (dlogits) {
     BTX_CUDA_OK(launch_router_backward(pl, BTX_F32, desc->routing, desc->lb_alpha, 1.0f, desc->lb_stopgrad_u, 0,
-                                       nullptr, nullptr, b, nullptr, nullptr, nullptr, dlogits, 0, st));
+                                       nullptr, nullptr, b, nullptr, nullptr, nullptr, dlogits, 0, 1.0f, st));
   }
   return BTX_OK;
 }

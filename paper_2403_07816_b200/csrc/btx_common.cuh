@@ -60,20 +60,24 @@ void mark_stage(int i, cudaStream_t st);
 // ---------------------------------------------------------------------------------------------
 // Launchers (defined in the .cu files).
 // ---------------------------------------------------------------------------------------------
+// `routing` is the effective rule (Sample Top-1 arrives as SWITCH, or TOPK for hard sampling, on the
+// logits perturbed by `noise` and scaled by `inv_tau`; noise == nullptr: no perturbation).
 cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, const void* x, const void* w_router,
-                          const float* bias, const float* given_logits, const Buffers& b, cudaStream_t st);
+                          const float* bias, const float* given_logits, const float* noise, float inv_tau,
+                          const Buffers& b, cudaStream_t st);
 cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st);
 // Router + loss + permutation in one single-block launch, for batches with T*k <= 1024.
 bool route_permute_small_fits(const Plan& pl);
 cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, float alpha, const void* x,
-                                       const void* w_router, const float* bias, const Buffers& b, cudaStream_t st);
+                                       const void* w_router, const float* bias, const float* noise, float inv_tau,
+                                       const Buffers& b, cudaStream_t st);
 cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st);
 // y[t] = sum over slots and over `splits` partial copies ([split][R][d]) of the expert rows
 cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, cudaStream_t st);
 cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float alpha, float lb_scale,
                                    int stopgrad_u, int have_dg, const void* x, const void* w_router, const Buffers& b,
                                    void* dx, float* dw_router, float* dbias, float* dlogits_out, int accumulate,
-                                   cudaStream_t st);
+                                   float dz_scale, cudaStream_t st);
 
 // Expert GEMMs: SIMT fp32 kernels for BTX_F32, tcgen05 kernels for BTX_BF16.
 cudaError_t launch_expert_forward_f32(const Plan& pl, const void* w1, const void* w3, const void* w2,

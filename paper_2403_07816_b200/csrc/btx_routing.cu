@@ -48,7 +48,7 @@ template <> struct Vec<__nv_bfloat16> {
 // Selection, gates and softmax for one token from the logits z[0..E) in shared memory (all lanes of
 // the calling warp take part).  On return lane e (< E) holds the dense gate and probability of expert e.
 __device__ __forceinline__ void route_select(int t, int E, int k, int routing, const float* z, int lane,
-                                             float* __restrict__ logits, int32_t* __restrict__ topk,
+                                             int32_t* __restrict__ topk,
                                              float* __restrict__ gates, float* __restrict__ probs, float& my_g,
                                              float& my_p) {
   uint32_t taken = 0;
@@ -85,10 +85,7 @@ __device__ __forceinline__ void route_select(int t, int E, int k, int routing, c
       if (lane == 0) { topk[(size_t)t * k + j] = sel[j]; gates[(size_t)t * k + j] = gj; }
     }
   }
-  if (lane < E) {
-    probs[(size_t)t * E + lane] = my_p;
-    logits[(size_t)t * E + lane] = z[lane];
-  }
+  if (lane < E) probs[(size_t)t * E + lane] = my_p;
   __syncwarp();
 }
 
@@ -98,7 +95,8 @@ __device__ __forceinline__ void route_select(int t, int E, int k, int routing, c
 template <typename T>
 __device__ __forceinline__ void route_token(int t, int d, int E, int k, int routing, const T* __restrict__ x,
                                             const T* __restrict__ wr, const float* __restrict__ bias,
-                                            const float* __restrict__ given_logits, float* z, int lane,
+                                            const float* __restrict__ given_logits,
+                                            const float* __restrict__ noise, float inv_tau, float* z, int lane,
                                             float* __restrict__ logits, int32_t* __restrict__ topk,
                                             float* __restrict__ gates, float* __restrict__ probs, float& my_g,
                                             float& my_p) {
@@ -135,13 +133,19 @@ __device__ __forceinline__ void route_token(int t, int d, int E, int k, int rout
     }
   }
   __syncwarp();
-  route_select(t, E, k, routing, z, lane, logits, topk, gates, probs, my_g, my_p);
+  if (lane < E) {
+    logits[(size_t)t * E + lane] = z[lane];                       // reported logits are unperturbed
+    if (noise != nullptr) z[lane] = (z[lane] + noise[(size_t)t * E + lane]) * inv_tau;
+  }
+  __syncwarp();
+  route_select(t, E, k, routing, z, lane, topk, gates, probs, my_g, my_p);
 }
 
 template <typename T>
 __global__ void __launch_bounds__(kRouterThreads)
 router_kernel(int Tn, int d, int E, int k, int routing, const T* __restrict__ x, const T* __restrict__ wr,
               const float* __restrict__ bias, const float* __restrict__ given_logits,
+              const float* __restrict__ noise, float inv_tau,
               float* __restrict__ logits, int32_t* __restrict__ topk, float* __restrict__ gates,
               float* __restrict__ probs, float* __restrict__ route_part) {
   __shared__ float zs[kRouterWarps][kMaxExperts];
@@ -150,8 +154,8 @@ router_kernel(int Tn, int d, int E, int k, int routing, const T* __restrict__ x,
   float u_acc = 0.f, p_acc = 0.f;      // lane e accumulates expert e over this warp's tokens
   for (int t = blockIdx.x * kRouterWarps + warp; t < Tn; t += gridDim.x * kRouterWarps) {
     float my_g, my_p;
-    route_token<T>(t, d, E, k, routing, x, wr, bias, given_logits, zs[warp], lane, logits, topk, gates, probs, my_g,
-                   my_p);
+    route_token<T>(t, d, E, k, routing, x, wr, bias, given_logits, noise, inv_tau, zs[warp], lane, logits, topk, gates,
+                   probs, my_g, my_p);
     u_acc += my_g;
     p_acc += my_p;
   }
@@ -298,7 +302,7 @@ template <typename T>
 __global__ void __launch_bounds__(kSmallThreads)
 route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha, int mt_max, int r_pad_max,
                            const T* __restrict__ x, const T* __restrict__ wr, const float* __restrict__ bias,
-                           float* logits, int32_t* topk, float* gates, float* probs, float* __restrict__ u,
+                           const float* __restrict__ noise, float inv_tau, float* logits, int32_t* topk, float* gates, float* probs, float* __restrict__ u,
                            float* __restrict__ p, float* __restrict__ loss, int32_t* __restrict__ counts,
                            int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
                            int32_t* __restrict__ tile_expert, int32_t* __restrict__ perm,
@@ -347,12 +351,15 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
   if (threadIdx.x < E) {
     float a = 0.f;
     for (int w = 0; w < NW; ++w) a += part[w][threadIdx.x];
-    z[threadIdx.x] = a + (bias ? bias[threadIdx.x] : 0.f);
+    a += bias ? bias[threadIdx.x] : 0.f;
+    logits[(size_t)t * E + threadIdx.x] = a;                      // reported logits are unperturbed
+    if (noise != nullptr) a = (a + noise[(size_t)t * E + threadIdx.x]) * inv_tau;
+    z[threadIdx.x] = a;
   }
   __syncthreads();
   if (warp == 0) {
     float my_g, my_p;
-    route_select(t, E, k, routing, z, lane, logits, topk, gates, probs, my_g, my_p);
+    route_select(t, E, k, routing, z, lane, topk, gates, probs, my_g, my_p);
   }
   __threadfence();
   __syncthreads();
@@ -501,7 +508,7 @@ __global__ void __launch_bounds__(256)
 router_dz_kernel(int Tn, int E, int k, int routing, float alpha, float lb_scale, int stopgrad_u, int nt_dact,
                  int r_pad_max, const int32_t* __restrict__ topk, const float* __restrict__ gates,
                  const float* __restrict__ probs, const float* __restrict__ u, const float* __restrict__ p,
-                 const int32_t* __restrict__ flat2row, const float* __restrict__ dg_part,
+                 const int32_t* __restrict__ flat2row, const float* __restrict__ dg_part, float dz_scale,
                  float* __restrict__ dz_out, float* __restrict__ dz_out2) {
   int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= Tn) return;
@@ -532,7 +539,7 @@ router_dz_kernel(int Tn, int E, int k, int routing, float alpha, float lb_scale,
   float pc = 0.f;
   for (int e = 0; e < E; ++e) pc += pt[e] * (lbc * u[e]);
   for (int e = 0; e < E; ++e) {
-    float v = dzv[e] + pt[e] * (lbc * u[e] - pc);
+    float v = (dzv[e] + pt[e] * (lbc * u[e] - pc)) * dz_scale;
     dz_out[(size_t)t * E + e] = v;
     if (dz_out2 != nullptr) dz_out2[(size_t)t * E + e] = v;
   }
@@ -604,15 +611,16 @@ router_dw_reduce_kernel(int d, int E, int chunks, const float* __restrict__ part
 // Launchers
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, const void* x, const void* w_router,
-                          const float* bias, const float* given_logits, const Buffers& b, cudaStream_t st) {
+                          const float* bias, const float* given_logits, const float* noise, float inv_tau,
+                          const Buffers& b, cudaStream_t st) {
   if (dtype == BTX_BF16) {
     router_kernel<__nv_bfloat16><<<pl.route_blocks, kRouterThreads, 0, st>>>(
         pl.T, pl.d, pl.E, pl.k, routing, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, given_logits,
-        b.logits, b.topk, b.gates, b.probs, b.route_part);
+        noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.route_part);
   } else {
     router_kernel<float><<<pl.route_blocks, kRouterThreads, 0, st>>>(
-        pl.T, pl.d, pl.E, pl.k, routing, (const float*)x, (const float*)w_router, bias, given_logits, b.logits,
-        b.topk, b.gates, b.probs, b.route_part);
+        pl.T, pl.d, pl.E, pl.k, routing, (const float*)x, (const float*)w_router, bias, given_logits, noise, inv_tau,
+        b.logits, b.topk, b.gates, b.probs, b.route_part);
   }
   lb_finalize_kernel<<<1, 256, 0, st>>>(pl.T, pl.E, pl.route_blocks, alpha, b.route_part, b.u, b.p, b.loss);
   return cudaGetLastError();
@@ -621,16 +629,17 @@ cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, c
 bool route_permute_small_fits(const Plan& pl) { return pl.R <= kSmallMaxR; }
 
 cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, float alpha, const void* x,
-                                       const void* w_router, const float* bias, const Buffers& b, cudaStream_t st) {
+                                       const void* w_router, const float* bias, const float* noise, float inv_tau,
+                                       const Buffers& b, cudaStream_t st) {
   if (dtype == BTX_BF16)
     route_permute_small_kernel<__nv_bfloat16><<<pl.T, kSmallThreads, 0, st>>>(
         pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, (const __nv_bfloat16*)x,
-        (const __nv_bfloat16*)w_router, bias, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets,
+        (const __nv_bfloat16*)w_router, bias, noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets,
         b.pad_offsets, b.tile_expert, b.perm, b.inv_perm, b.rowmap, b.flat2row, b.status + 8);
   else
     route_permute_small_kernel<float><<<pl.T, kSmallThreads, 0, st>>>(
         pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, (const float*)x, (const float*)w_router, bias,
-        b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets, b.pad_offsets, b.tile_expert, b.perm,
+        noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets, b.pad_offsets, b.tile_expert, b.perm,
         b.inv_perm, b.rowmap, b.flat2row, b.status + 8);
   return cudaGetLastError();
 }
@@ -669,10 +678,10 @@ cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int spl
 cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float alpha, float lb_scale,
                                    int stopgrad_u, int have_dg, const void* x, const void* w_router, const Buffers& b,
                                    void* dx, float* dw_router, float* dbias, float* dlogits_out, int accumulate,
-                                   cudaStream_t st) {
+                                   float dz_scale, cudaStream_t st) {
   router_dz_kernel<<<(pl.T + 255) / 256, 256, 0, st>>>(pl.T, pl.E, pl.k, routing, alpha, lb_scale, stopgrad_u,
                                                        pl.nt_dact, pl.r_pad_max, b.topk, b.gates, b.probs, b.u, b.p,
-                                                       b.flat2row, have_dg ? b.dg_part : nullptr, b.dz, dlogits_out);
+                                                       b.flat2row, have_dg ? b.dg_part : nullptr, dz_scale, b.dz, dlogits_out);
   if (x == nullptr) return cudaGetLastError();     // loss-only gradient (btx_lb_loss)
   dim3 grid(pl.wr_chunks, (pl.d / 2 + 255) / 256);
   float* bias_part = b.dwr_part + (size_t)pl.wr_chunks * pl.E * pl.d;

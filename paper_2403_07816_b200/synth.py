@@ -50,6 +50,14 @@ def moe_inputs(T, d_model, d_ff, E, seed, dtype=torch.float32, device="cpu", lay
     return out
 
 
+def gumbel_noise(T, E, seed, device="cpu", layer=0):
+    """Standard Gumbel noise G = -log(-log(U)), U ~ Uniform(0,1), fp32 [T, E]: the random numbers that
+    Sample Top-1 routing draws; they are an input of the layer."""
+    g = _gen(seed, 7, layer, device)
+    u = torch.rand((T, E), generator=g, device=device, dtype=torch.float32).clamp_(1e-7, 1.0 - 1e-7)
+    return (-torch.log(-torch.log(u))).contiguous()
+
+
 def skew_bias(E, device="cpu"):
     b = torch.zeros(E, dtype=torch.float32, device=device)
     b[0] = SKEW_BIAS_EXPERT0

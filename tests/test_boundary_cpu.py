@@ -59,6 +59,14 @@ def test_sizes_and_argument_validation(L):
         with pytest.raises(B.BtxError) as ei:
             B.btx_moe_sizes(desc)
         assert ei.value.status == 2
+    # Sample Top-1: one expert, defined without the load-balancing loss
+    B.btx_moe_sizes(B.make_desc(8, 256, 688, 4, 1, torch.float32, routing=B.ROUTE_SAMPLE1, lb_alpha=0.0, gumbel_tau=0.5))
+    with pytest.raises(B.BtxError) as ei:
+        B.btx_moe_sizes(B.make_desc(8, 256, 688, 4, 1, torch.float32, routing=B.ROUTE_SAMPLE1, lb_alpha=0.01))
+    assert ei.value.status == 2
+    with pytest.raises(B.BtxError) as ei:
+        B.btx_moe_sizes(B.make_desc(8, 256, 688, 4, 2, torch.float32, routing=B.ROUTE_SAMPLE1, lb_alpha=0.0))
+    assert ei.value.status == 1
     # soft routing ignores k
     B.btx_moe_sizes(B.make_desc(8, 256, 688, 4, 0, torch.float32, routing=B.ROUTE_SOFT))
 
@@ -66,14 +74,14 @@ def test_sizes_and_argument_validation(L):
 def test_null_and_misaligned_pointers_rejected_before_any_launch(L):
     d = B.make_desc(8, 64, 64, 4, 2, torch.float32)
     vp = C.c_void_p
-    s = L.btx_moe_forward(C.byref(d), None, None, None, None, None, None, None, None, None, None, 0, None)
+    s = L.btx_moe_forward(C.byref(d), None, None, None, None, None, None, None, None, None, None, None, 0, None)
     assert s == 1
     a = vp(4096)
-    s = L.btx_moe_forward(C.byref(d), vp(4100), a, None, a, a, a, a, None, None, a, 1 << 40, None)
+    s = L.btx_moe_forward(C.byref(d), vp(4100), a, None, None, a, a, a, a, None, None, a, 1 << 40, None)
     assert s == 1                                        # x not 16-byte aligned
-    s = L.btx_moe_forward(C.byref(d), a, a, None, a, a, a, a, None, None, a, 16, None)
+    s = L.btx_moe_forward(C.byref(d), a, a, None, None, a, a, a, a, None, None, a, 16, None)
     assert s == 3                                        # workspace too small
-    s = L.btx_moe_backward(C.byref(d), a, a, None, a, a, a, a, 1.0, None, a, a, None, a, a, a, 0, a, 1 << 40, None)
+    s = L.btx_moe_backward(C.byref(d), a, a, None, None, a, a, a, a, 1.0, None, a, a, None, a, a, a, 0, a, 1 << 40, None)
     assert s == 1                                        # saved missing
     sz = C.c_size_t(0)
     assert L.btx_merge_workspace_size(0, 3, C.byref(sz)) == 1

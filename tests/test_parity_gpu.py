@@ -107,6 +107,23 @@ def test_frozen_experts_skip_weight_gradients(dtype):
         check_backward(cpu, b64, z_gpu, got, 2, B.ROUTE_TOPK, 0.05, 1.0, False, TOL[dtype])
 
 
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
+@pytest.mark.parametrize("tau", [0.7, 0.0], ids=["soft", "hard"])
+def test_sample_top1_routing(dtype, tau):
+    # Gumbel noise is an input; tau > 0: gate = largest entry of SoftMax((z+G)/tau); tau = 0: hard sample, gate 1
+    for T in (96, 700):
+        inp = synth.moe_inputs(T, 64, 72, 4, 13, dtype, DEV)
+        noise = synth.gumbel_noise(T, 4, 13, DEV)
+        fwd = gpu_forward(inp, 1, B.ROUTE_SAMPLE1, alpha=0.0, noise=noise, tau=tau)
+        cpu, b64, z_gpu, ref = check_forward(inp, fwd, 1, B.ROUTE_SAMPLE1, 0.0, None, TOL[dtype], noise=noise, tau=tau)
+        if tau == 0.0:
+            assert bool((fwd["routing"].gates == 1.0).all())
+        got = gpu_backward(inp, fwd)
+        check_backward(cpu, b64, z_gpu, got, 1, B.ROUTE_SAMPLE1, 0.0, 1.0, False, TOL[dtype], noise=noise, tau=tau)
+        if tau == 0.0:
+            assert float(got["dw_router"].abs().max()) == 0.0
+
+
 def test_results_are_deterministic_across_runs():
     inp = synth.moe_inputs(256, 256, 688, 4, 0, torch.float32, DEV)
     a = gpu_forward(inp, 2)

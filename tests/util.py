@@ -20,19 +20,21 @@ def rel_err(got, ref):
     return float(np.max(np.abs(got - ref)) / denom)
 
 
-def gpu_forward(inp, k, routing=B.ROUTE_TOPK, alpha=0.01, bias=None, save=True, stopgrad_u=False, skip_wgrad=False):
+def gpu_forward(inp, k, routing=B.ROUTE_TOPK, alpha=0.01, bias=None, save=True, stopgrad_u=False, skip_wgrad=False,
+                noise=None, tau=0.0):
     x = inp["x"]
     T, d = x.shape
     E, F, _ = inp["w1"].shape
-    desc = B.make_desc(T, d, F, E, k, x.dtype, routing, alpha, stopgrad_u, save, skip_wgrad)
+    desc = B.make_desc(T, d, F, E, k, x.dtype, routing, alpha, stopgrad_u, save, skip_wgrad, tau)
     ws, saved = B.alloc_buffers(desc, x.device)
     ws.fill_(0x7F)           # poison: results must not depend on scratch contents
     saved.fill_(0x7F)
     r = B.Routing.empty(desc, x.device)
     y = torch.empty_like(x)
-    B.btx_moe_forward(desc, x, inp["w_router"], bias, inp["w1"], inp["w3"], inp["w2"], y, r, saved if save else None, ws)
+    B.btx_moe_forward(desc, x, inp["w_router"], bias, inp["w1"], inp["w3"], inp["w2"], y, r, saved if save else None, ws,
+                      router_noise=noise)
     assert B.btx_device_status(ws) == B.BTX_OK
-    return dict(desc=desc, y=y, routing=r, saved=saved, ws=ws)
+    return dict(desc=desc, y=y, routing=r, saved=saved, ws=ws, noise=noise, tau=tau)
 
 
 def gpu_backward(inp, fwd, lb_scale=1.0, bias=None, accumulate=False, init=None):
@@ -50,7 +52,7 @@ def gpu_backward(inp, fwd, lb_scale=1.0, bias=None, accumulate=False, init=None)
     fwd["ws"].fill_(0x7F)
     B.btx_moe_backward(desc, x, inp["w_router"], bias, inp["w1"], inp["w3"], inp["w2"], inp["dy"], lb_scale,
                        fwd["saved"], out["dx"], out["dw_router"], out["dbias"], out["dw1"], out["dw3"], out["dw2"],
-                       int(accumulate), fwd["ws"])
+                       int(accumulate), fwd["ws"], router_noise=fwd.get("noise"))
     assert B.btx_device_status(fwd["ws"]) == B.BTX_OK
     return out
 
@@ -59,7 +61,7 @@ def np64(t):
     return synth.to_f64_numpy(t)
 
 
-def check_forward(inp, fwd, k, routing, alpha, bias, tol):
+def check_forward(inp, fwd, k, routing, alpha, bias, tol, noise=None, tau=1.0):
     """Parity protocol: logits by tolerance; routing and permutation bit-exact given the GPU's
     fp32 logits; gates, probabilities, loss and y by tolerance."""
     r = fwd["routing"]
@@ -68,8 +70,9 @@ def check_forward(inp, fwd, k, routing, alpha, bias, tol):
     z_ref = o.router_logits(cpu["x"], cpu["w_router"], b64)
     z_gpu = r.logits.cpu().numpy()
     assert rel_err(z_gpu, z_ref) <= tol, "logits"
+    n64 = None if noise is None else np64(noise)
     ref = o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], k, routing, alpha,
-                        router_bias=b64, logits=z_gpu)
+                        router_bias=b64, logits=z_gpu, noise=n64, tau=tau)
     for name, got in [("topk_idx", r.topk_idx), ("counts", r.counts), ("offsets", r.offsets), ("perm", r.perm),
                       ("inv_perm", r.inv_perm)]:
         assert np.array_equal(got.cpu().numpy(), ref[name]), name
@@ -83,9 +86,10 @@ def check_forward(inp, fwd, k, routing, alpha, bias, tol):
     return cpu, b64, z_gpu, ref
 
 
-def check_backward(cpu, b64, z_gpu, got, k, routing, alpha, lb_scale, stopgrad_u, tol, base=None):
+def check_backward(cpu, b64, z_gpu, got, k, routing, alpha, lb_scale, stopgrad_u, tol, base=None, noise=None, tau=1.0):
+    n64 = None if noise is None else np64(noise)
     ref = o.moe_backward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], cpu["dy"], k, routing, alpha,
-                         lb_scale, stopgrad_u, router_bias=b64, logits=z_gpu)
+                         lb_scale, stopgrad_u, router_bias=b64, logits=z_gpu, noise=n64, tau=tau)
     errs = {}
     for name in ("dx", "dw_router", "dbias", "dw1", "dw3", "dw2"):
         if got[name] is None:
