@@ -175,6 +175,22 @@ btx_status btx_merge_workspace_size(int32_t n_models, uint64_t n_items, size_t* 
 btx_status btx_merge(int32_t n_models, int32_t dtype, const btx_merge_item* items, uint64_t n_items,
                      void* workspace, size_t workspace_bytes, void* stream);
 
+/* Feed-forward layouts of the MiX merge for ONE layer (Section 3.2 and Section 3.3 "Splitting Experts",
+ * "Blending Experts").  Sources: per model i, W1_i, W3_i [F,d] and W2_i [d,F] (host arrays of N device
+ * pointers).  Destinations: w1_dst, w3_dst [E',F',d], w2_dst [E',d,F'].
+ *   STACK  E' = N, F' = F: expert i is model i's FFN (what BTX_PARAM_FFN items do).
+ *   SPLIT  E' = N*chunks, F' = F/chunks: expert i*chunks+c holds hidden units c*F' .. (c+1)*F' of model i
+ *          (rows of W1/W3, columns of W2), so the un-gated sum of the chunks of model i equals FF_i.
+ *   BLEND  E' = N, F' = F (chunks is ignored, N chunks are used): expert n holds the n-th chunk of every
+ *          model, model i's chunk in hidden units i*F/N .. (i+1)*F/N.
+ * All copies are bit-exact.  F/chunks and d must span whole 16-byte vectors. */
+typedef enum { BTX_FFN_STACK = 0, BTX_FFN_SPLIT = 1, BTX_FFN_BLEND = 2 } btx_ffn_layout;
+btx_status btx_merge_ffn_workspace_size(int32_t n_models, int32_t chunks, size_t* workspace_bytes);
+btx_status btx_merge_ffn(int32_t n_models, int32_t dtype, int32_t layout, int32_t chunks, int32_t d_model,
+                         int32_t d_ff, const void* const* w1_src, const void* const* w3_src,
+                         const void* const* w2_src, void* w1_dst, void* w3_dst, void* w2_dst,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream` and reads the status word that kernels of earlier calls left in
  * `workspace`: *device_status (host) is BTX_OK or BTX_ERR_TIMEOUT. */
 btx_status btx_device_status(const void* workspace, void* stream, int32_t* device_status);

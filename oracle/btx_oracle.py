@@ -476,6 +476,39 @@ def merge_stack(sources):
     return np.stack([np.asarray(s) for s in sources], axis=0)
 
 
+FFN_STACK, FFN_SPLIT, FFN_BLEND = 0, 1, 2
+
+
+def merge_ffn_layout(w1s, w3s, w2s, layout, chunks=1):
+    """Expert tensors of one MoE layer from the N models' feed-forward matrices (lists of [F,d], [F,d],
+    [d,F] arrays).  STACK: expert i = model i.  SPLIT (Section 3.3, "Splitting Experts"): every FF is cut
+    into `chunks` pieces of d_ff/chunks hidden units, giving N*chunks experts.  BLEND ("Blending
+    Experts"): every FF is cut into N pieces and expert n collects the n-th piece of every model."""
+    N = len(w1s)
+    F, d = np.asarray(w1s[0]).shape
+    if layout == FFN_STACK:
+        return merge_stack(w1s), merge_stack(w3s), merge_stack(w2s)
+    C = chunks if layout == FFN_SPLIT else N
+    if F % C:
+        raise ValueError("d_ff must be divisible by the number of chunks")
+    Fc = F // C
+    piece = lambda i, c: (np.asarray(w1s[i])[c * Fc:(c + 1) * Fc], np.asarray(w3s[i])[c * Fc:(c + 1) * Fc],
+                          np.asarray(w2s[i])[:, c * Fc:(c + 1) * Fc])
+    o1, o3, o2 = [], [], []
+    if layout == FFN_SPLIT:
+        for i in range(N):
+            for c in range(C):
+                a, b, w = piece(i, c)
+                o1.append(a); o3.append(b); o2.append(w)
+    else:
+        for n in range(N):
+            parts = [piece(i, n) for i in range(N)]
+            o1.append(np.concatenate([q[0] for q in parts], axis=0))
+            o3.append(np.concatenate([q[1] for q in parts], axis=0))
+            o2.append(np.concatenate([q[2] for q in parts], axis=1))
+    return np.stack(o1), np.stack(o3), np.stack(o2)
+
+
 def merge_models(models, dtype):
     """models: list of N dicts name -> array (same names/shapes).  Names containing '.ffn.'
     are stacked along a new leading expert axis; all others are averaged."""

@@ -16,6 +16,7 @@ BTX_OK = 0
 BTX_F32, BTX_BF16 = 0, 1
 ROUTE_TOPK, ROUTE_SWITCH, ROUTE_SOFT, ROUTE_SAMPLE1 = 0, 1, 2, 3
 PARAM_AVERAGE, PARAM_FFN = 0, 1
+FFN_STACK, FFN_SPLIT, FFN_BLEND = 0, 1, 2
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbtx.so")
 _lib = None
@@ -46,7 +47,7 @@ class MergeItem(C.Structure):
 
 
 EXPORTS = ["btx_moe_sizes", "btx_moe_forward", "btx_moe_backward", "btx_moe_step_host",
-           "btx_lb_loss_workspace_size", "btx_lb_loss", "btx_lb_loss_noalloc", "btx_merge_workspace_size", "btx_merge",
+           "btx_lb_loss_workspace_size", "btx_lb_loss", "btx_lb_loss_noalloc", "btx_merge_workspace_size", "btx_merge", "btx_merge_ffn_workspace_size", "btx_merge_ffn",
            "btx_device_status", "btx_set_stage_events", "btx_status_string", "btx_version"]
 
 
@@ -69,6 +70,9 @@ def lib():
         L.btx_lb_loss_noalloc.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp]
         L.btx_merge_workspace_size.argtypes = [i32, C.c_uint64, C.POINTER(sz)]
         L.btx_merge.argtypes = [i32, i32, C.POINTER(MergeItem), C.c_uint64, vp, sz, vp]
+        L.btx_merge_ffn_workspace_size.argtypes = [i32, i32, C.POINTER(sz)]
+        L.btx_merge_ffn.argtypes = [i32, i32, i32, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp, vp, vp,
+                                    vp, sz, vp]
         L.btx_device_status.argtypes = [vp, vp, C.POINTER(i32)]
         L.btx_status_string.argtypes = [i32]
         L.btx_status_string.restype = C.c_char_p
@@ -267,6 +271,27 @@ def btx_merge(models, outputs, workspace=None):
     s = lib().btx_merge(n, _dtype_code(dtype), items, len(names), _ptr(workspace), workspace.numel(), _stream(device))
     if s != BTX_OK:
         raise BtxError(s, "btx_merge")
+    return workspace
+
+
+def btx_merge_ffn(w1s, w3s, w2s, layout, chunks, w1_dst, w3_dst, w2_dst, workspace=None):
+    """One layer's FFN matrices of N models (lists of [F,d], [F,d], [d,F] tensors) into expert tensors in
+    the STACK, SPLIT or BLEND layout; see btx.h."""
+    n = len(w1s)
+    F, d = w1s[0].shape
+    arr = lambda ts: (C.c_void_p * n)(*[_ptr(t).value for t in ts])
+    a1, a3, a2 = arr(w1s), arr(w3s), arr(w2s)
+    device = w1s[0].device
+    if workspace is None:
+        sz = C.c_size_t(0)
+        s = lib().btx_merge_ffn_workspace_size(n, max(1, chunks), C.byref(sz))
+        if s != BTX_OK:
+            raise BtxError(s, "btx_merge_ffn_workspace_size")
+        workspace = torch.empty(sz.value, dtype=torch.uint8, device=device)
+    s = lib().btx_merge_ffn(n, _dtype_code(w1s[0].dtype), layout, chunks, d, F, a1, a3, a2, _ptr(w1_dst), _ptr(w3_dst),
+                            _ptr(w2_dst), _ptr(workspace), workspace.numel(), _stream(device))
+    if s != BTX_OK:
+        raise BtxError(s, "btx_merge_ffn")
     return workspace
 
 

@@ -17,7 +17,8 @@ struct DevItem {
   uint64_t numel;
   void* dst;
   int32_t nsrc;                           // 1: copy, N: average
-  int32_t pad;
+  uint32_t row_vecs;                      // copies only: 0 = linear, else 16-byte vectors per row of a 2-D block
+  uint32_t src_pitch, dst_pitch;          // row pitches of the block in 16-byte vectors
   const void* src[kMaxModels];
 };
 
@@ -88,7 +89,15 @@ merge_kernel(const DevItem* __restrict__ items, const uint64_t* __restrict__ chu
     const int ns = it.nsrc;
     uint4* dst = reinterpret_cast<uint4*>(it.dst);
     constexpr int U = 4;                                    // vectors per thread per round
-    if (ns == 1) {
+    if (ns == 1 && it.row_vecs != 0) {
+      // 2-D block copy (a column range of W2, or a row range placed inside a wider tensor)
+      const uint4* s = reinterpret_cast<const uint4*>(it.src[0]);
+      const uint32_t rv = it.row_vecs;
+      for (uint64_t v = v0 + threadIdx.x; v < v1; v += kMergeThreads) {
+        const uint64_t r = v / rv, cidx = v - r * rv;
+        st_stream(dst + r * it.dst_pitch + cidx, ld_stream(s + r * it.src_pitch + cidx));
+      }
+    } else if (ns == 1) {
       const uint4* s = reinterpret_cast<const uint4*>(it.src[0]);
       uint64_t v = v0 + threadIdx.x;
       for (; v + (U - 1) * kMergeThreads < v1; v += U * kMergeThreads) {
@@ -168,6 +177,34 @@ uint64_t chunks_of(uint64_t numel, int per_vec) {
 
 using namespace btx;
 
+static btx_status launch_merge_items(std::vector<DevItem>& dev, std::vector<uint64_t>& start, uint64_t total,
+                                     int32_t dtype, void* workspace, size_t workspace_bytes, void* stream) {
+  if (dev.empty()) return BTX_OK;
+  start.push_back(total);
+  const size_t need = kStatusWords * 4 + dev.size() * sizeof(DevItem) + start.size() * sizeof(uint64_t);
+  if (workspace_bytes < need) return BTX_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* w = (char*)workspace + kStatusWords * 4;
+  DevItem* d_items = (DevItem*)w;
+  uint64_t* d_start = (uint64_t*)(w + dev.size() * sizeof(DevItem));
+  // pageable sources are staged before cudaMemcpyAsync returns, so the vectors may go out of scope
+  if (cudaMemcpyAsync(d_items, dev.data(), dev.size() * sizeof(DevItem), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return BTX_ERR_CUDA;
+  if (cudaMemcpyAsync(d_start, start.data(), start.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, st) !=
+      cudaSuccess)
+    return BTX_ERR_CUDA;
+  int sms = 148, dev_id = 0;
+  cudaGetDevice(&dev_id);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_id);
+  uint64_t grid = (uint64_t)sms * 8;
+  if (grid > total) grid = total;
+  if (dtype == BTX_BF16)
+    merge_kernel<__nv_bfloat16><<<(unsigned)grid, kMergeThreads, 0, st>>>(d_items, d_start, (int)dev.size(), total);
+  else
+    merge_kernel<float><<<(unsigned)grid, kMergeThreads, 0, st>>>(d_items, d_start, (int)dev.size(), total);
+  return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
+}
+
 extern "C" btx_status btx_merge_workspace_size(int32_t n_models, uint64_t n_items, size_t* workspace_bytes) {
   if (!workspace_bytes || n_models < 1 || n_models > kMaxModels) return BTX_ERR_INVALID_ARG;
   uint64_t sub = n_items * (uint64_t)n_models;             // an FFN item becomes n_models copies
@@ -212,26 +249,63 @@ extern "C" btx_status btx_merge(int32_t n_models, int32_t dtype, const btx_merge
       }
     }
   }
-  if (dev.empty()) return BTX_OK;
-  start.push_back(total);
-  cudaStream_t st = (cudaStream_t)stream;
-  char* w = (char*)workspace + kStatusWords * 4;
-  DevItem* d_items = (DevItem*)w;
-  uint64_t* d_start = (uint64_t*)(w + dev.size() * sizeof(DevItem));
-  // pageable sources are staged before cudaMemcpyAsync returns, so the vectors may go out of scope
-  if (cudaMemcpyAsync(d_items, dev.data(), dev.size() * sizeof(DevItem), cudaMemcpyHostToDevice, st) != cudaSuccess)
-    return BTX_ERR_CUDA;
-  if (cudaMemcpyAsync(d_start, start.data(), start.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, st) !=
-      cudaSuccess)
-    return BTX_ERR_CUDA;
-  int sms = 148, dev_id = 0;
-  cudaGetDevice(&dev_id);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_id);
-  uint64_t grid = (uint64_t)sms * 8;
-  if (grid > total) grid = total;
-  if (dtype == BTX_BF16)
-    merge_kernel<__nv_bfloat16><<<(unsigned)grid, kMergeThreads, 0, st>>>(d_items, d_start, (int)dev.size(), total);
-  else
-    merge_kernel<float><<<(unsigned)grid, kMergeThreads, 0, st>>>(d_items, d_start, (int)dev.size(), total);
-  return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
+  return launch_merge_items(dev, start, total, dtype, workspace, workspace_bytes, stream);
+}
+
+extern "C" btx_status btx_merge_ffn_workspace_size(int32_t n_models, int32_t chunks, size_t* workspace_bytes) {
+  if (!workspace_bytes || n_models < 1 || n_models > kMaxModels || chunks < 1 || chunks > 64) return BTX_ERR_INVALID_ARG;
+  const uint64_t c = chunks > n_models ? chunks : n_models;
+  const uint64_t items = 3ull * n_models * c + 8;
+  *workspace_bytes = kStatusWords * 4 + items * sizeof(DevItem) + (items + 1) * sizeof(uint64_t) + 256;
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_merge_ffn(int32_t n_models, int32_t dtype, int32_t layout, int32_t chunks, int32_t d_model,
+                                    int32_t d_ff, const void* const* w1_src, const void* const* w3_src,
+                                    const void* const* w2_src, void* w1_dst, void* w3_dst, void* w2_dst,
+                                    void* workspace, size_t workspace_bytes, void* stream) {
+  if (n_models < 1 || n_models > kMaxModels) return BTX_ERR_UNSUPPORTED;
+  if (dtype != BTX_F32 && dtype != BTX_BF16) return BTX_ERR_INVALID_ARG;
+  if (layout < BTX_FFN_STACK || layout > BTX_FFN_BLEND || d_model < 1 || d_ff < 1) return BTX_ERR_INVALID_ARG;
+  if (!w1_src || !w3_src || !w2_src || !w1_dst || !w3_dst || !w2_dst || !workspace) return BTX_ERR_INVALID_ARG;
+  const int C = layout == BTX_FFN_STACK ? 1 : (layout == BTX_FFN_BLEND ? n_models : chunks);
+  if (C < 1 || d_ff % C != 0) return BTX_ERR_INVALID_ARG;
+  const int esize = dtype == BTX_BF16 ? 2 : 4;
+  const int per_vec = 16 / esize;
+  const uint64_t Fc = (uint64_t)d_ff / C;                     // chunk width
+  if ((Fc * esize) % 16 != 0 || ((uint64_t)d_model * esize) % 16 != 0) return BTX_ERR_UNSUPPORTED;
+  auto bad = [](const void* p) { return p == nullptr || ((uintptr_t)p & 15) != 0; };
+  if (bad(w1_dst) || bad(w3_dst) || bad(w2_dst) || ((uintptr_t)workspace & 15)) return BTX_ERR_INVALID_ARG;
+  for (int m = 0; m < n_models; ++m)
+    if (bad(w1_src[m]) || bad(w3_src[m]) || bad(w2_src[m])) return BTX_ERR_INVALID_ARG;
+
+  std::vector<DevItem> dev;
+  std::vector<uint64_t> start;
+  uint64_t total = 0;
+  auto push = [&](const void* src, void* dst, uint64_t numel, uint32_t row_elems, uint64_t src_pitch, uint64_t dst_pitch) {
+    DevItem it = {};
+    it.numel = numel; it.dst = dst; it.nsrc = 1; it.src[0] = src;
+    if (row_elems != 0) {
+      it.row_vecs = row_elems / per_vec; it.src_pitch = (uint32_t)(src_pitch / per_vec); it.dst_pitch = (uint32_t)(dst_pitch / per_vec);
+    }
+    dev.push_back(it); start.push_back(total); total += chunks_of(numel, per_vec);
+  };
+  const uint64_t d = d_model, F = d_ff;
+  for (int i = 0; i < n_models; ++i) {
+    const char* s1 = (const char*)w1_src[i]; const char* s3 = (const char*)w3_src[i]; const char* s2 = (const char*)w2_src[i];
+    for (int c = 0; c < C; ++c) {
+      // destination expert and, for BLEND, the slot of model i inside it
+      const uint64_t e = layout == BTX_FFN_BLEND ? (uint64_t)c : (uint64_t)i * C + c;
+      const uint64_t Fd = layout == BTX_FFN_BLEND ? F : Fc;                  // width of a destination expert
+      const uint64_t slot = layout == BTX_FFN_BLEND ? (uint64_t)i * Fc : 0;   // first hidden unit inside the expert
+      // W1/W3 [F, d]: rows c*Fc .. (c+1)*Fc of model i, contiguous
+      const uint64_t src_rows = (uint64_t)c * Fc * d * esize;
+      const uint64_t dst_rows = (e * Fd + slot) * d * esize;
+      push(s1 + src_rows, (char*)w1_dst + dst_rows, Fc * d, 0, 0, 0);
+      push(s3 + src_rows, (char*)w3_dst + dst_rows, Fc * d, 0, 0, 0);
+      // W2 [d, F]: columns c*Fc .. (c+1)*Fc of model i -> columns slot .. slot+Fc of expert e
+      push(s2 + (uint64_t)c * Fc * esize, (char*)w2_dst + (e * d * Fd + slot) * esize, d * Fc, (uint32_t)Fc, F, Fd);
+    }
+  }
+  return launch_merge_items(dev, start, total, dtype, workspace, workspace_bytes, stream);
 }

@@ -462,3 +462,37 @@ def test_sample_top1_gradients_against_finite_differences():
             assert abs(fd - g[name][pos]) <= 2e-6 * max(1.0, abs(fd)), (name, pos, fd, g[name][pos])
     hard = o.moe_backward(x, wr, w1, w3, w2, G, k=1, routing=o.ROUTE_SAMPLE1, alpha=0.0, noise=noise, tau=0.0)
     assert np.all(hard["dw_router"] == 0.0)
+
+
+# ---- split / blend layouts of the merge ---------------------------------------------------------
+
+def test_split_and_blend_layouts_preserve_the_feed_forward_sums():
+    r = RNG(31)
+    N, F, d = 4, 24, 6
+    w1s = [r.standard_normal((F, d)) for _ in range(N)]
+    w3s = [r.standard_normal((F, d)) for _ in range(N)]
+    w2s = [r.standard_normal((d, F)) for _ in range(N)]
+    x = r.standard_normal((5, d))
+    ff = [o.swiglu_ffn(x, w1s[i], w3s[i], w2s[i]) for i in range(N)]
+    # splitting: the un-gated sum of the chunks of model i is FF_i (SwiGLU acts per hidden unit)
+    for C in (1, 2, 3):
+        s1, s3, s2 = o.merge_ffn_layout(w1s, w3s, w2s, o.FFN_SPLIT, C)
+        assert s1.shape == (N * C, F // C, d) and s2.shape == (N * C, d, F // C)
+        for i in range(N):
+            tot = sum(o.swiglu_ffn(x, s1[i * C + c], s3[i * C + c], s2[i * C + c]) for c in range(C))
+            np.testing.assert_allclose(tot, ff[i], rtol=1e-12, atol=1e-13)
+    # blending: every expert has the full width and the sum over all experts is the sum over all models
+    b1, b3, b2 = o.merge_ffn_layout(w1s, w3s, w2s, o.FFN_BLEND)
+    assert b1.shape == (N, F, d) and b2.shape == (N, d, F)
+    np.testing.assert_allclose(sum(o.swiglu_ffn(x, b1[n], b3[n], b2[n]) for n in range(N)), sum(ff), rtol=1e-12, atol=1e-13)
+    # expert n of the blend starts with the n-th chunk of model 0
+    Fc = F // N
+    assert (b1[2][:Fc] == w1s[0][2 * Fc:3 * Fc]).all() and (b2[2][:, Fc:2 * Fc] == w2s[1][:, 2 * Fc:3 * Fc]).all()
+    # blending identical models permutes hidden units only: each expert equals the seed FF
+    same = o.merge_ffn_layout([w1s[0]] * N, [w3s[0]] * N, [w2s[0]] * N, o.FFN_BLEND)
+    for n in range(N):
+        got = o.swiglu_ffn(x, same[0][n], same[1][n], same[2][n])
+        want = N * o.swiglu_ffn(x, w1s[0][n * Fc:(n + 1) * Fc], w3s[0][n * Fc:(n + 1) * Fc], w2s[0][:, n * Fc:(n + 1) * Fc])
+        np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
+    st = o.merge_ffn_layout(w1s, w3s, w2s, o.FFN_STACK)
+    assert (st[0][1] == w1s[1]).all() and (st[2][3] == w2s[3]).all()

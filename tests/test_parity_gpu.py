@@ -188,3 +188,19 @@ def test_merge_toy_models(dtype, name):
     for n in out:
         if ".ffn." not in n:
             assert torch.equal(out[n], models[0][n]), n
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
+def test_merge_split_and_blend_layouts(dtype):
+    N, F, d = 4, 704, 256            # F/4 = 176 hidden units: whole 16-byte vectors in both dtypes
+    w1s = [synth.normal((F, d), 0.02, 7, 10 + i, dtype, DEV) for i in range(N)]
+    w3s = [synth.normal((F, d), 0.02, 7, 20 + i, dtype, DEV) for i in range(N)]
+    w2s = [synth.normal((d, F), 0.02, 7, 30 + i, dtype, DEV) for i in range(N)]
+    cpu = [[np64(t) for t in ts] for ts in (w1s, w3s, w2s)]
+    for layout, chunks in [(B.FFN_STACK, 1), (B.FFN_SPLIT, 2), (B.FFN_SPLIT, 4), (B.FFN_BLEND, 0)]:
+        ref = o.merge_ffn_layout(cpu[0], cpu[1], cpu[2], layout, chunks)
+        outs = [torch.full(r.shape, 3.0, dtype=dtype, device=DEV) for r in ref]
+        B.btx_merge_ffn(w1s, w3s, w2s, layout, chunks, *outs)
+        torch.cuda.synchronize()
+        for got, want in zip(outs, ref):
+            assert np.array_equal(np64(got), want), (layout, chunks)       # pure copies: bit-exact
