@@ -119,8 +119,10 @@ btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void*
  * runs btx_moe_forward (saving for backward) and btx_moe_backward, and copies y, dx and the
  * load-balancing loss back to y_host, dx_host, loss_host.  Weights, gradients, staging buffers,
  * `saved` and `workspace` are device memory as in the two calls it composes; desc.save_for_backward
- * must be 1.  Everything is enqueued on `stream`; the host results are valid after the stream
- * has been synchronised. */
+ * must be 1.  Everything is ordered on `stream`; the host results are valid after the stream
+ * has been synchronised.  `copy_stream` (optional, NULL = none) is a second stream of the caller on
+ * which the dy upload overlaps the forward pass and the y download overlaps the backward pass; the
+ * call joins it back into `stream` before it returns. */
 btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_host, const void* dy_host,
                              void* y_host, void* dx_host, float* loss_host,
                              void* x_dev, void* dy_dev, void* y_dev, void* dx_dev,
@@ -128,7 +130,7 @@ btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_host, const
                              const void* w1, const void* w3, const void* w2, float lb_grad_scale,
                              float* dw_router, float* dbias, float* dw1, float* dw3, float* dw2,
                              int32_t accumulate, void* saved, void* workspace, size_t workspace_bytes,
-                             void* stream);
+                             void* stream, void* copy_stream);
 
 /* L_LB = alpha * E * sum_i u_i p_i with u_i the batch mean of the gate of expert i and p_i the
  * batch mean of SoftMax_i (Section 3.3), from given fp32 logits[T,E] (bias, if any, already

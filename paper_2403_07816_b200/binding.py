@@ -63,7 +63,7 @@ def lib():
                                       sz, vp]
         L.btx_moe_backward.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp, vp,
                                        vp, i32, vp, sz, vp]
-        L.btx_moe_step_host.argtypes = [C.POINTER(MoeDesc)] + [vp] * 15 + [f32] + [vp] * 5 + [i32, vp, vp, sz, vp]
+        L.btx_moe_step_host.argtypes = [C.POINTER(MoeDesc)] + [vp] * 15 + [f32] + [vp] * 5 + [i32, vp, vp, sz, vp, vp]
         L.btx_set_stage_events.argtypes = [C.POINTER(vp), i32]
         L.btx_lb_loss_workspace_size.argtypes = [C.POINTER(MoeDesc), C.POINTER(sz)]
         L.btx_lb_loss.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, sz, vp]
@@ -181,8 +181,9 @@ def btx_moe_backward(desc, x, w_router, router_bias, w1, w3, w2, dy, lb_grad_sca
 
 def btx_moe_step_host(desc, x_host, dy_host, y_host, dx_host, loss_host, x_dev, dy_dev, y_dev, dx_dev, w_router,
                       router_bias, w1, w3, w2, lb_grad_scale, dw_router, dbias, dw1, dw3, dw2, accumulate, saved,
-                      workspace, router_noise=None):
-    """Forward + backward with activations in (pinned) host tensors; see btx.h."""
+                      workspace, router_noise=None, copy_stream=None):
+    """Forward + backward with activations in (pinned) host tensors; see btx.h.  `copy_stream` is an
+    optional torch.cuda.Stream on which the dy upload and the y download overlap the compute."""
     for t in (x_host, dy_host, y_host, dx_host, loss_host):
         if t.is_cuda or not t.is_contiguous():
             raise RuntimeError("btx_moe_step_host: host tensors must be contiguous CPU tensors")
@@ -192,7 +193,8 @@ def btx_moe_step_host(desc, x_host, dy_host, y_host, dx_host, loss_host, x_dev, 
                                 _ptr(router_bias), _ptr(router_noise), _ptr(w1), _ptr(w3), _ptr(w2),
                                 float(lb_grad_scale),
                                 _ptr(dw_router), _ptr(dbias), _ptr(dw1), _ptr(dw3), _ptr(dw2), int(accumulate),
-                                _ptr(saved), _ptr(workspace), workspace.numel(), _stream(x_dev.device))
+                                _ptr(saved), _ptr(workspace), workspace.numel(), _stream(x_dev.device),
+                                C.c_void_p(copy_stream.cuda_stream) if copy_stream is not None else None)
     if s != BTX_OK:
         raise BtxError(s, "btx_moe_step_host")
 

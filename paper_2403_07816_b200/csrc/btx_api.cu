@@ -270,7 +270,7 @@ extern "C" btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_
                                         const float* router_noise, const void* w1, const void* w3, const void* w2, float lb_grad_scale,
                                         float* dw_router, float* dbias, float* dw1, float* dw3, float* dw2,
                                         int32_t accumulate, void* saved, void* workspace, size_t workspace_bytes,
-                                        void* stream) {
+                                        void* stream, void* copy_stream) {
   Plan pl;
   btx_status s = make_plan(desc, &pl, false);
   if (s != BTX_OK) return s;
@@ -278,21 +278,46 @@ extern "C" btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_
     return BTX_ERR_INVALID_ARG;
   if (!desc->save_for_backward) return BTX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
+  cudaStream_t cs = (cudaStream_t)copy_stream;
+  const bool overlap = copy_stream != nullptr && copy_stream != stream;
   const size_t act_bytes = (size_t)pl.T * pl.d * pl.esize;
+  cudaEvent_t ev_start = nullptr, ev_dy = nullptr, ev_fwd = nullptr, ev_y = nullptr;
+  if (overlap) {
+    // dy travels to the device while the forward runs, y travels back while the backward runs
+    const unsigned f = cudaEventDisableTiming;
+    if (cudaEventCreateWithFlags(&ev_start, f) != cudaSuccess || cudaEventCreateWithFlags(&ev_dy, f) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ev_fwd, f) != cudaSuccess || cudaEventCreateWithFlags(&ev_y, f) != cudaSuccess)
+      return BTX_ERR_CUDA;
+    BTX_CUDA_OK(cudaEventRecord(ev_start, st));             // the copy stream joins the caller's ordering
+    BTX_CUDA_OK(cudaStreamWaitEvent(cs, ev_start, 0));
+    BTX_CUDA_OK(cudaMemcpyAsync(dy_dev, dy_host, act_bytes, cudaMemcpyHostToDevice, cs));
+    BTX_CUDA_OK(cudaEventRecord(ev_dy, cs));
+  }
   BTX_CUDA_OK(cudaMemcpyAsync(x_dev, x_host, act_bytes, cudaMemcpyHostToDevice, st));
-  BTX_CUDA_OK(cudaMemcpyAsync(dy_dev, dy_host, act_bytes, cudaMemcpyHostToDevice, st));
+  if (!overlap) BTX_CUDA_OK(cudaMemcpyAsync(dy_dev, dy_host, act_bytes, cudaMemcpyHostToDevice, st));
   btx_routing_out ro;
   memset(&ro, 0, sizeof(ro));
   if ((s = btx_moe_forward(desc, x_dev, w_router, router_bias, router_noise, w1, w3, w2, y_dev, &ro, saved, workspace,
                            workspace_bytes, stream)) != BTX_OK)
     return s;
+  if (overlap) {
+    BTX_CUDA_OK(cudaEventRecord(ev_fwd, st));
+    BTX_CUDA_OK(cudaStreamWaitEvent(cs, ev_fwd, 0));
+    BTX_CUDA_OK(cudaMemcpyAsync(y_host, y_dev, act_bytes, cudaMemcpyDeviceToHost, cs));
+    BTX_CUDA_OK(cudaEventRecord(ev_y, cs));
+    BTX_CUDA_OK(cudaStreamWaitEvent(st, ev_dy, 0));
+  }
   if ((s = btx_moe_backward(desc, x_dev, w_router, router_bias, router_noise, w1, w3, w2, dy_dev, lb_grad_scale, saved,
-                            dx_dev,
-                            dw_router, dbias, dw1, dw3, dw2, accumulate, workspace, workspace_bytes, stream)) != BTX_OK)
+                            dx_dev, dw_router, dbias, dw1, dw3, dw2, accumulate, workspace, workspace_bytes, stream)) !=
+      BTX_OK)
     return s;
-  BTX_CUDA_OK(cudaMemcpyAsync(y_host, y_dev, act_bytes, cudaMemcpyDeviceToHost, st));
+  if (!overlap) BTX_CUDA_OK(cudaMemcpyAsync(y_host, y_dev, act_bytes, cudaMemcpyDeviceToHost, st));
   BTX_CUDA_OK(cudaMemcpyAsync(dx_host, dx_dev, act_bytes, cudaMemcpyDeviceToHost, st));
   BTX_CUDA_OK(cudaMemcpyAsync(loss_host, (const char*)saved + pl.s_loss, 4, cudaMemcpyDeviceToHost, st));
+  if (overlap) {
+    BTX_CUDA_OK(cudaStreamWaitEvent(st, ev_y, 0));          // everything is complete when `stream` is
+    cudaEventDestroy(ev_start); cudaEventDestroy(ev_dy); cudaEventDestroy(ev_fwd); cudaEventDestroy(ev_y);
+  }
   return BTX_OK;
 }
 

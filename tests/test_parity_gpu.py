@@ -204,3 +204,42 @@ def test_merge_split_and_blend_layouts(dtype):
         torch.cuda.synchronize()
         for got, want in zip(outs, ref):
             assert np.array_equal(np64(got), want), (layout, chunks)       # pure copies: bit-exact
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("overlap", [False, True], ids=["one_stream", "copy_stream"])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_step_host_matches_oracle(dtype, overlap):
+    """The host-buffer entry point (pinned x, dy in; y, dx, loss out), with and without a second
+    stream for the copies, gives the oracle's y, dx, loss and weight gradients."""
+    dev = torch.device(DEV)
+    T, d, F, E, k = 777, 128, 328, 4, 2
+    inp = synth.moe_inputs(T, d, F, E, 41, dtype, DEV)
+    desc = B.make_desc(T, d, F, E, k, dtype, B.ROUTE_TOPK, 0.01, False, True)
+    ws, saved = B.alloc_buffers(desc, dev)
+    hx, hdy = inp["x"].cpu().pin_memory(), inp["dy"].cpu().pin_memory()
+    hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+    hloss = torch.zeros(1, dtype=torch.float32).pin_memory()
+    xd, dyd, yd, dxd = (torch.empty_like(inp["x"]) for _ in range(4))
+    f32 = dict(dtype=torch.float32, device=dev)
+    out = dict(dw_router=torch.empty(E, d, **f32), dbias=torch.empty(E, **f32), dw1=torch.empty(E, F, d, **f32),
+               dw3=torch.empty(E, F, d, **f32), dw2=torch.empty(E, d, F, **f32))
+    cs = torch.cuda.Stream(device=dev) if overlap else None
+    for _ in range(2):       # the second call reuses every buffer: the copy stream must be joined back
+        hy.zero_(); hdx.zero_()
+        B.btx_moe_step_host(desc, hx, hdy, hy, hdx, hloss, xd, dyd, yd, dxd, inp["w_router"], None, inp["w1"],
+                            inp["w3"], inp["w2"], 1.0, out["dw_router"], out["dbias"], out["dw1"], out["dw3"],
+                            out["dw2"], 0, saved, ws, copy_stream=cs)
+        torch.cuda.current_stream(dev).synchronize()
+        assert B.btx_device_status(ws) == B.BTX_OK
+    tol = TOL[dtype]
+    cpu = {n: np64(t) for n, t in inp.items()}
+    # routing decisions are taken on the GPU's fp32 logits (the same kernel, run through the device entry point)
+    z_ref = gpu_forward(inp, k, save=False)["routing"].logits.cpu().numpy()
+    fwd = o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], k, B.ROUTE_TOPK, 0.01,
+                        logits=z_ref)
+    assert rel_err(np64(hy), fwd["y"]) <= tol
+    assert abs(float(hloss.item()) - fwd["lb_loss"]) <= tol * abs(fwd["lb_loss"])
+    got = dict(out, dx=hdx)
+    check_backward(cpu, None, z_ref, got, k, B.ROUTE_TOPK, 0.01, 1.0, False, tol)
+    assert torch.equal(yd.cpu(), hy) and torch.equal(dxd.cpu(), hdx)
