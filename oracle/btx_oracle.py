@@ -35,6 +35,8 @@ invariants, brute force, finite differences, the paper's Table 4 parameter count
 """
 from __future__ import annotations
 
+import math
+
 import numpy as np
 
 ROUTE_TOPK = 0
@@ -144,24 +146,55 @@ def lb_loss_from_logits(z, k, routing, alpha):
 # Dispatch permutation (implementation structure: assignments sorted by expert, then token)
 # --------------------------------------------------------------------------------------
 
-def dispatch(idx, E):
+def expert_capacity(T, k, E, capacity_factor):
+    """Rows one expert accepts: ceil(CF * T * k / E), CF held as an fp32 number (Section 4.1 sets
+    CF = 1.5 for Switch routing, where k = 1; 0 means no limit)."""
+    cf = float(np.float32(capacity_factor))
+    if cf <= 0.0:
+        return T * k
+    return int(math.ceil(cf * float(T * k) / float(E)))
+
+
+def capacity_keep(idx, E, capacity):
+    """keep[T, k]: an expert takes its assignments in order of flat id (token, then slot) until it
+    holds `capacity` of them; the hard limit of Section 4.1 drops the rest."""
+    idx = np.asarray(idx)
+    T, k = idx.shape
+    keep = np.zeros((T, k), dtype=bool)
+    held = [0] * E
+    for t in range(T):
+        for slot in range(k):
+            e = int(idx[t, slot])
+            if held[e] < capacity:
+                held[e] += 1
+                keep[t, slot] = True
+    return keep
+
+
+def dispatch(idx, E, keep=None):
     """counts[E], offsets[E+1], perm[R], inv_perm[R] for the R = T*k assignments.
 
     Assignment (t, slot) has flat id t*k + slot.  Sorted order is by expert id ascending and,
     inside one expert, by token index ascending (a token meets an expert at most once).
     perm[r] = flat id of the assignment in sorted row r; inv_perm[flat id] = r.
+    With `keep` (capacity limit) only kept assignments are counted and sorted: a dropped one has
+    inv_perm = -1 and the unused tail of perm is -1.
     """
     idx = np.asarray(idx)
     T, k = idx.shape
     flat = idx.reshape(-1).astype(np.int64)
+    kept = np.ones(T * k, dtype=bool) if keep is None else np.asarray(keep, dtype=bool).reshape(-1)
     counts = np.zeros(E, dtype=np.int32)
     for e in range(E):
-        counts[e] = int(np.sum(flat == e))
+        counts[e] = int(np.sum((flat == e) & kept))
     offsets = np.zeros(E + 1, dtype=np.int32)
     offsets[1:] = np.cumsum(counts)
-    perm = np.argsort(flat, kind="stable").astype(np.int32)
-    inv_perm = np.empty_like(perm)
-    inv_perm[perm] = np.arange(T * k, dtype=np.int32)
+    order = np.argsort(flat, kind="stable")
+    order = order[kept[order]]
+    perm = np.full(T * k, -1, dtype=np.int32)
+    perm[:len(order)] = order
+    inv_perm = np.full(T * k, -1, dtype=np.int32)
+    inv_perm[order] = np.arange(len(order), dtype=np.int32)
     return counts, offsets, perm, inv_perm
 
 
@@ -222,8 +255,11 @@ def route(x, w_router, k, routing=ROUTE_TOPK, router_bias=None, logits=None, noi
 
 
 def moe_forward(x, w_router, w1, w3, w2, k, routing=ROUTE_TOPK, alpha=0.01,
-                router_bias=None, logits=None, tokens=None, noise=None, tau=1.0):
+                router_bias=None, logits=None, tokens=None, noise=None, tau=1.0, capacity_factor=0.0):
     """FF_MoE(x) = sum_i g_i(W_l x) FF_i(x), skipping experts whose gate is zero.
+
+    capacity_factor > 0 (Section 4.1, Switch routing): an assignment beyond its expert's capacity
+    is dropped, i.e. contributes nothing to y; gates, probabilities and L_LB are those of the router.
 
     w1, w3: [E, F, d]; w2: [E, d, F].  `logits` (optional, [T, E]) replaces W_l x so that the
     routing decision can be taken on exactly the numbers another implementation produced.
@@ -236,19 +272,23 @@ def moe_forward(x, w_router, w1, w3, w2, k, routing=ROUTE_TOPK, alpha=0.01,
     z, idx, g, p_tok = route(x, w_router, k, routing, router_bias, logits, noise, tau)
     gd = dense_gates(idx, g, E)
     loss, u, p = lb_loss(gd, p_tok, alpha)
-    counts, offsets, perm, inv_perm = dispatch(idx, E)
+    kk = idx.shape[1]
+    if capacity_factor > 0 and routing == ROUTE_SOFT:
+        raise ValueError("a capacity limit has no meaning when every expert takes every token")
+    keep = capacity_keep(idx, E, expert_capacity(T, kk, E, capacity_factor)) if capacity_factor > 0 \
+        else np.ones(idx.shape, dtype=bool)
+    counts, offsets, perm, inv_perm = dispatch(idx, E, keep)
 
     tok = np.arange(T) if tokens is None else np.asarray(tokens, dtype=np.int64)
     y = np.zeros((len(tok), d), dtype=_F64)
-    kk = idx.shape[1]
     for slot in range(kk):                       # slot order, as the combine is defined
         for e in range(E):
-            m = idx[tok, slot] == e
+            m = (idx[tok, slot] == e) & keep[tok, slot]
             if not np.any(m):
                 continue
             y[m] += g[tok[m], slot][:, None] * swiglu_ffn(x[tok[m]], w1[e], w3[e], w2[e])
     return dict(logits=z, topk_idx=idx, gates=g, probs=p_tok, y=y, lb_loss=loss, u=u, p=p,
-                counts=counts, offsets=offsets, perm=perm, inv_perm=inv_perm, tokens=tok)
+                counts=counts, offsets=offsets, perm=perm, inv_perm=inv_perm, tokens=tok, keep=keep)
 
 
 def moe_forward_all_experts(x, w_router, w1, w3, w2, k, routing=ROUTE_TOPK, router_bias=None):
@@ -298,8 +338,11 @@ def router_backward_dz(idx, gates, probs, dgate, u, alpha, lb_grad_scale, routin
 
 
 def moe_backward(x, w_router, w1, w3, w2, dy, k, routing=ROUTE_TOPK, alpha=0.01,
-                 lb_grad_scale=1.0, lb_stopgrad_u=False, router_bias=None, logits=None, noise=None, tau=1.0):
-    """Gradients of  <Y, dY> + lb_grad_scale * L_LB  w.r.t. x, W_l, bias, W1, W3, W2 (all tokens)."""
+                 lb_grad_scale=1.0, lb_stopgrad_u=False, router_bias=None, logits=None, noise=None, tau=1.0,
+                 capacity_factor=0.0):
+    """Gradients of  <Y, dY> + lb_grad_scale * L_LB  w.r.t. x, W_l, bias, W1, W3, W2 (all tokens).
+    A dropped assignment (capacity_factor > 0) is absent from Y, so nothing flows through it; the
+    keep/drop decision itself is piecewise constant."""
     x = _f64(x)
     dy = _f64(dy)
     T, d = x.shape
@@ -310,6 +353,8 @@ def moe_backward(x, w_router, w1, w3, w2, dy, k, routing=ROUTE_TOPK, alpha=0.01,
     kk = idx.shape[1]
     gd = dense_gates(idx, g, E)
     _, u, p = lb_loss(gd, p_tok, alpha)
+    keep = capacity_keep(idx, E, expert_capacity(T, kk, E, capacity_factor)) if capacity_factor > 0 \
+        else np.ones(idx.shape, dtype=bool)
 
     dx = np.zeros_like(x)
     dw1 = np.zeros((E, F, d), dtype=_F64)
@@ -318,7 +363,7 @@ def moe_backward(x, w_router, w1, w3, w2, dy, k, routing=ROUTE_TOPK, alpha=0.01,
     dgate = np.zeros((T, kk), dtype=_F64)
     for slot in range(kk):
         for e in range(E):
-            m = idx[:, slot] == e
+            m = (idx[:, slot] == e) & keep[:, slot]
             if not np.any(m):
                 continue
             xe = x[m]
@@ -374,8 +419,9 @@ def lb_loss_grad(z, k, routing, alpha, lb_stopgrad_u=False):
 
 def moe_backward_token_slice(x, w_router, w1, w3, w2, dy, idx, gates, probs, u, p, tokens,
                              routing=ROUTE_TOPK, alpha=0.01, lb_grad_scale=1.0,
-                             lb_stopgrad_u=False):
-    """dx, dlogits and dgate for the listed tokens only, given the routing of the whole batch."""
+                             lb_stopgrad_u=False, keep=None):
+    """dx, dlogits and dgate for the listed tokens only, given the routing of the whole batch
+    (`keep`: the whole batch's capacity decisions, all kept when None)."""
     x = _f64(x)
     dy = _f64(dy)
     tok = np.asarray(tokens, dtype=np.int64)
@@ -384,11 +430,12 @@ def moe_backward_token_slice(x, w_router, w1, w3, w2, dy, idx, gates, probs, u, 
     idx = np.asarray(idx)
     g = _f64(gates)
     kk = idx.shape[1]
+    keep = np.ones(idx.shape, dtype=bool) if keep is None else np.asarray(keep, dtype=bool)
     dx = np.zeros((len(tok), x.shape[1]), dtype=_F64)
     dgate = np.zeros((len(tok), kk), dtype=_F64)
     for slot in range(kk):
         for e in range(E):
-            m = idx[tok, slot] == e
+            m = (idx[tok, slot] == e) & keep[tok, slot]
             if not np.any(m):
                 continue
             xe = x[tok[m]]
@@ -407,8 +454,8 @@ def moe_backward_token_slice(x, w_router, w1, w3, w2, dy, idx, gates, probs, u, 
     return dict(dx=dx, dlogits=dz, dgate=dgate)
 
 
-def expert_wgrad_hidden_slice(x, w1, w3, w2, dy, idx, gates, e, hidden):
-    """dW1[e, J, :], dW3[e, J, :], dW2[e, :, J] for hidden units J, over all tokens of expert e.
+def expert_wgrad_hidden_slice(x, w1, w3, w2, dy, idx, gates, e, hidden, keep=None):
+    """dW1[e, J, :], dW3[e, J, :], dW2[e, :, J] for hidden units J, over all (kept) tokens of expert e.
 
     Uses da[t, J] = g_t * sum_c dY[t, c] W2[c, J], so the cost grows with |J| only.
     """
@@ -422,8 +469,9 @@ def expert_wgrad_hidden_slice(x, w1, w3, w2, dy, idx, gates, e, hidden):
     dw3 = np.zeros((len(J), d), dtype=_F64)
     dw2 = np.zeros((d, len(J)), dtype=_F64)
     w1J, w3J, w2J = _f64(w1[e][J]), _f64(w3[e][J]), _f64(w2[e][:, J])
+    keep = np.ones(idx.shape, dtype=bool) if keep is None else np.asarray(keep, dtype=bool)
     for slot in range(idx.shape[1]):
-        m = idx[:, slot] == e
+        m = (idx[:, slot] == e) & keep[:, slot]
         if not np.any(m):
             continue
         xe = x[m]

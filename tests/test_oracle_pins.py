@@ -496,3 +496,113 @@ def test_split_and_blend_layouts_preserve_the_feed_forward_sums():
         np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
     st = o.merge_ffn_layout(w1s, w3s, w2s, o.FFN_STACK)
     assert (st[0][1] == w1s[1]).all() and (st[2][3] == w2s[3]).all()
+
+
+# ---- capacity factor (Section 4.1: Switch routing with a hard limit, beyond which tokens drop) ---
+
+def test_capacity_closed_forms_and_worked_example():
+    assert o.expert_capacity(16384, 1, 4, 1.5) == 6144           # the paper's CF on the bench batch
+    assert o.expert_capacity(10, 1, 4, 1.0) == 3                 # ceil(2.5)
+    assert o.expert_capacity(10, 2, 4, 1.0) == 5
+    assert o.expert_capacity(7, 1, 4, 0.0) == 7                  # 0 = no limit
+    idx = np.array([[0], [0], [1], [0], [1], [0], [2]])
+    keep = o.capacity_keep(idx, 3, 2)
+    assert keep[:, 0].tolist() == [True, True, True, False, True, False, True]
+    counts, offsets, perm, inv_perm = o.dispatch(idx, 3, keep)
+    assert counts.tolist() == [2, 2, 1] and offsets.tolist() == [0, 2, 4, 5]
+    assert perm.tolist() == [0, 1, 2, 4, 6, -1, -1]
+    assert inv_perm.tolist() == [0, 1, 2, -1, 3, -1, 4]
+    # top-2: slots of one token are taken in slot order
+    idx2 = np.array([[0, 1], [1, 0], [0, 1]])
+    assert o.capacity_keep(idx2, 2, 2).tolist() == [[True, True], [True, True], [False, False]]
+
+
+def test_capacity_forward_drops_exactly_the_overflow():
+    x, wr, w1, w3, w2, dy = small_problem(31, T=40, scale_r=2.0)
+    for routing, k in [(o.ROUTE_SWITCH, 1), (o.ROUTE_TOPK, 2)]:
+        free = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing, alpha=0.3)
+        # a limit nobody reaches changes nothing
+        big = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing, alpha=0.3, capacity_factor=4.0)
+        assert np.array_equal(big["y"], free["y"]) and np.array_equal(big["perm"], free["perm"])
+        cf = 0.6
+        cap = o.expert_capacity(40, k, 4, cf)
+        assert max(free["counts"]) > cap                          # the case does drop
+        lim = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing, alpha=0.3, capacity_factor=cf)
+        assert lim["counts"].tolist() == [min(int(c), cap) for c in free["counts"]]
+        # router outputs and the loss are those of the router, whatever is dropped
+        for name in ("topk_idx", "gates", "probs", "u", "p"):
+            assert np.array_equal(lim[name], free[name])
+        assert lim["lb_loss"] == free["lb_loss"]
+        # y of a token: the sum over its kept slots only, each term as without a limit
+        for t in range(40):
+            want = np.zeros(12)
+            for slot in range(k):
+                if lim["keep"][t, slot]:
+                    e = int(free["topk_idx"][t, slot])
+                    want += free["gates"][t, slot] * o.swiglu_ffn(x[t:t + 1], w1[e], w3[e], w2[e])[0]
+            np.testing.assert_allclose(lim["y"][t], want, rtol=1e-12, atol=1e-14)
+        # per expert the kept ones are the first `cap` in token order
+        for e in range(4):
+            flat = [t * k + s for t in range(40) for s in range(k) if free["topk_idx"][t, s] == e]
+            kept = [f for f in flat if lim["keep"][f // k, f % k]]
+            assert kept == flat[:cap]
+            assert lim["perm"][lim["offsets"][e]:lim["offsets"][e + 1]].tolist() == kept
+
+
+def test_capacity_backward_equals_backward_on_the_kept_sub_batch():
+    """Switch routing, alpha = 0: the step with a limit is the step without one on the kept tokens
+    (same logits), and a dropped token receives no gradient at all."""
+    x, wr, w1, w3, w2, dy = small_problem(32, T=36, scale_r=2.0)
+    cf = 0.5
+    fwd = o.moe_forward(x, wr, w1, w3, w2, k=1, routing=o.ROUTE_SWITCH, alpha=0.0, capacity_factor=cf)
+    keep = fwd["keep"][:, 0]
+    assert 0 < keep.sum() < 36
+    g = o.moe_backward(x, wr, w1, w3, w2, dy, k=1, routing=o.ROUTE_SWITCH, alpha=0.0, capacity_factor=cf)
+    sub = o.moe_backward(x[keep], wr, w1, w3, w2, dy[keep], k=1, routing=o.ROUTE_SWITCH, alpha=0.0)
+    for name in ("dw1", "dw3", "dw2", "dw_router", "dbias"):
+        np.testing.assert_allclose(g[name], sub[name], rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(g["dx"][keep], sub["dx"], rtol=1e-11, atol=1e-13)
+    assert np.all(g["dx"][~keep] == 0.0) and np.all(g["dlogits"][~keep] == 0.0)
+
+
+def test_capacity_gradients_against_finite_differences_and_slices():
+    x, wr, w1, w3, w2, G = small_problem(33, T=14, d=6, F=7, E=4, scale_r=1.5)
+    alpha, lam, cf = 0.7, 1.3, 0.6
+    z = o.router_logits(x, wr)
+    assert np.min(np.diff(np.sort(z, axis=1), axis=1)) > 1e-3
+    for routing, k in [(o.ROUTE_SWITCH, 1), (o.ROUTE_TOPK, 2)]:
+        fwd = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing, alpha=alpha, capacity_factor=cf)
+        assert not fwd["keep"].all()
+        g = o.moe_backward(x, wr, w1, w3, w2, G, k=k, routing=routing, alpha=alpha, lb_grad_scale=lam,
+                           capacity_factor=cf)
+
+        def loss():
+            out = o.moe_forward(x, wr, w1, w3, w2, k=k, routing=routing, alpha=alpha, capacity_factor=cf)
+            return float(np.sum(out["y"] * G)) + lam * out["lb_loss"]
+
+        r = RNG(5)
+        h = 1e-6
+        for pname, arr, gname in [("x", x, "dx"), ("wr", wr, "dw_router"), ("w1", w1, "dw1"), ("w3", w3, "dw3"),
+                                  ("w2", w2, "dw2")]:
+            for _ in range(8):
+                pos = tuple(int(r.integers(0, s)) for s in arr.shape)
+                old = arr[pos]
+                arr[pos] = old + h
+                lp = loss()
+                arr[pos] = old - h
+                lm = loss()
+                arr[pos] = old
+                fd = (lp - lm) / (2 * h)
+                assert abs(fd - g[gname][pos]) <= 2e-6 * max(1.0, abs(fd)), (pname, pos, fd, g[gname][pos])
+        # the slice forms agree with the full backward under a limit
+        tok = np.arange(14)
+        sl = o.moe_backward_token_slice(x, wr, w1, w3, w2, G, fwd["topk_idx"], fwd["gates"], fwd["probs"],
+                                        fwd["u"], fwd["p"], tok, routing=routing, alpha=alpha, lb_grad_scale=lam,
+                                        keep=fwd["keep"])
+        np.testing.assert_allclose(sl["dx"], g["dx"], rtol=1e-11, atol=1e-13)
+        J = np.array([1, 6])
+        for e in range(4):
+            d1, d3, d2 = o.expert_wgrad_hidden_slice(x, w1, w3, w2, G, fwd["topk_idx"], fwd["gates"], e, J,
+                                                     keep=fwd["keep"])
+            np.testing.assert_allclose(d1, g["dw1"][e][J], rtol=1e-11, atol=1e-13)
+            np.testing.assert_allclose(d2, g["dw2"][e][:, J], rtol=1e-11, atol=1e-13)
