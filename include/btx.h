@@ -61,13 +61,19 @@ typedef struct {
   int32_t skip_wgrad;         /* backward: experts frozen (the paper's freeze ablation, Section */
                               /* 4.3.1): no dW1/dW3/dW2, only dx and the router gradients       */
   float   gumbel_tau;         /* SAMPLE1 only: temperature of the Gumbel softmax; 0 = hard      */
+  float   capacity_factor;    /* 0: no limit.  > 0 (Section 4.1 uses 1.5 for Switch routing): an */
+                              /* expert accepts ceil(capacity_factor * T * k / E) assignments,   */
+                              /* taken in order of t*k+slot; the rest are dropped: they add      */
+                              /* nothing to y and receive no gradient through y.  Gates, probs,  */
+                              /* u, p and the loss stay the router's.  Not valid with SOFT.      */
 } btx_moe_desc;
 
 /* Optional routing outputs of btx_moe_forward; any member may be NULL.  All device pointers.
  *   logits[T,E], probs[T,E] (full softmax), topk_idx[T,k], gates[T,k]; counts[E] tokens per
  *   expert, offsets[E+1] exclusive scan; perm[R]: sorted row -> t*k+slot with rows ordered by
  *   (expert ascending, token ascending); inv_perm[R] its inverse; u[E], p[E], lb_loss[1] of
- *   Section 3.3. */
+ *   Section 3.3.  Under a capacity limit counts/offsets/perm cover the kept assignments only:
+ *   perm reads -1 past offsets[E] and inv_perm reads -1 for a dropped assignment. */
 typedef struct {
   float*   logits;
   int32_t* topk_idx;

@@ -33,7 +33,7 @@ class MoeDesc(C.Structure):
     _fields_ = [("T", C.c_int32), ("d_model", C.c_int32), ("d_ff", C.c_int32), ("E", C.c_int32), ("k", C.c_int32),
                 ("dtype", C.c_int32), ("routing", C.c_int32), ("lb_alpha", C.c_float),
                 ("lb_stopgrad_u", C.c_int32), ("save_for_backward", C.c_int32), ("skip_wgrad", C.c_int32),
-                ("gumbel_tau", C.c_float)]
+                ("gumbel_tau", C.c_float), ("capacity_factor", C.c_float)]
 
 
 class RoutingOut(C.Structure):
@@ -107,10 +107,10 @@ def _stream(device):
 
 
 def make_desc(T, d_model, d_ff, E, k, dtype, routing=ROUTE_TOPK, lb_alpha=0.01, lb_stopgrad_u=False,
-              save_for_backward=False, skip_wgrad=False, gumbel_tau=0.0) -> MoeDesc:
+              save_for_backward=False, skip_wgrad=False, gumbel_tau=0.0, capacity_factor=0.0) -> MoeDesc:
     code = _dtype_code(dtype) if isinstance(dtype, torch.dtype) else int(dtype)
     return MoeDesc(T, d_model, d_ff, E, k, code, routing, lb_alpha, int(lb_stopgrad_u), int(save_for_backward),
-                   int(skip_wgrad), float(gumbel_tau))
+                   int(skip_wgrad), float(gumbel_tau), float(capacity_factor))
 
 
 def btx_moe_sizes(desc: MoeDesc):

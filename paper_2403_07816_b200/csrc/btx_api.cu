@@ -1,5 +1,6 @@
 // C ABI entry points: argument validation, the buffer plan, and the launch sequences of the
 // forward and backward passes (see include/btx.h for the contract of every call).
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -20,6 +21,8 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   if (k < 1 || k > desc->E) return BTX_ERR_INVALID_ARG;
   if ((desc->routing == BTX_ROUTE_SWITCH || desc->routing == BTX_ROUTE_SAMPLE1) && k != 1) return BTX_ERR_INVALID_ARG;
   if (desc->routing == BTX_ROUTE_SAMPLE1 && (desc->gumbel_tau < 0.f || desc->lb_alpha != 0.f)) return BTX_ERR_UNSUPPORTED;
+  if (!(desc->capacity_factor >= 0.f)) return BTX_ERR_INVALID_ARG;
+  if (desc->capacity_factor > 0.f && desc->routing == BTX_ROUTE_SOFT) return BTX_ERR_INVALID_ARG;
   if (desc->E > kMaxExperts) return BTX_ERR_UNSUPPORTED;
   const int gran = desc->dtype == BTX_BF16 ? 8 : 4;         // rows must be whole 16-byte vectors
   if (!routing_only && (desc->d_model % gran || desc->d_ff % gran)) return BTX_ERR_UNSUPPORTED;
@@ -31,6 +34,12 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   p.d = routing_only ? 0 : desc->d_model;
   p.F = routing_only ? 0 : desc->d_ff;
   p.esize = desc->dtype == BTX_BF16 ? 2 : 4;
+  p.capped = desc->capacity_factor > 0.f;
+  p.capacity = p.R;
+  if (p.capped) {     // ceil(CF * T * k / E) in double; never more than the R assignments there are
+    const double c = ceil((double)desc->capacity_factor * (double)p.R / (double)p.E);
+    if (c < (double)p.R) p.capacity = (int)c;
+  }
   p.r_pad_max = (int)align_up((size_t)p.R + (size_t)p.E * (kRowTile - 1), kRowTile);
   p.mt_max = p.r_pad_max / kRowTile;
   p.nt_dact = desc->dtype == BTX_BF16 ? 2 * ((p.F + 255) / 256) : (p.F + 63) / 64;   // row-dot partials per row
@@ -199,7 +208,7 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
     if ((s = launch_expert_forward_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
   }
   mark_stage(3, st);
-  BTX_CUDA_OK(launch_combine(pl, desc->dtype, expert_rows, splits, y, st));
+  BTX_CUDA_OK(launch_combine(pl, desc->dtype, expert_rows, splits, y, b, st));
   mark_stage(4, st);
 
   if (routing) {

@@ -28,6 +28,8 @@ struct Plan {
   int wr_chunks;                     // token chunks of the router-weight gradient
   int small;                         // BF16 batch with T*k <= 1024: weight-streaming forward kernels
   int dec_s1, dec_s2;                // their contraction splits (pass 1: W1/W3, pass 2: W2)
+  int capacity;                      // rows one expert accepts (R when there is no limit)
+  int capped;                        // a capacity limit is set: assignments may be dropped
   // saved
   size_t s_topk, s_gates, s_probs, s_logits, s_u, s_p, s_loss, s_counts, s_offsets, s_pad_offsets,
       s_tile_expert, s_rowmap, s_flat2row, s_perm, s_inv_perm, s_xs, s_h1, s_h3, saved_bytes;
@@ -45,7 +47,7 @@ struct Buffers {
   float* u;           float* p;       float* loss;
   int32_t* counts;    int32_t* offsets;   int32_t* pad_offsets;   int32_t* tile_expert;
   int32_t* rowmap;    // padded sorted row -> flat assignment id (t*k+slot), -1 for padding rows
-  int32_t* flat2row;  // flat assignment id -> padded sorted row
+  int32_t* flat2row;  // flat assignment id -> padded sorted row (-1: dropped by the capacity limit)
   int32_t* perm;      int32_t* inv_perm;
   void* xs;  void* h1;  void* h3;
   int32_t* status;    float* route_part;  int32_t* perm_counts;  int32_t* perm_base;
@@ -73,7 +75,8 @@ cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, f
                                        const Buffers& b, cudaStream_t st);
 cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st);
 // y[t] = sum over slots and over `splits` partial copies ([split][R][d]) of the expert rows
-cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, cudaStream_t st);
+cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, const Buffers& b,
+                           cudaStream_t st);
 cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float alpha, float lb_scale,
                                    int stopgrad_u, int have_dg, const void* x, const void* w_router, const Buffers& b,
                                    void* dx, float* dw_router, float* dbias, float* dlogits_out, int accumulate,

@@ -201,7 +201,7 @@ swiglu_fixup_kernel(int F, int S, size_t split_stride, const float* __restrict__
                     __nv_bfloat16* __restrict__ h1s, __nv_bfloat16* __restrict__ h3s) {
   const int flat = blockIdx.y;
   const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (f >= F) return;
+  if (f >= F || flat2row[flat] < 0) return;          // a dropped assignment holds no row
   const size_t src = (size_t)flat * F + f;
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
   for (int s = 0; s < S; ++s) {

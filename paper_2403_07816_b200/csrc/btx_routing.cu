@@ -210,7 +210,7 @@ perm_count_kernel(int R, int E, int nblocks, const int32_t* __restrict__ topk, i
   if (threadIdx.x < E) perm_counts[threadIdx.x * nblocks + blockIdx.x] = hist[threadIdx.x];
 }
 
-__global__ void perm_scan_kernel(int E, int nblocks, int mt_max, const int32_t* __restrict__ perm_counts,
+__global__ void perm_scan_kernel(int E, int nblocks, int mt_max, int cap, const int32_t* __restrict__ perm_counts,
                                  int32_t* __restrict__ perm_base, int32_t* __restrict__ counts,
                                  int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
                                  int32_t* __restrict__ tile_expert) {
@@ -223,6 +223,7 @@ __global__ void perm_scan_kernel(int E, int nblocks, int mt_max, const int32_t* 
       perm_base[tid * nblocks + b] = run;
       run += perm_counts[tid * nblocks + b];
     }
+    run = min(run, cap);               // rows kept under the capacity limit
     scnt[tid] = run;
     counts[tid] = run;
   }
@@ -246,7 +247,8 @@ __global__ void perm_scan_kernel(int E, int nblocks, int mt_max, const int32_t* 
 }
 
 __global__ void __launch_bounds__(kPermThreads)
-perm_scatter_kernel(int R, int E, int nblocks, const int32_t* __restrict__ topk, const int32_t* __restrict__ perm_base,
+perm_scatter_kernel(int R, int E, int nblocks, int cap, const int32_t* __restrict__ topk,
+                    const int32_t* __restrict__ perm_base,
                     const int32_t* __restrict__ offsets, const int32_t* __restrict__ pad_offsets,
                     int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
                     int32_t* __restrict__ flat2row) {
@@ -269,13 +271,18 @@ perm_scatter_kernel(int R, int E, int nblocks, const int32_t* __restrict__ topk,
     if (i < end) {
       int before = 0;
       for (int w = 0; w < warp; ++w) before += wcnt[w][e];
-      int within = running[e] + before + rank;
-      int r = offsets[e] + within;                   // tight sorted row
-      int rp = pad_offsets[e] + within;              // padded sorted row
-      perm[r] = i;
-      inv_perm[i] = r;
-      rowmap[rp] = i;
-      flat2row[i] = rp;
+      int within = running[e] + before + rank;       // stable rank inside the expert
+      if (within < cap) {
+        int r = offsets[e] + within;                 // tight sorted row
+        int rp = pad_offsets[e] + within;            // padded sorted row
+        perm[r] = i;
+        inv_perm[i] = r;
+        rowmap[rp] = i;
+        flat2row[i] = rp;
+      } else {                                       // beyond the expert's capacity: dropped
+        inv_perm[i] = -1;
+        flat2row[i] = -1;
+      }
     }
     __syncthreads();
     if (threadIdx.x < E) {
@@ -300,7 +307,7 @@ constexpr int kSmallMaxR = 1024;
 // permutation.  Every sum runs in a fixed order, so results do not depend on which block is last.
 template <typename T>
 __global__ void __launch_bounds__(kSmallThreads)
-route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha, int mt_max, int r_pad_max,
+route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha, int mt_max, int r_pad_max, int cap,
                            const T* __restrict__ x, const T* __restrict__ wr, const float* __restrict__ bias,
                            const float* __restrict__ noise, float inv_tau, float* logits, int32_t* topk, float* gates, float* probs, float* __restrict__ u,
                            float* __restrict__ p, float* __restrict__ loss, int32_t* __restrict__ counts,
@@ -389,6 +396,8 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
   // ---- permutation: histogram, scan, stable scatter in rounds of one block ----
   if (threadIdx.x <= kMaxExperts) hist[threadIdx.x] = 0;
   for (int j = threadIdx.x; j < r_pad_max; j += kSmallThreads) rowmap[j] = -1;
+  if (cap < R)
+    for (int j = threadIdx.x; j < R; j += kSmallThreads) perm[j] = -1;
   __syncthreads();
   for (int i = threadIdx.x; i < R; i += kSmallThreads) atomicAdd(&hist[__ldcg(topk + i)], 1);
   __syncthreads();
@@ -398,7 +407,7 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
     loss[0] = (float)((double)alpha * (double)E * acc);
     int o = 0, po = 0;
     for (int q = 0; q < E; ++q) {
-      const int c = hist[q];
+      const int c = min(hist[q], cap);
       counts[q] = c; offsets[q] = o; pad_offsets[q] = po; soff[q] = o; spad[q] = po; running[q] = 0;
       o += c;
       po += (c + kRowTile - 1) / kRowTile * kRowTile;
@@ -426,8 +435,12 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
       int before = 0;
       for (int w = 0; w < warp; ++w) before += wcnt[w][e];
       const int within = running[e] + before + rank;
-      const int r = soff[e] + within, rp = spad[e] + within;
-      perm[r] = i; inv_perm[i] = r; rowmap[rp] = i; flat2row[i] = rp;
+      if (within < cap) {
+        const int r = soff[e] + within, rp = spad[e] + within;
+        perm[r] = i; inv_perm[i] = r; rowmap[rp] = i; flat2row[i] = rp;
+      } else {
+        inv_perm[i] = -1; flat2row[i] = -1;
+      }
     }
     __syncthreads();
     if (threadIdx.x < E) {
@@ -471,10 +484,12 @@ template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16*
 }
 
 // y[t, :] = sum_slot sum_split rows[split][t*k + slot, :]   (+ sum_e dz[t,e] * wr[e, :] when dz != nullptr)
+// `kept` (optional): flat assignment -> sorted row; a negative entry is a dropped assignment, whose
+// row was never written and counts as zero.
 template <typename T>
 __global__ void __launch_bounds__(256)
 combine_kernel(int Tn, int d, int k, int E, int splits, const float* __restrict__ rows, const float* __restrict__ dz,
-               const T* __restrict__ wr, T* __restrict__ y) {
+               const T* __restrict__ wr, const int32_t* __restrict__ kept, T* __restrict__ y) {
   const size_t split_stride = (size_t)Tn * k * d;
   const int vecs = d >> 2;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)Tn * vecs;
@@ -482,6 +497,7 @@ combine_kernel(int Tn, int d, int k, int E, int splits, const float* __restrict_
     int t = (int)(i / vecs), c = (int)(i % vecs) * 4;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < k; ++s) {
+      if (kept != nullptr && kept[(size_t)t * k + s] < 0) continue;
       for (int sp = 0; sp < splits; ++sp) {
         float4 v = *reinterpret_cast<const float4*>(rows + sp * split_stride + ((size_t)t * k + s) * d + c);
         acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
@@ -520,7 +536,8 @@ router_dz_kernel(int Tn, int E, int k, int routing, float alpha, float lb_scale,
     float a = 0.f;
     if (dg_part != nullptr) {
       int rp = flat2row[(size_t)t * k + s];
-      for (int n = 0; n < nt_dact; ++n) a += dg_part[(size_t)n * r_pad_max + rp];
+      if (rp >= 0)                                   // a dropped assignment has no path into y
+        for (int n = 0; n < nt_dact; ++n) a += dg_part[(size_t)n * r_pad_max + rp];
     }
     if (!stopgrad_u) a += lbc * p[topk[(size_t)t * k + s]];
     dg[s] = a;
@@ -633,12 +650,13 @@ cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, f
                                        const Buffers& b, cudaStream_t st) {
   if (dtype == BTX_BF16)
     route_permute_small_kernel<__nv_bfloat16><<<pl.T, kSmallThreads, 0, st>>>(
-        pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, (const __nv_bfloat16*)x,
+        pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, pl.capacity, (const __nv_bfloat16*)x,
         (const __nv_bfloat16*)w_router, bias, noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets,
         b.pad_offsets, b.tile_expert, b.perm, b.inv_perm, b.rowmap, b.flat2row, b.status + 8);
   else
     route_permute_small_kernel<float><<<pl.T, kSmallThreads, 0, st>>>(
-        pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, (const float*)x, (const float*)w_router, bias,
+        pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, pl.capacity, (const float*)x,
+        (const float*)w_router, bias,
         noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets, b.pad_offsets, b.tile_expert, b.perm,
         b.inv_perm, b.rowmap, b.flat2row, b.status + 8);
   return cudaGetLastError();
@@ -647,10 +665,14 @@ cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, f
 cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st) {
   cudaError_t e = cudaMemsetAsync(b.rowmap, 0xFF, (size_t)pl.r_pad_max * sizeof(int32_t), st);
   if (e != cudaSuccess) return e;
+  if (pl.capacity < pl.R) {      // the tail of perm past the kept rows reads -1
+    e = cudaMemsetAsync(b.perm, 0xFF, (size_t)pl.R * sizeof(int32_t), st);
+    if (e != cudaSuccess) return e;
+  }
   perm_count_kernel<<<pl.perm_blocks, kPermThreads, 0, st>>>(pl.R, pl.E, pl.perm_blocks, b.topk, b.perm_counts);
-  perm_scan_kernel<<<1, 256, 0, st>>>(pl.E, pl.perm_blocks, pl.mt_max, b.perm_counts, b.perm_base, b.counts,
+  perm_scan_kernel<<<1, 256, 0, st>>>(pl.E, pl.perm_blocks, pl.mt_max, pl.capacity, b.perm_counts, b.perm_base, b.counts,
                                       b.offsets, b.pad_offsets, b.tile_expert);
-  perm_scatter_kernel<<<pl.perm_blocks, kPermThreads, 0, st>>>(pl.R, pl.E, pl.perm_blocks, b.topk, b.perm_base,
+  perm_scatter_kernel<<<pl.perm_blocks, kPermThreads, 0, st>>>(pl.R, pl.E, pl.perm_blocks, pl.capacity, b.topk, b.perm_base,
                                                                b.offsets, b.pad_offsets, b.perm, b.inv_perm, b.rowmap,
                                                                b.flat2row);
   return cudaGetLastError();
@@ -664,14 +686,17 @@ cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted
   return cudaGetLastError();
 }
 
-cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, cudaStream_t st) {
+cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, const Buffers& b,
+                           cudaStream_t st) {
   size_t n = (size_t)pl.T * (pl.d / 4);
   int blocks = (int)min((n + 255) / 256, (size_t)148 * 32);
+  const int32_t* kept = pl.capped ? b.flat2row : nullptr;
   if (dtype == BTX_BF16)
-    combine_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr,
+    combine_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr, kept,
                                                           (__nv_bfloat16*)y);
   else
-    combine_kernel<float><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr, (float*)y);
+    combine_kernel<float><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr, kept,
+                                                  (float*)y);
   return cudaGetLastError();
 }
 
@@ -687,16 +712,17 @@ cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float
   float* bias_part = b.dwr_part + (size_t)pl.wr_chunks * pl.E * pl.d;
   size_t n = (size_t)pl.T * (pl.d / 4);
   int cblocks = (int)min((n + 255) / 256, (size_t)148 * 32);
+  const int32_t* kept = pl.capped ? b.flat2row : nullptr;
   if (dtype == BTX_BF16) {
     router_dw_partial_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(pl.T, pl.d, pl.E, (const __nv_bfloat16*)x, b.dz,
                                                                   b.dwr_part, bias_part);
     combine_kernel<__nv_bfloat16><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, 1, b.dxp, b.dz,
-                                                           (const __nv_bfloat16*)w_router, (__nv_bfloat16*)dx);
+                                                           (const __nv_bfloat16*)w_router, kept, (__nv_bfloat16*)dx);
   } else {
     router_dw_partial_kernel<float><<<grid, 256, 0, st>>>(pl.T, pl.d, pl.E, (const float*)x, b.dz, b.dwr_part,
                                                           bias_part);
     combine_kernel<float><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, 1, b.dxp, b.dz, (const float*)w_router,
-                                                   (float*)dx);
+                                                   kept, (float*)dx);
   }
   router_dw_reduce_kernel<<<(pl.E * pl.d + 255) / 256, 256, 0, st>>>(pl.d, pl.E, pl.wr_chunks, b.dwr_part, bias_part,
                                                                      dw_router, dbias, accumulate);

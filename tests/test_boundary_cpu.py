@@ -69,6 +69,14 @@ def test_sizes_and_argument_validation(L):
     assert ei.value.status == 1
     # soft routing ignores k
     B.btx_moe_sizes(B.make_desc(8, 256, 688, 4, 0, torch.float32, routing=B.ROUTE_SOFT))
+    # capacity factor: non-negative, and meaningless when every expert takes every token
+    B.btx_moe_sizes(B.make_desc(8, 256, 688, 4, 1, torch.float32, routing=B.ROUTE_SWITCH, capacity_factor=1.5))
+    for desc in [B.make_desc(8, 256, 688, 4, 1, torch.float32, routing=B.ROUTE_SWITCH, capacity_factor=-1.0),
+                 B.make_desc(8, 256, 688, 4, 1, torch.float32, capacity_factor=float("nan")),
+                 B.make_desc(8, 256, 688, 4, 4, torch.float32, routing=B.ROUTE_SOFT, capacity_factor=1.5)]:
+        with pytest.raises(B.BtxError) as ei:
+            B.btx_moe_sizes(desc)
+        assert ei.value.status == 1
 
 
 def test_null_and_misaligned_pointers_rejected_before_any_launch(L):

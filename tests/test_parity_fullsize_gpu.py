@@ -19,9 +19,10 @@ TOL = 1e-2
 ALPHA = 0.01
 
 
-def full_size_case(T, k, seed, routing=B.ROUTE_TOPK, bias=None, backward=True, n_tok=192, n_hidden=24, F=F, E=E):
+def full_size_case(T, k, seed, routing=B.ROUTE_TOPK, bias=None, backward=True, n_tok=192, n_hidden=24, F=F, E=E,
+                   capacity_factor=0.0):
     inp = synth.moe_inputs(T, D, F, E, seed, torch.bfloat16, DEV, with_dy=backward)
-    fwd = gpu_forward(inp, k, routing, ALPHA, bias, save=backward)
+    fwd = gpu_forward(inp, k, routing, ALPHA, bias, save=backward, capacity_factor=capacity_factor)
     r = fwd["routing"]
     kk = E if routing == B.ROUTE_SOFT else k
     cpu = {n: np64(t) for n, t in inp.items()}
@@ -34,7 +35,8 @@ def full_size_case(T, k, seed, routing=B.ROUTE_TOPK, bias=None, backward=True, n
     assert rel_err(z_gpu, o.router_logits(cpu["x"], cpu["w_router"], b64)) <= TOL
     z, idx, g, p_tok = o.route(cpu["x"], cpu["w_router"], kk, routing, b64, logits=z_gpu)
     assert np.array_equal(r.topk_idx.cpu().numpy(), idx)
-    counts, offsets, perm, inv_perm = o.dispatch(idx, E)
+    keep = o.capacity_keep(idx, E, o.expert_capacity(T, kk, E, capacity_factor)) if capacity_factor > 0 else None
+    counts, offsets, perm, inv_perm = o.dispatch(idx, E, keep)
     for name, want in [("counts", counts), ("offsets", offsets), ("perm", perm), ("inv_perm", inv_perm)]:
         assert np.array_equal(getattr(r, name).cpu().numpy(), want), name
     assert rel_err(r.gates.cpu().numpy(), g) <= 1e-5 and rel_err(r.probs.cpu().numpy(), p_tok) <= 1e-5
@@ -44,16 +46,19 @@ def full_size_case(T, k, seed, routing=B.ROUTE_TOPK, bias=None, backward=True, n
 
     # y on sampled tokens
     ref = o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], kk, routing, ALPHA,
-                        router_bias=b64, logits=z_gpu, tokens=tok)
+                        router_bias=b64, logits=z_gpu, tokens=tok, capacity_factor=capacity_factor)
     y = np64(fwd["y"])
     assert np.all(np.isfinite(y))
     e_y = np.max(np.abs(y[tok] - ref["y"])) / np.max(np.abs(ref["y"]))
     assert e_y <= TOL, f"y {e_y}"
+    if keep is not None and kk == 1:
+        dropped = torch.from_numpy(~keep[:, 0]).to(DEV)
+        assert float(fwd["y"][dropped].abs().max()) == 0.0                # a dropped token's output is exactly 0
     if not backward:
         return counts
     got = gpu_backward(inp, fwd, 1.0, bias)
     sl = o.moe_backward_token_slice(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], cpu["dy"], idx, g,
-                                    p_tok, u, p, tok, routing, ALPHA, 1.0, False)
+                                    p_tok, u, p, tok, routing, ALPHA, 1.0, False, keep=keep)
     dx = np64(got["dx"])
     assert np.all(np.isfinite(dx))
     e_dx = np.max(np.abs(dx[tok] - sl["dx"])) / np.max(np.abs(sl["dx"]))
@@ -61,7 +66,8 @@ def full_size_case(T, k, seed, routing=B.ROUTE_TOPK, bias=None, backward=True, n
     # weight gradients on sampled hidden units, over all tokens of the expert
     for e in range(E):
         J = np.sort(rng.choice(F, size=n_hidden, replace=False))
-        d1, d3, d2 = o.expert_wgrad_hidden_slice(cpu["x"], cpu["w1"], cpu["w3"], cpu["w2"], cpu["dy"], idx, g, e, J)
+        d1, d3, d2 = o.expert_wgrad_hidden_slice(cpu["x"], cpu["w1"], cpu["w3"], cpu["w2"], cpu["dy"], idx, g, e, J,
+                                                 keep=keep)
         Jt = torch.from_numpy(J).to(DEV)
         for name, want, have in [("dw1", d1, got["dw1"][e][Jt]), ("dw3", d3, got["dw3"][e][Jt]),
                                  ("dw2", d2, got["dw2"][e][:, Jt])]:
@@ -101,6 +107,21 @@ def test_skewed_top2_T16384_seed3():
     bias = synth.skew_bias(E, DEV)
     counts = full_size_case(16384, 2, seed=3, bias=bias, n_tok=128, n_hidden=16)
     assert counts[0] > 0.4 * 32768                                        # expert 0 takes the largest share
+
+
+def test_switch_capacity_factor_T16384_seed7():
+    # Section 4.1: Switch routing with capacity factor 1.5; the skewed router overflows expert 0,
+    # whose later tokens are dropped
+    bias = synth.skew_bias(E, DEV)
+    counts = full_size_case(16384, 1, seed=7, routing=B.ROUTE_SWITCH, bias=bias, n_tok=128, n_hidden=16,
+                            capacity_factor=1.5)
+    assert counts[0] == 6144 and counts.sum() < 16384
+
+
+def test_top2_capacity_factor_T4096_seed8():
+    bias = synth.skew_bias(E, DEV)
+    counts = full_size_case(4096, 2, seed=8, bias=bias, n_tok=96, n_hidden=12, capacity_factor=1.25)
+    assert counts[0] == 2560 and counts.sum() < 8192
 
 
 def test_split_expert_shapes_E8():

@@ -243,3 +243,40 @@ def test_step_host_matches_oracle(dtype, overlap):
     got = dict(out, dx=hdx)
     check_backward(cpu, None, z_ref, got, k, B.ROUTE_TOPK, 0.01, 1.0, False, tol)
     assert torch.equal(yd.cpu(), hy) and torch.equal(dxd.cpu(), hdx)
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
+@pytest.mark.parametrize("routing,k,cf", [(B.ROUTE_SWITCH, 1, 1.5), (B.ROUTE_SWITCH, 1, 0.5), (B.ROUTE_TOPK, 2, 0.75),
+                                          (B.ROUTE_TOPK, 1, 1.0)])
+def test_capacity_factor_drops_tokens(dtype, routing, k, cf):
+    """Expert capacity with token dropping (Section 4.1): kept rows, permutation and drop marks
+    bit-exact; y, dx and every gradient within tolerance; a skewed router makes expert 0 overflow."""
+    T, d, F, E = 1500, 128, 328, 4
+    inp = synth.moe_inputs(T, d, F, E, 51, dtype, DEV)
+    bias = synth.skew_bias(E, DEV)
+    tol = TOL[dtype]
+    fwd = gpu_forward(inp, k, routing, 0.01, bias, capacity_factor=cf)
+    cpu, b64, z_gpu, ref = check_forward(inp, fwd, k, routing, 0.01, bias, tol, capacity_factor=cf)
+    assert not ref["keep"].all() and (fwd["routing"].inv_perm.cpu().numpy() < 0).sum() == (~ref["keep"]).sum()
+    got = gpu_backward(inp, fwd, 1.0, bias)
+    check_backward(cpu, b64, z_gpu, got, k, routing, 0.01, 1.0, False, tol, capacity_factor=cf)
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
+def test_capacity_factor_small_batch_and_limits(dtype):
+    """The one-launch routing path (T*k <= 1024) under a limit; a limit nobody reaches changes
+    nothing; SOFT routing with a limit is refused."""
+    T, d, F, E, k = 300, 256, 512, 4, 2
+    inp = synth.moe_inputs(T, d, F, E, 52, dtype, DEV)
+    bias = synth.skew_bias(E, DEV)
+    tol = TOL[dtype]
+    fwd = gpu_forward(inp, k, B.ROUTE_TOPK, 0.01, bias, capacity_factor=0.75)
+    cpu, b64, z_gpu, ref = check_forward(inp, fwd, k, B.ROUTE_TOPK, 0.01, bias, tol, capacity_factor=0.75)
+    assert not ref["keep"].all()
+    got = gpu_backward(inp, fwd, 1.0, bias)
+    check_backward(cpu, b64, z_gpu, got, k, B.ROUTE_TOPK, 0.01, 1.0, False, tol, capacity_factor=0.75)
+    free = gpu_forward(inp, k, B.ROUTE_TOPK, 0.01, bias)
+    wide = gpu_forward(inp, k, B.ROUTE_TOPK, 0.01, bias, capacity_factor=float(E))
+    assert torch.equal(free["y"], wide["y"]) and torch.equal(free["routing"].perm, wide["routing"].perm)
+    with pytest.raises(B.BtxError):
+        gpu_forward(inp, E, B.ROUTE_SOFT, 0.01, None, capacity_factor=1.5)

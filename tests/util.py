@@ -21,11 +21,11 @@ def rel_err(got, ref):
 
 
 def gpu_forward(inp, k, routing=B.ROUTE_TOPK, alpha=0.01, bias=None, save=True, stopgrad_u=False, skip_wgrad=False,
-                noise=None, tau=0.0):
+                noise=None, tau=0.0, capacity_factor=0.0):
     x = inp["x"]
     T, d = x.shape
     E, F, _ = inp["w1"].shape
-    desc = B.make_desc(T, d, F, E, k, x.dtype, routing, alpha, stopgrad_u, save, skip_wgrad, tau)
+    desc = B.make_desc(T, d, F, E, k, x.dtype, routing, alpha, stopgrad_u, save, skip_wgrad, tau, capacity_factor)
     ws, saved = B.alloc_buffers(desc, x.device)
     ws.fill_(0x7F)           # poison: results must not depend on scratch contents
     saved.fill_(0x7F)
@@ -61,7 +61,7 @@ def np64(t):
     return synth.to_f64_numpy(t)
 
 
-def check_forward(inp, fwd, k, routing, alpha, bias, tol, noise=None, tau=1.0):
+def check_forward(inp, fwd, k, routing, alpha, bias, tol, noise=None, tau=1.0, capacity_factor=0.0):
     """Parity protocol: logits by tolerance; routing and permutation bit-exact given the GPU's
     fp32 logits; gates, probabilities, loss and y by tolerance."""
     r = fwd["routing"]
@@ -72,7 +72,7 @@ def check_forward(inp, fwd, k, routing, alpha, bias, tol, noise=None, tau=1.0):
     assert rel_err(z_gpu, z_ref) <= tol, "logits"
     n64 = None if noise is None else np64(noise)
     ref = o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], k, routing, alpha,
-                        router_bias=b64, logits=z_gpu, noise=n64, tau=tau)
+                        router_bias=b64, logits=z_gpu, noise=n64, tau=tau, capacity_factor=capacity_factor)
     for name, got in [("topk_idx", r.topk_idx), ("counts", r.counts), ("offsets", r.offsets), ("perm", r.perm),
                       ("inv_perm", r.inv_perm)]:
         assert np.array_equal(got.cpu().numpy(), ref[name]), name
@@ -86,10 +86,12 @@ def check_forward(inp, fwd, k, routing, alpha, bias, tol, noise=None, tau=1.0):
     return cpu, b64, z_gpu, ref
 
 
-def check_backward(cpu, b64, z_gpu, got, k, routing, alpha, lb_scale, stopgrad_u, tol, base=None, noise=None, tau=1.0):
+def check_backward(cpu, b64, z_gpu, got, k, routing, alpha, lb_scale, stopgrad_u, tol, base=None, noise=None, tau=1.0,
+                   capacity_factor=0.0):
     n64 = None if noise is None else np64(noise)
     ref = o.moe_backward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], cpu["dy"], k, routing, alpha,
-                         lb_scale, stopgrad_u, router_bias=b64, logits=z_gpu, noise=n64, tau=tau)
+                         lb_scale, stopgrad_u, router_bias=b64, logits=z_gpu, noise=n64, tau=tau,
+                         capacity_factor=capacity_factor)
     errs = {}
     for name in ("dx", "dw_router", "dbias", "dw1", "dw3", "dw2"):
         if got[name] is None:
