@@ -13,6 +13,8 @@ namespace btx {
 constexpr int kRowTile = 256;        // expert segments of the sorted buffers are padded to this many rows
 constexpr int kMaxExperts = 32;
 constexpr int kStatusWords = 64;     // first 256 bytes of every workspace: device status block
+                                     // (word 0: error code; word 8: ticket of the one-launch routing;
+constexpr int kTileCounterWord = 16; //  words 16..23: tile counters of a call's tensor-core launches)
 
 // ---------------------------------------------------------------------------------------------
 // Buffer plan.  All offsets are bytes from the start of `saved` / `workspace`.

@@ -40,7 +40,9 @@ constexpr int BN = 256, STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / 2) * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int EPI_WARPS = 8;
 constexpr int TC_THREADS = 64 + EPI_WARPS * 32;
+constexpr int SCHED_SLOTS = 4;                           // tile numbers in flight between the scheduler and its readers
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+static_assert(STAGES * 16 + 48 + SCHED_SLOTS * 20 <= 256, "control block fits behind the ring");
 constexpr int GROUP_N = 8;                               // column tiles per raster group
 static_assert(2 * BM == kRowTile, "a CTA pair covers one padded row tile");
 
@@ -67,11 +69,15 @@ struct TcParams {
   int save, accumulate;
   int wide;                     // all epilogue rows start on 32-byte boundaries
   int32_t* status;
+  int32_t* next_tile;           // tile counter of this launch (zero when the kernel starts)
 };
 
 // ---------------------------------------------------------------------------------------------
-// Tile schedule: the same function is evaluated by the producer, the MMA issuer and the epilogue
-// of both CTAs.  A tile is 256 output rows (128 per CTA) by 256 columns.
+// Tile schedule.  A tile is 256 output rows (128 per CTA) by 256 columns; tiles are numbered in
+// raster order (get_tile).  CTA pairs draw tile numbers from one global counter, so the tiles in
+// flight are always a contiguous window of the raster, whose operand panels fit in L2, however the
+// pairs' speeds differ.  The leader's producer thread draws the number and posts it to both CTAs
+// (TileFeed); the other producer, the MMA issuer and the epilogue warps read it from there.
 // ---------------------------------------------------------------------------------------------
 struct Tile {
   int m0;        // first output row of the pair's tile
@@ -80,6 +86,42 @@ struct Tile {
   int k_base;    // WGRAD: first contraction row
   int kb;        // K blocks
 };
+
+struct TileFeed {
+  uint32_t full, empty, slots;     // shared-memory addresses: SCHED_SLOTS barriers, barriers, words
+  uint32_t empty_leader;           // `empty` in the leader CTA (shared::cluster address)
+  uint32_t q, phase;
+  volatile int* abort_flag;
+  int32_t* status;
+
+  __device__ __forceinline__ void init(uint32_t ctl_addr, volatile int* af, int32_t* st) {
+    full = ctl_addr; empty = full + SCHED_SLOTS * 8; slots = empty + SCHED_SLOTS * 8;
+    empty_leader = map_to_cta(empty, 0);
+    q = 0; phase = 0; abort_flag = af; status = st;
+  }
+  __device__ __forceinline__ void advance() { if (++q == SCHED_SLOTS) { q = 0; phase ^= 1u; } }
+  // Scheduler (one thread of the leader): next tile number, posted to both CTAs.  -1 on time-out.
+  __device__ __forceinline__ int draw(int32_t* counter) {
+    if (!mbar_wait(empty + q * 8, phase ^ 1u, abort_flag, status)) return -1;
+    const int t = atomicAdd(counter, 1);
+    post_word(slots + q * 4, full + q * 8, 0, (uint32_t)t);
+    post_word(slots + q * 4, full + q * 8, 1, (uint32_t)t);
+    advance();
+    return t;
+  }
+  // Reader: the next posted tile number.  Called by one thread (whole_warp = false) or by all 32
+  // lanes of a warp; one arrival per caller group hands the slot back.  -1 on time-out.
+  __device__ __forceinline__ int next(bool whole_warp, bool releaser) {
+    if (!mbar_wait(full + q * 8, phase, abort_flag, status)) return -1;
+    const int t = (int)ld_shared_u32(slots + q * 4);
+    if (whole_warp) __syncwarp();
+    if (releaser) mbar_arrive_cluster(empty_leader + q * 8);
+    advance();
+    return t;
+  }
+};
+// readers per slot: the peer's producer, the leader's MMA issuer, the epilogue warps of both CTAs
+constexpr int SCHED_READERS = 2 + 2 * EPI_WARPS;
 
 template <int MODE>
 __device__ __forceinline__ int total_tiles(const TcParams& p) {
@@ -136,16 +178,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const uint32_t bar_tempty = bar_tfull + 16;                           // 2 x 8 B (used in the leader)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + STAGES * 16 + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + STAGES * 16 + 40);
+  TileFeed feed;
+  feed.init(bar_full + STAGES * 16 + 48, abort_flag, p.status);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();                              // 0 = leader of the pair
-  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   constexpr bool A_MN = (MODE == G_WGRAD);
   constexpr bool B_MN = (MODE == G_DACT || MODE == G_DX || MODE == G_WGRAD);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + s * 8, 1); mbar_init(bar_empty + s * 8, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + a * 8, 1); mbar_init(bar_tempty + a * 8, 2 * EPI_WARPS * 32); }
+    for (int s = 0; s < SCHED_SLOTS; ++s) { mbar_init(feed.full + s * 8, 1); mbar_init(feed.empty + s * 8, SCHED_READERS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -167,7 +211,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       uint32_t stage = 0, phase = 0;
       uint32_t uses = 0;                                  // stages filled so far (for the final drain)
       bool ok = true;
-      for (int t = pair; t < n_total && ok; t += n_pairs) {
+      while (ok) {
+        const int t = rank == 0 ? feed.draw(p.next_tile) : feed.next(false, true);
+        if (t < 0 || t >= n_total) break;                 // timed out, or the raster is exhausted
         const Tile tl = get_tile<MODE>(p, t);
         const int m0 = tl.m0 + (int)rank * BM;            // this CTA's rows
         for (int kb = 0; kb < tl.kb; ++kb) {
@@ -225,7 +271,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                                  ((uint32_t)((2 * BM) >> 4) << 24);
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
-      for (int t = pair; t < n_total && ok; t += n_pairs) {
+      while (ok) {
+        const int t = feed.next(false, true);
+        if (t < 0 || t >= n_total) break;
         const Tile tl = get_tile<MODE>(p, t);
         if (tl.kb == 0) continue;
         if (!(ok = mbar_wait(bar_tempty + acc * 8, acc_phase ^ 1u, abort_flag, p.status))) break;
@@ -261,7 +309,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     const uint32_t tempty_leader = map_to_cta(bar_tempty, 0);
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
-    for (int t = pair; t < n_total && ok; t += n_pairs) {
+    while (ok) {
+      const int t = feed.next(true, lane == 0);
+      if (t < 0 || t >= n_total) break;
       const Tile tl = get_tile<MODE>(p, t);
       const bool have_acc = tl.kb > 0;
       if (have_acc) {
@@ -406,7 +456,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 
 template <int MODE>
 btx_status launch_tc(const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0, const CUtensorMap& b1,
-                     const TcParams& p, int max_tiles, cudaStream_t st) {
+                     const TcParams& params, int max_tiles, int launch_index, cudaStream_t st) {
+  // every launch of one forward or backward call draws from its own counter in the status block,
+  // which the call zeroed before its first kernel
+  TcParams p = params;
+  p.next_tile = params.status + kTileCounterWord + launch_index;
   if (cudaFuncSetAttribute(tc_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
     return BTX_ERR_CUDA;
   int pairs = sm_count() / 2;
@@ -440,13 +494,13 @@ btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void
   p.o0 = (__nv_bfloat16*)b.act; p.o1 = (__nv_bfloat16*)b.h1; p.o2 = (__nv_bfloat16*)b.h3; p.save = save;
   const bool f_pitch32 = pl.F % 16 == 0;                  // bf16 rows of F elements start on 32-byte boundaries
   p.wide = f_pitch32 && aligned32(b.act) && aligned32(b.h1) && aligned32(b.h3);
-  if ((s = launch_tc<G_FWD1>(a, a, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
+  if ((s = launch_tc<G_FWD1>(a, a, b0, b1, p, pl.mt_max * p.n_tiles, 0, st)) != BTX_OK) return s;
   mark_stage(2, st);
   // GEMM-2: gate-scaled expert rows = act W2^T
   if (!make_map(&a, b.act, F, RP, 0, 64, 128) || !make_map(&b0, w2, F, d, E, 64, 128)) return BTX_ERR_CUDA;
   p.n_tiles = (pl.d + BN - 1) / BN; p.kb_total = (pl.F + BK - 1) / BK; p.N = pl.d; p.of = b.yp;
   p.wide = aligned32(b.yp);                               // fp32 rows of d (a multiple of 8) elements
-  return launch_tc<G_FWD2>(a, a, b0, b0, p, pl.mt_max * p.n_tiles, st);
+  return launch_tc<G_FWD2>(a, a, b0, b0, p, pl.mt_max * p.n_tiles, 1, st);
 }
 
 btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
@@ -462,7 +516,7 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   p.h1 = (const __nv_bfloat16*)b.h1; p.h3 = (const __nv_bfloat16*)b.h3;
   p.o0 = (__nv_bfloat16*)b.dh1; p.o1 = (__nv_bfloat16*)b.dh3; p.o2 = (__nv_bfloat16*)b.ga; p.dg_part = b.dg_part;
   p.wide = pl.F % 16 == 0 && aligned32(b.h1) && aligned32(b.h3) && aligned32(b.dh1) && aligned32(b.dh3) && aligned32(b.ga);
-  if ((s = launch_tc<G_DACT>(a0, a0, b0, b0, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
+  if ((s = launch_tc<G_DACT>(a0, a0, b0, b0, p, pl.mt_max * p.n_tiles, 0, st)) != BTX_OK) return s;
   mark_stage(2, st);
   // dgrad-1: dXs = dh1 W1 + dh3 W3 (weights read N-major), scatter to t*k+slot rows
   if (!make_map(&a0, b.dh1, F, RP, 0, 64, 128) || !make_map(&a1, b.dh3, F, RP, 0, 64, 128) ||
@@ -470,7 +524,7 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
     return BTX_ERR_CUDA;
   p.n_tiles = (pl.d + BN - 1) / BN; p.kb_half = (pl.F + BK - 1) / BK; p.kb_total = 2 * p.kb_half; p.N = pl.d;
   p.of = b.dxp; p.wide = aligned32(b.dxp);
-  if ((s = launch_tc<G_DX>(a0, a1, b0, b1, p, pl.mt_max * p.n_tiles, st)) != BTX_OK) return s;
+  if ((s = launch_tc<G_DX>(a0, a1, b0, b1, p, pl.mt_max * p.n_tiles, 1, st)) != BTX_OK) return s;
   mark_stage(3, st);
   if (skip_wgrad) return BTX_OK;
   // wgrads: contraction over the expert's padded token rows, both operands MN-major.  The operand
@@ -479,16 +533,16 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   p.accumulate = accumulate;
   if (!make_map(&a0, b.ga, F, RP, 0, 64, 64) || !make_map(&b0, b.dys, d, RP, 0, 64, 64)) return BTX_ERR_CUDA;
   p.M = pl.F; p.N = pl.d; p.m_tiles = (pl.F + kRowTile - 1) / kRowTile; p.n_tiles = (pl.d + BN - 1) / BN; p.of = dw2;
-  if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
+  if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, 2, st)) != BTX_OK) return s;
   mark_stage(4, st);
   if (!make_map(&a0, b.xs, d, RP, 0, 64, 64) || !make_map(&b0, b.dh1, F, RP, 0, 64, 64) ||
       !make_map(&b1, b.dh3, F, RP, 0, 64, 64))
     return BTX_ERR_CUDA;
   p.M = pl.d; p.N = pl.F; p.m_tiles = (pl.d + kRowTile - 1) / kRowTile; p.n_tiles = (pl.F + BN - 1) / BN; p.of = dw1;
-  if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, st)) != BTX_OK) return s;
+  if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, 3, st)) != BTX_OK) return s;
   mark_stage(5, st);
   p.of = dw3;
-  s = launch_tc<G_WGRAD>(a0, a0, b1, b1, p, pl.E * p.m_tiles * p.n_tiles, st);
+  s = launch_tc<G_WGRAD>(a0, a0, b1, b1, p, pl.E * p.m_tiles * p.n_tiles, 4, st);
   mark_stage(6, st);
   return s;
 }

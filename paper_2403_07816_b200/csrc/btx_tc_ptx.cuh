@@ -46,6 +46,21 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Hand one 32-bit word to CTA `rank` of the cluster: the word lands in that CTA's shared memory at
+// `slot` and completes 4 bytes on its barrier `bar` (same offsets as in this CTA), which this call
+// arms with one arrival; a thread that waits on the barrier then sees the word.
+__device__ __forceinline__ void post_word(uint32_t slot, uint32_t bar, uint32_t rank, uint32_t value) {
+  const uint32_t rslot = map_to_cta(slot, rank), rbar = map_to_cta(bar, rank);
+  asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(rbar), "r"(4u)
+               : "memory");
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+               ::"r"(rslot), "r"(value), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
 // One poll of the barrier.  The hint lets the hardware park the thread (up to about 10 us) until
 // the phase completes instead of spinning on shared memory.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
