@@ -30,6 +30,9 @@ WORKLOADS = {
     "decode": (32, 4096, 11008, 4, 2, 4),
 }
 ALPHA = 0.01
+# dram__bytes_read.sum + dram__bytes_write.sum of the seven tc_gemm_kernel launches of one training step
+# at T=16384 (26.38 GB read + 7.43 GB written); the algorithmic minimum is 10.3 GB read + 7.6 GB written
+TC_GEMM_DRAM_BYTES_PER_STEP = 33.81e9
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -322,8 +325,11 @@ def run_moe(args, workload):
         achieved = flops_step / (gemm_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops_sustained"]
         line["stages_ms"] = {kname: round(v, 4) for kname, v in stages.items()}
+        # DRAM bytes (read + write) of the seven launches of one step, from the ncu capture summarised in
+        # profiles/tc_gemm_kernel_fwd_bwd_T16384_dram.txt; it holds for that workload only
+        traffic = TC_GEMM_DRAM_BYTES_PER_STEP if (train and (T, d, F, E, k) == (16384, 4096, 11008, 4, 2)) else None
         line["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                            "frac": achieved / peak, "traffic": None, "peak_source": peaks["_source"] + " sustained",
+                            "frac": achieved / peak, "traffic": traffic, "peak_source": peaks["_source"] + " sustained",
                             "kernel": f"tc_gemm_kernel, {len(gemm_keys)} launches per step (flops of all / summed time)",
                             "frac_of_nominal_2250": achieved / 2250.0}
 

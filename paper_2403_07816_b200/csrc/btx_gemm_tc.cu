@@ -7,7 +7,8 @@
 // single-CTA 128 x 256 tile needs, and each CTA keeps a 128 x 256 fp32 accumulator in its TMEM.
 //
 //   warp 0      TMA producer (one lane): fills a 6-stage ring of (A 128x64, B 128x64) bf16 tiles;
-//               both CTAs signal the leader CTA's "full" barrier
+//               both CTAs signal the leader CTA's "full" barrier.  The leader's producer also
+//               draws the pair's next tile from a global counter and posts it to every role
 //   warp 1      allocates TMEM; in the leader CTA one lane issues the MMAs for the pair and
 //               commits (multicast) to the barriers of both CTAs
 //   warps 2-9   epilogue: tcgen05.ld of the CTA's accumulator (one row per thread, two warps per
