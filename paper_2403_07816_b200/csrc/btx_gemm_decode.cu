@@ -76,19 +76,34 @@ tc_swapk_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  allow_dependents();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < D_STAGES; ++s) { mbar_init(bar_full + s * 8, 1); mbar_init(bar_empty + s * 8, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + a * 8, 1); mbar_init(bar_tempty + a * 8, 2 * D_EPI_WARPS * 32); }
     *abort_flag = 0;
-    // expert segments start with their real rows, so a chunk holds tokens iff its first row does
-    int n = 0;
-    const int all = p.pad_offsets[p.E] / TOK;
-    for (int c = 0; c < all && n < D_MAX_CHUNKS; ++c)
-      if (p.rowmap[c * TOK] >= 0) chunks[1 + n++] = c;
-    chunks[0] = n;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  // Barriers and TMEM are set up while the kernel before this one may still run; everything below
+  // reads what it wrote.
+  grid_dependency_wait();
+  if (warp == 0) {
+    // List of the chunks that hold tokens (expert segments start with their real rows, so a chunk
+    // holds tokens iff its first row does).  The 32 lanes probe 32 chunks at a time: one round of
+    // global-memory latency instead of one per chunk, which used to dominate the kernel's start.
+    __syncwarp();
+    const int all = p.pad_offsets[p.E] / TOK;
+    int n = 0;
+    for (int c0 = 0; c0 < all; c0 += 32) {
+      const int c = c0 + lane;
+      const bool holds = c < all && p.rowmap[c * TOK] >= 0;
+      const unsigned m = __ballot_sync(0xffffffffu, holds);
+      const int pos = n + __popc(m & ((1u << lane) - 1u));
+      if (holds && pos < D_MAX_CHUNKS) chunks[1 + pos] = c;
+      n += __popc(m);
+    }
+    if (lane == 0) chunks[0] = min(n, D_MAX_CHUNKS);
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
@@ -201,6 +216,8 @@ swiglu_fixup_kernel(int F, int S, size_t split_stride, const float* __restrict__
                     __nv_bfloat16* __restrict__ h1s, __nv_bfloat16* __restrict__ h3s) {
   const int flat = blockIdx.y;
   const int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  allow_dependents();
+  grid_dependency_wait();
   if (f >= F || flat2row[flat] < 0) return;          // a dropped assignment holds no row
   const size_t src = (size_t)flat * F + f;
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
@@ -229,8 +246,8 @@ btx_status launch_swapk(const CUtensorMap& w0, const CUtensorMap& w1, const CUte
     return BTX_ERR_CUDA;
   int pairs = sm_count() / 2;
   if (pairs < 1) pairs = 1;
-  tc_swapk_kernel<<<2 * pairs, D_THREADS, D_SMEM_BYTES, st>>>(w0, w1, x, p);
-  return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
+  return launch_after_predecessor(tc_swapk_kernel, dim3(2 * pairs), dim3(D_THREADS), D_SMEM_BYTES, st, true, w0, w1, x,
+                                  p) == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
 }
 
 }  // namespace
@@ -268,10 +285,12 @@ btx_status launch_expert_forward_small_bf16(const Plan& pl, const void* w1, cons
   p.split_stride = (size_t)pl.R * pl.F;
   p.out0 = b.part; p.out1 = b.part + (size_t)pl.dec_s1 * p.split_stride; p.gates = nullptr;
   if ((s = launch_swapk(m0, m1, mx, p, st)) != BTX_OK) return s;
-  swiglu_fixup_kernel<<<dim3((pl.F / 4 + 255) / 256, pl.R), 256, 0, st>>>(
-      pl.F, pl.dec_s1, p.split_stride, p.out0, p.out1, b.flat2row, (__nv_bfloat16*)b.act,
-      save ? (__nv_bfloat16*)b.h1 : nullptr, save ? (__nv_bfloat16*)b.h3 : nullptr);
-  if (cudaGetLastError() != cudaSuccess) return BTX_ERR_CUDA;
+  if (launch_after_predecessor(swiglu_fixup_kernel, dim3((pl.F / 4 + 255) / 256, pl.R), dim3(256), 0, st, true, pl.F,
+                               pl.dec_s1, p.split_stride, (const float*)p.out0, (const float*)p.out1,
+                               (const int32_t*)b.flat2row, (__nv_bfloat16*)b.act,
+                               save ? (__nv_bfloat16*)b.h1 : (__nv_bfloat16*)nullptr,
+                               save ? (__nv_bfloat16*)b.h3 : (__nv_bfloat16*)nullptr) != cudaSuccess)
+    return BTX_ERR_CUDA;
   mark_stage(2, st);
   // pass 2: partial gate-scaled expert rows
   if (!make_map(&m0, w2, F, d, E, 64, WM) || !make_map(&mx, b.act, F, RP, 0, 64, TOK / 2)) return BTX_ERR_CUDA;

@@ -326,6 +326,7 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = blockIdx.x;
   const int R = Tn * k;
+  allow_dependents();
 
   const T* xr = x + (size_t)t * d;
   for (int eb = 0; eb < E; eb += 8) {
@@ -459,6 +460,8 @@ __global__ void __launch_bounds__(256)
 gather_rows_kernel(int k, int row_vecs, const uint4* __restrict__ src, uint4* __restrict__ dst,
                    const int32_t* __restrict__ rowmap, const int32_t* __restrict__ pad_offsets, int E) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  allow_dependents();
+  grid_dependency_wait();
   const int total = pad_offsets[E];
   for (int rp = blockIdx.x * 8 + warp; rp < total; rp += gridDim.x * 8) {
     int flat = rowmap[rp];
@@ -492,6 +495,8 @@ combine_kernel(int Tn, int d, int k, int E, int splits, const float* __restrict_
                const T* __restrict__ wr, const int32_t* __restrict__ kept, T* __restrict__ y) {
   const size_t split_stride = (size_t)Tn * k * d;
   const int vecs = d >> 2;
+  allow_dependents();
+  grid_dependency_wait();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)Tn * vecs;
        i += (size_t)gridDim.x * blockDim.x) {
     int t = (int)(i / vecs), c = (int)(i % vecs) * 4;
@@ -681,9 +686,10 @@ cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st) {
 cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st) {
   int row_vecs = pl.d * pl.esize / 16;
   int blocks = min(pl.r_pad_max / 8, 148 * 16);
-  gather_rows_kernel<<<blocks, 256, 0, st>>>(pl.k, row_vecs, (const uint4*)src, (uint4*)dst_sorted, b.rowmap,
-                                             b.pad_offsets, pl.E);
-  return cudaGetLastError();
+  // small batches: the gather's launch overlaps the routing kernel's run
+  return launch_after_predecessor(gather_rows_kernel, dim3(blocks), dim3(256), 0, st, pl.small != 0, pl.k, row_vecs,
+                                  (const uint4*)src, (uint4*)dst_sorted, (const int32_t*)b.rowmap,
+                                  (const int32_t*)b.pad_offsets, pl.E);
 }
 
 cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, const Buffers& b,
@@ -692,11 +698,10 @@ cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int spl
   int blocks = (int)min((n + 255) / 256, (size_t)148 * 32);
   const int32_t* kept = pl.capped ? b.flat2row : nullptr;
   if (dtype == BTX_BF16)
-    combine_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr, kept,
-                                                          (__nv_bfloat16*)y);
-  else
-    combine_kernel<float><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr, kept,
-                                                  (float*)y);
+    return launch_after_predecessor(combine_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, pl.small != 0, pl.T,
+                                    pl.d, pl.k, pl.E, splits, rows, (const float*)nullptr,
+                                    (const __nv_bfloat16*)nullptr, kept, (__nv_bfloat16*)y);
+  combine_kernel<float><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr, kept, (float*)y);
   return cudaGetLastError();
 }
 
