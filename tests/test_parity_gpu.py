@@ -46,6 +46,15 @@ def test_ragged_shapes(dtype, T, d, F, E, k):
 
 
 @pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
+@pytest.mark.parametrize("T,d,F,routing,k", [(200, 72, 40, B.ROUTE_TOPK, 8), (150, 64, 72, B.ROUTE_SOFT, 32),
+                                             (40, 8, 8, B.ROUTE_TOPK, 32), (2500, 64, 64, B.ROUTE_SWITCH, 1)])
+def test_maximum_expert_count_and_smallest_widths(dtype, T, d, F, routing, k):
+    """E = 32 (the library's limit): sparse loads with experts that receive nothing, every expert
+    selected (k = E), rows of a single 16-byte vector, and more padded row tiles than tokens."""
+    run_case(T, d, F, 32, k, dtype, seed=17, routing=routing, alpha=0.05, lb_scale=0.7)
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
 def test_switch_routing(dtype):
     run_case(200, 128, 136, 4, 1, dtype, seed=3, routing=B.ROUTE_SWITCH, alpha=0.02)
 
