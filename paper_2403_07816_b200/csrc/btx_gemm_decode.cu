@@ -252,7 +252,10 @@ btx_status launch_swapk(const CUtensorMap& w0, const CUtensorMap& w1, const CUte
 
 }  // namespace
 
-// Number of contraction splits that makes base_tiles * S fill whole rounds of the CTA pairs.
+// Smallest number of contraction splits with which base_tiles * S work items keep at least 85 % of
+// the CTA pairs busy in every round.  That is enough to saturate HBM: at the Llama-2-7B shape one
+// un-split round of 64 items on 74 pairs streams W2 as fast as 512 items in seven rounds did, and
+// fewer splits mean fewer partial products to write and to sum.
 int pick_decode_splits(int base_tiles, int kb_total) {
   const int pairs = 74;                                   // 148 SMs; only a balance heuristic
   int best = 1;
@@ -261,7 +264,7 @@ int pick_decode_splits(int base_tiles, int kb_total) {
     const int tiles = base_tiles * S;
     const double eff = (double)tiles / (double)(((tiles + pairs - 1) / pairs) * pairs);
     if (eff > best_eff + 1e-9) { best_eff = eff; best = S; }
-    if (eff >= 0.96) return S;
+    if (eff >= 0.85) return S;
   }
   return best;
 }
