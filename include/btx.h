@@ -11,6 +11,9 @@
  *   - Element type of x, weights, y, dy, dx is given by btx_moe_desc.dtype (BTX_F32: float,
  *     BTX_BF16: bfloat16 with fp32 accumulation).  Logits, gates, probabilities, the loss and all
  *     weight gradients are fp32.  Index outputs are int32.
+ *   - A `workspace` serves one call at a time (its first 256 bytes hold the device status word,
+ *     a routing ticket and the tile counters of the call's kernels); calls that may overlap on the
+ *     GPU, e.g. on different streams, need a workspace (and `saved` buffer) each.
  *   - Errors: a btx_status is returned; nothing is launched when it is not BTX_OK.  Device-side
  *     bounded waits that expire are recorded in the workspace and read with btx_device_status.
  *

@@ -290,7 +290,11 @@ extern "C" btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_
   cudaStream_t cs = (cudaStream_t)copy_stream;
   const bool overlap = copy_stream != nullptr && copy_stream != stream;
   const size_t act_bytes = (size_t)pl.T * pl.d * pl.esize;
-  cudaEvent_t ev_start = nullptr, ev_dy = nullptr, ev_fwd = nullptr, ev_y = nullptr;
+  struct Events {                     // destroyed on every return path; destruction waits for nothing
+    cudaEvent_t e[4] = {nullptr, nullptr, nullptr, nullptr};
+    ~Events() { for (cudaEvent_t x : e) if (x) cudaEventDestroy(x); }
+  } evs;
+  cudaEvent_t &ev_start = evs.e[0], &ev_dy = evs.e[1], &ev_fwd = evs.e[2], &ev_y = evs.e[3];
   if (overlap) {
     // dy travels to the device while the forward runs, y travels back while the backward runs
     const unsigned f = cudaEventDisableTiming;
@@ -325,7 +329,6 @@ extern "C" btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_
   BTX_CUDA_OK(cudaMemcpyAsync(loss_host, (const char*)saved + pl.s_loss, 4, cudaMemcpyDeviceToHost, st));
   if (overlap) {
     BTX_CUDA_OK(cudaStreamWaitEvent(st, ev_y, 0));          // everything is complete when `stream` is
-    cudaEventDestroy(ev_start); cudaEventDestroy(ev_dy); cudaEventDestroy(ev_fwd); cudaEventDestroy(ev_y);
   }
   return BTX_OK;
 }
