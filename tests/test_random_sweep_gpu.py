@@ -1,0 +1,67 @@
+"""Seeded sweep over combinations of the layer's options (routing mode, k, bias, capacity limit,
+frozen experts, accumulation, loss settings) at ragged shapes: every case is compared with the
+oracle exactly as the single-feature tests do.  Plus run-to-run bit-exactness of the BF16
+tensor-core path, whose tiles are handed to CTA pairs in an order that differs between runs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2403_07816_b200 import binding as B
+from paper_2403_07816_b200 import synth
+from util import TOL, check_backward, check_forward, gpu_backward, gpu_forward
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def make_cases(n, seed):
+    r = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        E = int(r.integers(1, 13))
+        routing = [B.ROUTE_TOPK, B.ROUTE_TOPK, B.ROUTE_SWITCH, B.ROUTE_SOFT, B.ROUTE_SAMPLE1][int(r.integers(0, 5))]
+        k = int(r.integers(1, E + 1)) if routing == B.ROUTE_TOPK else (E if routing == B.ROUTE_SOFT else 1)
+        c = dict(T=int(r.integers(96, 1400)), d=8 * int(r.integers(2, 33)), F=8 * int(r.integers(2, 49)), E=E, k=k,
+                 routing=routing, seed=1000 + i,
+                 alpha=0.0 if routing == B.ROUTE_SAMPLE1 else float(r.choice([0.0, 0.01, 0.3])),
+                 tau=float(r.choice([0.0, 0.6, 1.4])) if routing == B.ROUTE_SAMPLE1 else 0.0,
+                 bias=bool(r.integers(0, 2)), stopgrad=bool(r.integers(0, 2)), frozen=bool(r.integers(0, 2)),
+                 accumulate=bool(r.integers(0, 2)), lb_scale=float(r.choice([1.0, 0.4, 2.5])),
+                 cf=0.0 if routing == B.ROUTE_SOFT else float(r.choice([0.0, 0.0, 0.6, 1.0, 1.5])))
+        cases.append(c)
+    return cases
+
+
+CASES = make_cases(14, 20240311)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("c", CASES, ids=[f"case{i}" for i in range(len(CASES))])
+def test_option_combinations(c, dtype):
+    inp = synth.moe_inputs(c["T"], c["d"], c["F"], c["E"], c["seed"], dtype, DEV)
+    tol = TOL[dtype]
+    bias = synth.normal((c["E"],), 0.5, c["seed"], 77, torch.float32, DEV) if c["bias"] else None
+    noise = synth.gumbel_noise(c["T"], c["E"], c["seed"], DEV) if c["routing"] == B.ROUTE_SAMPLE1 else None
+    fwd = gpu_forward(inp, c["k"], c["routing"], c["alpha"], bias, save=True, stopgrad_u=c["stopgrad"],
+                      skip_wgrad=c["frozen"], noise=noise, tau=c["tau"], capacity_factor=c["cf"])
+    cpu, b64, z_gpu, ref = check_forward(inp, fwd, c["k"], c["routing"], c["alpha"], bias, tol, noise=noise,
+                                         tau=c["tau"], capacity_factor=c["cf"])
+    init = 0.25 if c["accumulate"] else None
+    got = gpu_backward(inp, fwd, c["lb_scale"], bias, accumulate=c["accumulate"], init=init)
+    check_backward(cpu, b64, z_gpu, got, c["k"], c["routing"], c["alpha"], c["lb_scale"], c["stopgrad"], tol,
+                   base=init, noise=noise, tau=c["tau"], capacity_factor=c["cf"])
+
+
+def test_bf16_tensor_core_path_is_bit_exact_run_to_run():
+    # 20 row tiles x (8 + 4 + ...) column tiles per launch: several tiles per CTA pair, drawn in a different
+    # order every run
+    inp = synth.moe_inputs(2500, 1024, 2048, 4, 5, torch.bfloat16, DEV)
+    outs = []
+    for _ in range(3):
+        fwd = gpu_forward(inp, 2)
+        got = gpu_backward(inp, fwd)
+        outs.append((fwd["y"].clone(), {n: t.clone() for n, t in got.items() if t is not None}))
+    for y, g in outs[1:]:
+        assert torch.equal(y, outs[0][0])
+        for n, t in g.items():
+            assert torch.equal(t, outs[0][1][n]), n
