@@ -46,11 +46,14 @@ struct SwapParams {
 struct DTile { int which, chunk, mt, e, kb0, kb1, s; };
 
 __device__ __forceinline__ DTile d_tile(const SwapParams& p, const int* chunks, int n_valid, int t) {
+  // The token chunk varies fastest: an expert that holds more than one chunk of tokens has the items
+  // that read the same weight tile next to one another, so the tile comes from HBM once and from L2
+  // for the other chunks.
   DTile tl;
+  const int ci = t % n_valid; t /= n_valid;
   tl.s = t % p.S; t /= p.S;
-  tl.mt = t % p.m_tiles; t /= p.m_tiles;
-  const int ci = t % n_valid;
-  tl.which = t / n_valid;
+  tl.mt = t % p.m_tiles;
+  tl.which = t / p.m_tiles;
   tl.chunk = chunks[ci];
   tl.e = p.tile_expert[(tl.chunk * TOK) / kRowTile];
   tl.kb0 = (int)((long long)tl.s * p.kb_total / p.S);
