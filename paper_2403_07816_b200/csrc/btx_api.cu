@@ -50,7 +50,7 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   // The weight-streaming expert kernels pay off while an expert holds about one 64-token chunk; beyond
   // that the 256-row tiles of the training-shaped kernels use the tensor cores better (measured at the
   // Llama-2-7B shape, E = 4: equal at R = 256, 25 to 40 % slower at R = 512 and 1024).
-  p.small = !routing_only && desc->dtype == BTX_BF16 && route_permute_small_fits(p) && p.R <= 64 * p.E;
+  p.small = !routing_only && desc->dtype == BTX_BF16 && route_permute_small_fits(p);
   if (p.small) {
     const int chunks = p.E < p.R ? p.E : p.R;             // typical: every expert holds one token chunk
     p.dec_s1 = pick_decode_splits(2 * chunks * ((p.F + 255) / 256), (p.d + 63) / 64);

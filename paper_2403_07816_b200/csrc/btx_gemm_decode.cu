@@ -2,8 +2,9 @@
 //
 // With a few tokens per expert the layer is bound by reading the expert weights once from HBM.
 // The weights therefore take the M side of the tensor-core tile (256 weight rows per CTA pair,
-// tcgen05.mma.cta_group::2) and a narrow chunk of 64 token rows takes the N side, so an MMA costs
-// 32 cycles instead of 128 and the tensor pipe never limits the stream.  The contraction is split
+// tcgen05.mma.cta_group::2) and the tokens of one padded 256-row tile of an expert take the N side,
+// N = the tile's real rows rounded up to 16: with 16 tokens an MMA costs 8 cycles instead of 128, so
+// the tensor pipe does not limit the stream, and nothing is spent on padding rows.  The contraction is split
 // into S parts per tile so that the number of work items is a multiple of the CTA pairs; every
 // item writes its fp32 partial product for the valid tokens only, addressed [split][t*k+slot][row]:
 // a lane owns a weight row, so the 32 lanes of a warp write one 128-byte line per token.
@@ -12,7 +13,7 @@
 //   pass 2   partial gate * W2_e a             -> combine kernel sums parts and slots into y
 //
 // Same warp roles, barriers and bounded waits as the training-shaped kernel: warp 0 TMA producer
-// (9 stages of 128x64 weights + 32x64 tokens per CTA), warp 1 MMA issuer in the leader CTA,
+// (128x64 weights + 32, 64 or 128 x 64 tokens per CTA and stage; 9, 8 or 6 stages), warp 1 MMA issuer in the leader CTA,
 // warps 2-9 epilogue.
 #include "btx_tc_ptx.cuh"
 
@@ -22,19 +23,23 @@ namespace {
 using namespace tcx;
 
 constexpr int WM = 128;                                  // weight rows per CTA (256 per pair)
-constexpr int TOK = 64;                                  // token rows per chunk (MMA N)
-constexpr int D_STAGES = 9;
-constexpr int DA_BYTES = WM * BK * 2, DB_BYTES = (TOK / 2) * BK * 2, D_STAGE_BYTES = DA_BYTES + DB_BYTES;
+constexpr int CH = kRowTile;                             // a chunk is one padded row tile of an expert (MMA N <= 256)
+constexpr int D_MAX_STAGES = 9;
+constexpr int DA_BYTES = WM * BK * 2;                    // weights per CTA and stage
+constexpr int D_RING_BYTES = 192 * 1024;                 // stages = min(9, ring / (DA_BYTES + token box))
 constexpr int D_EPI_WARPS = 8;
 constexpr int D_THREADS = 64 + D_EPI_WARPS * 32;
-constexpr int D_MAX_CHUNKS = 192;                        // (1024 + 32 * 255) / 64 rounded up
-constexpr int D_SMEM_BYTES = D_STAGES * D_STAGE_BYTES + 1024 + 256 + (D_MAX_CHUNKS + 2) * 4;
+constexpr int D_MAX_CHUNKS = 64;                         // (1024 + 32 * 255) / 256 rounded up, with room
+constexpr int D_SMEM_BYTES = D_RING_BYTES + 1024 + 256 + (D_MAX_CHUNKS + 2) * 4;
 
 struct SwapParams {
   int W;                        // weight rows per expert (F in pass 1, d in pass 2)
   int E, S, n_w, m_tiles, kb_total;
+  int box_rows;                 // token rows each CTA loads per stage (32, 64 or 128): >= N/2 of every chunk
+  int stages;                   // ring depth for that box
   const int32_t* pad_offsets;
   const int32_t* tile_expert;
+  const int32_t* counts;        // rows per expert
   const int32_t* rowmap;
   const float* gates;           // non-null: scale every token column by its gate
   float* out0;                  // [S][R][W]
@@ -43,7 +48,7 @@ struct SwapParams {
   int32_t* status;
 };
 
-struct DTile { int which, chunk, mt, e, kb0, kb1, s; };
+struct DTile { int which, chunk, n, mt, e, kb0, kb1, s; };   // n = MMA N of the chunk (multiple of 16)
 
 __device__ __forceinline__ DTile d_tile(const SwapParams& p, const int* chunks, int n_valid, int t) {
   // The token chunk varies fastest: an expert that holds more than one chunk of tokens has the items
@@ -54,8 +59,9 @@ __device__ __forceinline__ DTile d_tile(const SwapParams& p, const int* chunks, 
   tl.s = t % p.S; t /= p.S;
   tl.mt = t % p.m_tiles;
   tl.which = t / p.m_tiles;
-  tl.chunk = chunks[ci];
-  tl.e = p.tile_expert[(tl.chunk * TOK) / kRowTile];
+  tl.chunk = chunks[ci] & 0xFFFF;
+  tl.n = chunks[ci] >> 16;
+  tl.e = p.tile_expert[tl.chunk];
   tl.kb0 = (int)((long long)tl.s * p.kb_total / p.S);
   tl.kb1 = (int)((long long)(tl.s + 1) * p.kb_total / p.S);
   return tl;
@@ -67,14 +73,16 @@ tc_swapk_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t ring = (raw + 1023u) & ~1023u;
-  uint8_t* ctl = smem_raw + (ring - raw) + D_STAGES * D_STAGE_BYTES;
+  uint8_t* ctl = smem_raw + (ring - raw) + D_RING_BYTES;
   const uint32_t bar_full = smem_u32(ctl);
-  const uint32_t bar_empty = bar_full + D_STAGES * 8;
-  const uint32_t bar_tfull = bar_empty + D_STAGES * 8;
+  const uint32_t bar_empty = bar_full + D_MAX_STAGES * 8;
+  const uint32_t bar_tfull = bar_empty + D_MAX_STAGES * 8;
   const uint32_t bar_tempty = bar_tfull + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + D_STAGES * 16 + 32);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + D_STAGES * 16 + 40);
-  int* chunks = reinterpret_cast<int*>(ctl + 256);        // [0] = count, [1..] = chunk ids that hold tokens
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + D_MAX_STAGES * 16 + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + D_MAX_STAGES * 16 + 40);
+  int* chunks = reinterpret_cast<int*>(ctl + 256);        // [0] = count, [1..] = chunk id | N << 16 of the chunks with tokens
+  const int n_stages = p.stages;
+  const uint32_t stage_bytes = DA_BYTES + (uint32_t)p.box_rows * (BK * 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -82,7 +90,7 @@ tc_swapk_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
   allow_dependents();
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < D_STAGES; ++s) { mbar_init(bar_full + s * 8, 1); mbar_init(bar_empty + s * 8, 1); }
+    for (int s = 0; s < D_MAX_STAGES; ++s) { mbar_init(bar_full + s * 8, 1); mbar_init(bar_empty + s * 8, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + a * 8, 1); mbar_init(bar_tempty + a * 8, 2 * D_EPI_WARPS * 32); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -92,18 +100,23 @@ tc_swapk_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
   // reads what it wrote.
   grid_dependency_wait();
   if (warp == 0) {
-    // List of the chunks that hold tokens (expert segments start with their real rows, so a chunk
-    // holds tokens iff its first row does).  The 32 lanes probe 32 chunks at a time: one round of
-    // global-memory latency instead of one per chunk, which used to dominate the kernel's start.
+    // List of the chunks (row tiles) that hold tokens, each with its MMA N: an expert's segment starts
+    // with its real rows, so tile j of expert e holds min(256, counts[e] - 256 j) of them.  The 32
+    // lanes probe 32 tiles at a time: one round of global-memory latency, not one per tile.
     __syncwarp();
-    const int all = p.pad_offsets[p.E] / TOK;
+    const int all = p.pad_offsets[p.E] / CH;
     int n = 0;
     for (int c0 = 0; c0 < all; c0 += 32) {
       const int c = c0 + lane;
-      const bool holds = c < all && p.rowmap[c * TOK] >= 0;
+      int rows = 0;
+      if (c < all) {
+        const int e = p.tile_expert[c];
+        if (e >= 0) rows = min(CH, p.counts[e] - (c * CH - p.pad_offsets[e]));
+      }
+      const bool holds = rows > 0;
       const unsigned m = __ballot_sync(0xffffffffu, holds);
       const int pos = n + __popc(m & ((1u << lane) - 1u));
-      if (holds && pos < D_MAX_CHUNKS) chunks[1 + pos] = c;
+      if (holds && pos < D_MAX_CHUNKS) chunks[1 + pos] = c | (((rows + 15) & ~15) << 16);
       n += __popc(m);
     }
     if (lane == 0) chunks[0] = min(n, D_MAX_CHUNKS);
@@ -130,22 +143,22 @@ tc_swapk_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
           if (!(ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status))) break;
           const uint32_t full_local = bar_full + stage * 8;
           const uint32_t full = map_to_cta(full_local, 0);
-          const uint32_t sA = ring + stage * D_STAGE_BYTES, sB = sA + DA_BYTES;
-          if (rank == 0) mbar_expect_tx(full_local, 2 * D_STAGE_BYTES);
+          const uint32_t sA = ring + stage * stage_bytes, sB = sA + DA_BYTES;
+          if (rank == 0) mbar_expect_tx(full_local, 2 * stage_bytes);
           tma_load_3d(sA, tl.which ? &tmW1 : &tmW0, kb * BK, tl.mt * 2 * WM + (int)rank * WM, tl.e, full);
-          tma_load_2d(sB, &tmX, kb * BK, tl.chunk * TOK + (int)rank * (TOK / 2), full);
-          if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+          // this CTA's half of the chunk's N token rows leads its box; rows past it are not used
+          tma_load_2d(sB, &tmX, kb * BK, tl.chunk * CH + (int)rank * (tl.n / 2), full);
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
         }
       }
-      for (int i = 0; i < D_STAGES && ok; ++i) {          // drain: all commits to this CTA have landed
+      for (int i = 0; i < n_stages && ok; ++i) {          // drain: all commits to this CTA have landed
         ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status);
-        if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+        if (++stage == n_stages) { stage = 0; phase ^= 1u; }
       }
     }
   } else if (warp == 1) {
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TOK >> 3) << 17) |
-                                 ((uint32_t)((2 * WM) >> 4) << 24);
+      constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * WM) >> 4) << 24);
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
       for (int t = pair; t < n_total && ok; t += n_pairs) {
@@ -154,17 +167,18 @@ tc_swapk_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
         if (!(ok = mbar_wait(bar_tempty + acc * 8, acc_phase ^ 1u, abort_flag, p.status))) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * 256;
+        const uint32_t idesc = idesc_base | ((uint32_t)(tl.n >> 3) << 17);
         for (int kb = tl.kb0; kb < tl.kb1; ++kb) {
           if (!(ok = mbar_wait(bar_full + stage * 8, phase, abort_flag, p.status))) break;
           tc_fence_after();
-          const uint32_t sA = ring + stage * D_STAGE_BYTES, sB = sA + DA_BYTES;
+          const uint32_t sA = ring + stage * stage_bytes, sB = sA + DA_BYTES;
           const uint64_t da = smem_desc(sA, false), db = smem_desc(sB, false);
 #pragma unroll
           for (int k16 = 0; k16 < BK / 16; ++k16)
             tc_mma_pair(tmem_d, da + (uint64_t)(2 * k16), db + (uint64_t)(2 * k16), idesc,
                         (kb > tl.kb0 || k16 > 0) ? 1u : 0u);
           tc_commit_pair(bar_empty + stage * 8);
-          if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         tc_commit_pair(bar_tfull + acc * 8);
@@ -180,25 +194,28 @@ tc_swapk_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
     for (int t = pair; t < n_total && ok; t += n_pairs) {
       const DTile tl = d_tile(p, chunks + 1, n_valid, t);
       if (tl.kb1 <= tl.kb0) continue;
-      // token of this lane's column: lane i of the warp looks up column half*32 + i
-      const int my_flat = p.rowmap[tl.chunk * TOK + half * 32 + lane];
-      const float my_gate = (p.gates != nullptr && my_flat >= 0) ? p.gates[my_flat] : 1.0f;
       if (!(ok = mbar_wait(bar_tfull + acc * 8, acc_phase, abort_flag, p.status))) break;
       tc_fence_after();
-      float v[32];
-      tc_ld32(tmem_base + acc * 256 + half * 32 + ((uint32_t)(q * 32) << 16), v);
+      const int wrow = tl.mt * 2 * WM + (int)rank * WM + q * 32 + lane;
+      float* out = (tl.which ? p.out1 : p.out0) + (size_t)tl.s * p.split_stride + wrow;
+      // the two warps of a lane quarter take alternate groups of 32 token columns
+      for (int c0 = half * 32; c0 < tl.n; c0 += 64) {
+        // token of this lane's column: lane i of the warp looks up column c0 + i
+        const int my_flat = p.rowmap[tl.chunk * CH + c0 + lane];
+        const float my_gate = (p.gates != nullptr && my_flat >= 0) ? p.gates[my_flat] : 1.0f;
+        float v[32];
+        tc_ld32(tmem_base + acc * 256 + c0 + ((uint32_t)(q * 32) << 16), v);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int flat = __shfl_sync(0xffffffffu, my_flat, i);
+          const float g = __shfl_sync(0xffffffffu, my_gate, i);
+          if (flat >= 0 && wrow < p.W) out[(size_t)flat * p.W] = g * v[i];
+        }
+      }
       tc_fence_before();
       mbar_arrive_cluster(tempty_leader + acc * 8);
       acc ^= 1u;
       if (acc == 0) acc_phase ^= 1u;
-      const int wrow = tl.mt * 2 * WM + (int)rank * WM + q * 32 + lane;
-      float* out = (tl.which ? p.out1 : p.out0) + (size_t)tl.s * p.split_stride + wrow;
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const int flat = __shfl_sync(0xffffffffu, my_flat, i);
-        const float g = __shfl_sync(0xffffffffu, my_gate, i);
-        if (flat >= 0 && wrow < p.W) out[(size_t)flat * p.W] = g * v[i];
-      }
     }
   }
 
@@ -279,13 +296,19 @@ btx_status launch_expert_forward_small_bf16(const Plan& pl, const void* w1, cons
   btx_status s;
   SwapParams p = {};
   p.E = pl.E; p.pad_offsets = b.pad_offsets; p.tile_expert = b.tile_expert; p.rowmap = b.rowmap; p.status = b.status;
+  p.counts = b.counts;
+  // a chunk holds at most min(T, 256) tokens (a token meets an expert once): each CTA loads half of them
+  const int n_max = ((pl.T < CH ? pl.T : CH) + 15) & ~15;
+  p.box_rows = n_max / 2 <= 32 ? 32 : (n_max / 2 <= 64 ? 64 : 128);
+  p.stages = D_RING_BYTES / (DA_BYTES + p.box_rows * BK * 2);
+  if (p.stages > D_MAX_STAGES) p.stages = D_MAX_STAGES;
   if (save) {   // backward reads whole padded tiles of h1/h3: rows without a token must be finite
     if (cudaMemsetAsync(b.h1, 0, (size_t)RP * F * 2, st) != cudaSuccess ||
         cudaMemsetAsync(b.h3, 0, (size_t)RP * F * 2, st) != cudaSuccess)
       return BTX_ERR_CUDA;
   }
   // pass 1: partial h1, h3
-  if (!make_map(&m0, w1, d, F, E, 64, WM) || !make_map(&m1, w3, d, F, E, 64, WM) || !make_map(&mx, b.xs, d, RP, 0, 64, TOK / 2))
+  if (!make_map(&m0, w1, d, F, E, 64, WM) || !make_map(&m1, w3, d, F, E, 64, WM) || !make_map(&mx, b.xs, d, RP, 0, 64, p.box_rows))
     return BTX_ERR_CUDA;
   p.W = pl.F; p.n_w = 2; p.m_tiles = (pl.F + 2 * WM - 1) / (2 * WM); p.kb_total = (pl.d + BK - 1) / BK; p.S = pl.dec_s1;
   p.split_stride = (size_t)pl.R * pl.F;
@@ -299,7 +322,7 @@ btx_status launch_expert_forward_small_bf16(const Plan& pl, const void* w1, cons
     return BTX_ERR_CUDA;
   mark_stage(2, st);
   // pass 2: partial gate-scaled expert rows
-  if (!make_map(&m0, w2, F, d, E, 64, WM) || !make_map(&mx, b.act, F, RP, 0, 64, TOK / 2)) return BTX_ERR_CUDA;
+  if (!make_map(&m0, w2, F, d, E, 64, WM) || !make_map(&mx, b.act, F, RP, 0, 64, p.box_rows)) return BTX_ERR_CUDA;
   p.W = pl.d; p.n_w = 1; p.m_tiles = (pl.d + 2 * WM - 1) / (2 * WM); p.kb_total = (pl.F + BK - 1) / BK; p.S = pl.dec_s2;
   p.split_stride = (size_t)pl.R * pl.d;
   p.out0 = b.part; p.out1 = b.part; p.gates = b.gates;
