@@ -47,9 +47,9 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   if (p.route_blocks > 148 * 8) p.route_blocks = 148 * 8;
   p.perm_blocks = (p.R + 1023) / 1024;
   p.wr_chunks = (p.T + 127) / 128;
-  // The weight-streaming expert kernels pay off while an expert holds about one 64-token chunk; beyond
-  // that the 256-row tiles of the training-shaped kernels use the tensor cores better (measured at the
-  // Llama-2-7B shape, E = 4: equal at R = 256, 25 to 40 % slower at R = 512 and 1024).
+  // Small BF16 batches stream the expert weights through the swap-AB kernels (weights on the M side,
+  // an expert's tokens on the N side); measured at the Llama-2-7B shape with E = 4 they beat the
+  // training-shaped kernels up to the routing kernel's limit of 1024 assignments.
   p.small = !routing_only && desc->dtype == BTX_BF16 && route_permute_small_fits(p);
   if (p.small) {
     const int chunks = p.E < p.R ? p.E : p.R;             // typical: every expert holds one token chunk
