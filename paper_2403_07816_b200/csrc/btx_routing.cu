@@ -109,7 +109,7 @@ __device__ __forceinline__ void route_token(int t, int d, int E, int k, int rout
       float acc[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-#pragma unroll 4
+#pragma unroll 2
       for (int c = lane * VN; c < d; c += 32 * VN) {
         float xv[VN];
         Vec<T>::load(xr + c, xv);
@@ -142,7 +142,7 @@ __device__ __forceinline__ void route_token(int t, int d, int E, int k, int rout
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kRouterThreads)
+__global__ void __launch_bounds__(kRouterThreads, 4)      // at most 64 registers: the x stream needs the occupancy
 router_kernel(int Tn, int d, int E, int k, int routing, const T* __restrict__ x, const T* __restrict__ wr,
               const float* __restrict__ bias, const float* __restrict__ given_logits,
               const float* __restrict__ noise, float inv_tau,
@@ -523,11 +523,23 @@ combine_kernel(int Tn, int d, int k, int E, int splits, const float* __restrict_
 // ---------------------------------------------------------------------------------------------
 // Router backward
 // ---------------------------------------------------------------------------------------------
-// One thread per token: d gate of every slot (row-dot partials of the dgrad-2 epilogue summed in
-// tile order, plus the u-term of L_LB), then the softmax Jacobians and the p-term of L_LB.
+// Row-dot partials of the dgrad-2 epilogue, [column tile][padded row]: summed over the column tiles in
+// tile order, one thread per padded row (consecutive rows, so every load is coalesced), into tile 0.
 __global__ void __launch_bounds__(256)
-router_dz_kernel(int Tn, int E, int k, int routing, float alpha, float lb_scale, int stopgrad_u, int nt_dact,
-                 int r_pad_max, const int32_t* __restrict__ topk, const float* __restrict__ gates,
+dg_rowsum_kernel(int nt, int r_pad_max, int E, const int32_t* __restrict__ pad_offsets, float* __restrict__ dg_part) {
+  const int rp = blockIdx.x * blockDim.x + threadIdx.x;
+  if (rp >= pad_offsets[E]) return;
+  float a = 0.f;
+#pragma unroll 8
+  for (int n = 0; n < nt; ++n) a += dg_part[(size_t)n * r_pad_max + rp];
+  dg_part[rp] = a;
+}
+
+// One thread per token: d gate of every slot (the summed row-dot of its row plus the u-term of L_LB),
+// then the softmax Jacobians and the p-term of L_LB.
+__global__ void __launch_bounds__(64)
+router_dz_kernel(int Tn, int E, int k, int routing, float alpha, float lb_scale, int stopgrad_u,
+                 const int32_t* __restrict__ topk, const float* __restrict__ gates,
                  const float* __restrict__ probs, const float* __restrict__ u, const float* __restrict__ p,
                  const int32_t* __restrict__ flat2row, const float* __restrict__ dg_part, float dz_scale,
                  float* __restrict__ dz_out, float* __restrict__ dz_out2) {
@@ -541,8 +553,7 @@ router_dz_kernel(int Tn, int E, int k, int routing, float alpha, float lb_scale,
     float a = 0.f;
     if (dg_part != nullptr) {
       int rp = flat2row[(size_t)t * k + s];
-      if (rp >= 0)                                   // a dropped assignment has no path into y
-        for (int n = 0; n < nt_dact; ++n) a += dg_part[(size_t)n * r_pad_max + rp];
+      if (rp >= 0) a = dg_part[rp];                  // a dropped assignment has no path into y
     }
     if (!stopgrad_u) a += lbc * p[topk[(size_t)t * k + s]];
     dg[s] = a;
@@ -569,43 +580,51 @@ router_dz_kernel(int Tn, int E, int k, int routing, float alpha, float lb_scale,
 
 constexpr int kWrTokens = 128;   // tokens per chunk of the router-weight gradient
 
-// partial[chunk][e][c] = sum over the chunk's tokens of dz[t,e] * x[t,c]; each thread owns 2 columns.
+// partial[chunk][e][c] = sum over the chunk's tokens of dz[t,e] * x[t,c]; each thread owns one 16-byte
+// vector of columns (8 in BF16, 4 in FP32) and four experts at a time.
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 router_dw_partial_kernel(int Tn, int d, int E, const T* __restrict__ x, const float* __restrict__ dz,
                          float* __restrict__ part, float* __restrict__ bias_part) {
+  constexpr int VN = Vec<T>::N;
   __shared__ float sdz[kWrTokens * kMaxExperts];
   const int chunk = blockIdx.x;
   const int t0 = chunk * kWrTokens, t1 = min(Tn, t0 + kWrTokens);
   for (int i = threadIdx.x; i < (t1 - t0) * E; i += blockDim.x) sdz[i] = dz[(size_t)t0 * E + i];
   __syncthreads();
-  const int c = (blockIdx.y * blockDim.x + threadIdx.x) * 2;
+  const int c = (blockIdx.y * blockDim.x + threadIdx.x) * VN;
   if (blockIdx.y == 0 && threadIdx.x < E) {
     float s = 0.f;
     for (int t = 0; t < t1 - t0; ++t) s += sdz[t * E + threadIdx.x];
     bias_part[(size_t)chunk * E + threadIdx.x] = s;
   }
   if (c >= d) return;
-  for (int eb = 0; eb < E; eb += 8) {
-    float acc[8][2];
+  for (int eb = 0; eb < E; eb += 4) {
+    float acc[4][VN];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j][0] = acc[j][1] = 0.f;
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int v = 0; v < VN; ++v) acc[j][v] = 0.f;
+#pragma unroll 4
     for (int t = t0; t < t1; ++t) {
-      float x0 = to_f32(x[(size_t)t * d + c]), x1 = to_f32(x[(size_t)t * d + c + 1]);
+      float xv[VN];
+      Vec<T>::load(x + (size_t)t * d + c, xv);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < 4; ++j) {
         if (eb + j < E) {
-          float g = sdz[(t - t0) * E + eb + j];
-          acc[j][0] = fmaf(g, x0, acc[j][0]);
-          acc[j][1] = fmaf(g, x1, acc[j][1]);
+          const float g = sdz[(t - t0) * E + eb + j];
+#pragma unroll
+          for (int v = 0; v < VN; ++v) acc[j][v] = fmaf(g, xv[v], acc[j][v]);
         }
       }
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < 4; ++j) {
       if (eb + j < E) {
         float* o = part + ((size_t)chunk * E + eb + j) * d + c;
-        o[0] = acc[j][0]; o[1] = acc[j][1];
+#pragma unroll
+        for (int v = 0; v < VN; v += 4)
+          *reinterpret_cast<float4*>(o + v) = make_float4(acc[j][v], acc[j][v + 1], acc[j][v + 2], acc[j][v + 3]);
       }
     }
   }
@@ -709,22 +728,25 @@ cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float
                                    int stopgrad_u, int have_dg, const void* x, const void* w_router, const Buffers& b,
                                    void* dx, float* dw_router, float* dbias, float* dlogits_out, int accumulate,
                                    float dz_scale, cudaStream_t st) {
-  router_dz_kernel<<<(pl.T + 255) / 256, 256, 0, st>>>(pl.T, pl.E, pl.k, routing, alpha, lb_scale, stopgrad_u,
-                                                       pl.nt_dact, pl.r_pad_max, b.topk, b.gates, b.probs, b.u, b.p,
-                                                       b.flat2row, have_dg ? b.dg_part : nullptr, dz_scale, b.dz, dlogits_out);
+  if (have_dg)
+    dg_rowsum_kernel<<<(pl.r_pad_max + 255) / 256, 256, 0, st>>>(pl.nt_dact, pl.r_pad_max, pl.E, b.pad_offsets, b.dg_part);
+  router_dz_kernel<<<(pl.T + 63) / 64, 64, 0, st>>>(pl.T, pl.E, pl.k, routing, alpha, lb_scale, stopgrad_u, b.topk,
+                                                    b.gates, b.probs, b.u, b.p, b.flat2row,
+                                                    have_dg ? b.dg_part : nullptr, dz_scale, b.dz, dlogits_out);
   if (x == nullptr) return cudaGetLastError();     // loss-only gradient (btx_lb_loss)
-  dim3 grid(pl.wr_chunks, (pl.d / 2 + 255) / 256);
+  const int vn = dtype == BTX_BF16 ? 8 : 4;
+  dim3 grid(pl.wr_chunks, (pl.d / vn + 127) / 128);
   float* bias_part = b.dwr_part + (size_t)pl.wr_chunks * pl.E * pl.d;
   size_t n = (size_t)pl.T * (pl.d / 4);
   int cblocks = (int)min((n + 255) / 256, (size_t)148 * 32);
   const int32_t* kept = pl.capped ? b.flat2row : nullptr;
   if (dtype == BTX_BF16) {
-    router_dw_partial_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(pl.T, pl.d, pl.E, (const __nv_bfloat16*)x, b.dz,
+    router_dw_partial_kernel<__nv_bfloat16><<<grid, 128, 0, st>>>(pl.T, pl.d, pl.E, (const __nv_bfloat16*)x, b.dz,
                                                                   b.dwr_part, bias_part);
     combine_kernel<__nv_bfloat16><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, 1, b.dxp, b.dz,
                                                            (const __nv_bfloat16*)w_router, kept, (__nv_bfloat16*)dx);
   } else {
-    router_dw_partial_kernel<float><<<grid, 256, 0, st>>>(pl.T, pl.d, pl.E, (const float*)x, b.dz, b.dwr_part,
+    router_dw_partial_kernel<float><<<grid, 128, 0, st>>>(pl.T, pl.d, pl.E, (const float*)x, b.dz, b.dwr_part,
                                                           bias_part);
     combine_kernel<float><<<cblocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, 1, b.dxp, b.dz, (const float*)w_router,
                                                    kept, (float*)dx);
