@@ -279,7 +279,7 @@ def run_moe(args, workload):
     R = T * k
     flops_step = (18 if train else 6) * R * d * F * layers
     fwd_launches = 6 if T * k <= 1024 else 9        # small batches: routing+permutation in one launch, two passes + fix-up
-    launches_per_step = (fwd_launches + (10 if train else 0)) * layers
+    launches_per_step = (fwd_launches + (11 if train else 0)) * layers
     line = {
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "clocks": clocks,
