@@ -511,12 +511,17 @@ def round_to_storage(v, dtype):
     raise ValueError(dtype)
 
 
-def merge_average(sources, dtype):
-    """Uniform mean over the N models in float64, rounded once to the storage type."""
+def merge_mean(sources):
+    """Uniform mean over the N models in float64, unrounded."""
     acc = np.zeros_like(_f64(sources[0]))
     for s in sources:
         acc = acc + _f64(s)
-    return round_to_storage(acc / len(sources), dtype)
+    return acc / len(sources)
+
+
+def merge_average(sources, dtype):
+    """Uniform mean over the N models in float64, rounded once to the storage type."""
+    return round_to_storage(merge_mean(sources), dtype)
 
 
 def merge_stack(sources):

@@ -91,7 +91,7 @@ def test_forward_T4096_seed1():
 
 
 def test_forward_backward_T16384_seed2():
-    counts = full_size_case(16384, 2, seed=2)
+    counts = full_size_case(16384, 2, seed=2, n_tok=256, n_hidden=64)
     assert counts.min() > 0.2 * 32768 and counts.max() < 0.3 * 32768      # roughly uniform loads
 
 
@@ -141,3 +141,42 @@ def test_decode_shaped_T32_two_layers_seed4():
         assert np.array_equal(fwd["routing"].topk_idx.cpu().numpy(), ref["topk_idx"])
         assert np.array_equal(fwd["routing"].perm.cpu().numpy(), ref["perm"])
         assert rel_err(np64(fwd["y"]), ref["y"]) <= TOL
+
+
+def test_merge_llama2_7b_shaped_tensors_seed4():
+    """MiX merge at the sizes of the Llama-2-7B shape (Section 3.2): two layers plus embeddings, head and final
+    norm of four BF16 parameter sets (5.4 GB read).  Averaged tensors against the fp64 mean rounded once;
+    stacked feed-forward slots bit for bit, compared on the device."""
+    models = synth.expert_models(4, 2, D, F, 32000, seed=4, dtype=torch.bfloat16, device=DEV)
+    out = {}
+    for n, t in models[0].items():
+        out[n] = torch.empty(((4,) + tuple(t.shape)) if ".ffn." in n else tuple(t.shape), dtype=torch.bfloat16, device=DEV)
+    B.btx_merge(models, out)
+    torch.cuda.synchronize()
+    for n in out:
+        if ".ffn." in n:
+            for m in range(4):
+                assert torch.equal(out[n][m], models[m][n]), (n, m)
+            continue
+        if out[n].numel() > (1 << 24):
+            # the two [32000, 4096] tensors: 2048 sampled rows through the oracle, and on the device every
+            # element between the smallest and the largest of its four sources
+            rows = torch.from_numpy(np.sort(np.random.default_rng(4).choice(out[n].shape[0], 2048, replace=False))).to(DEV)
+            stack = torch.stack([m[n] for m in models]).float()
+            assert bool(((out[n].float() >= stack.amin(0)) & (out[n].float() <= stack.amax(0))).all()), n
+            del stack
+            srcs = [np64(m[n][rows]) for m in models]
+            got = np64(out[n][rows])
+        else:
+            srcs = [np64(m[n]) for m in models]
+            got = np64(out[n])
+        mean = o.merge_mean(srcs)
+        # The kernel sums in fp32 in model order (three roundings of at most 2^-24 of a partial sum) and rounds
+        # once to bf16: the result lies within half a bf16 ulp of the exact mean's binade plus that fp32 error.
+        # (Where the exact mean sits that close to a rounding boundary the stored value may be the other
+        # neighbour, one ulp from the oracle's rounding; both are within the bound.)
+        mean_abs = sum(np.abs(a) for a in srcs) / 4
+        half_ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(mean), 2.0 ** -126))) - 8.0)
+        assert np.all(np.abs(got - mean) <= half_ulp * (1 + 1e-9) + 3 * 2.0 ** -24 * mean_abs), n
+        assert np.mean(got != o.merge_average(srcs, "bf16")) < 1e-3, n
+        del srcs, mean, got
