@@ -206,6 +206,14 @@ btx_status btx_merge_ffn(int32_t n_models, int32_t dtype, int32_t layout, int32_
  * `workspace`: *device_status (host) is BTX_OK or BTX_ERR_TIMEOUT. */
 btx_status btx_device_status(const void* workspace, void* stream, int32_t* device_status);
 
+/* Self-test of the bounded device-side waits (the paper has no counterpart).  Clears the status block at
+ * the start of `workspace` (at least 256 bytes) and runs a kernel in which one thread waits, with a 50 ms
+ * limit, on a barrier nobody arrives at: the wait gives up, records BTX_ERR_TIMEOUT in the status word and
+ * the kernel returns normally, which is what every wait of the tensor-core kernels does (after about two
+ * seconds) if a copy or a partner CTA never signals.  btx_device_status then reports BTX_ERR_TIMEOUT; the
+ * CUDA context stays usable and the next call that uses the workspace clears the word again. */
+btx_status btx_selftest_wait_expiry(void* workspace, size_t workspace_bytes, void* stream);
+
 /* Optional stage timing for the calling host thread.  `events` is a host array of n
  * cudaEvent_t (as void*), or NULL to switch the hook off.  While set, btx_moe_forward records
  * events[0..4] on its stream: start, after routing+permutation+gather, after GEMM-1 (W1/W3 +

@@ -13,6 +13,7 @@ from dataclasses import dataclass
 import torch
 
 BTX_OK = 0
+BTX_ERR_INVALID_ARG, BTX_ERR_UNSUPPORTED, BTX_ERR_WORKSPACE, BTX_ERR_ARCH, BTX_ERR_CUDA, BTX_ERR_TIMEOUT = 1, 2, 3, 4, 5, 6
 BTX_F32, BTX_BF16 = 0, 1
 ROUTE_TOPK, ROUTE_SWITCH, ROUTE_SOFT, ROUTE_SAMPLE1 = 0, 1, 2, 3
 PARAM_AVERAGE, PARAM_FFN = 0, 1
@@ -48,7 +49,7 @@ class MergeItem(C.Structure):
 
 EXPORTS = ["btx_moe_sizes", "btx_moe_forward", "btx_moe_backward", "btx_moe_step_host",
            "btx_lb_loss_workspace_size", "btx_lb_loss", "btx_lb_loss_noalloc", "btx_merge_workspace_size", "btx_merge", "btx_merge_ffn_workspace_size", "btx_merge_ffn",
-           "btx_device_status", "btx_set_stage_events", "btx_status_string", "btx_version"]
+           "btx_device_status", "btx_selftest_wait_expiry", "btx_set_stage_events", "btx_status_string", "btx_version"]
 
 
 def lib():
@@ -65,6 +66,7 @@ def lib():
                                        vp, i32, vp, sz, vp]
         L.btx_moe_step_host.argtypes = [C.POINTER(MoeDesc)] + [vp] * 15 + [f32] + [vp] * 5 + [i32, vp, vp, sz, vp, vp]
         L.btx_set_stage_events.argtypes = [C.POINTER(vp), i32]
+        L.btx_selftest_wait_expiry.argtypes = [vp, sz, vp]
         L.btx_lb_loss_workspace_size.argtypes = [C.POINTER(MoeDesc), C.POINTER(sz)]
         L.btx_lb_loss.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, sz, vp]
         L.btx_lb_loss_noalloc.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp]
@@ -295,6 +297,14 @@ def btx_merge_ffn(w1s, w3s, w2s, layout, chunks, w1_dst, w3_dst, w2_dst, workspa
     if s != BTX_OK:
         raise BtxError(s, "btx_merge_ffn")
     return workspace
+
+
+def btx_selftest_wait_expiry(workspace):
+    """Makes one bounded device-side wait run out on purpose; see btx.h."""
+    s = lib().btx_selftest_wait_expiry(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                       _stream(workspace.device))
+    if s != BTX_OK:
+        raise BtxError(s, "btx_selftest_wait_expiry")
 
 
 def btx_device_status(workspace):

@@ -422,6 +422,17 @@ extern "C" btx_status btx_device_status(const void* workspace, void* stream, int
   return BTX_OK;
 }
 
+extern "C" btx_status btx_selftest_wait_expiry(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace || misaligned(workspace)) return BTX_ERR_INVALID_ARG;
+  if (workspace_bytes < (size_t)kStatusWords * 4) return BTX_ERR_WORKSPACE;
+  btx_status s = check_device();
+  if (s != BTX_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  BTX_CUDA_OK(cudaMemsetAsync(workspace, 0, kStatusWords * 4, st));
+  BTX_CUDA_OK(launch_wait_expiry_selftest((int32_t*)workspace, st));
+  return BTX_OK;
+}
+
 extern "C" const char* btx_status_string(btx_status s) {
   switch (s) {
     case BTX_OK: return "ok";

@@ -70,6 +70,7 @@ cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, c
                           const float* bias, const float* given_logits, const float* noise, float inv_tau,
                           const Buffers& b, cudaStream_t st);
 cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st);
+cudaError_t launch_wait_expiry_selftest(int32_t* status, cudaStream_t st);
 // Router + loss + permutation in one single-block launch, for batches with T*k <= 1024.
 bool route_permute_small_fits(const Plan& pl);
 cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, float alpha, const void* x,

@@ -471,6 +471,19 @@ btx_status launch_tc(const CUtensorMap& a0, const CUtensorMap& a1, const CUtenso
   return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
 }
 
+// One thread waits, with a 50 ms limit, on a barrier that nobody will ever arrive at.
+__global__ void wait_expiry_kernel(int32_t* status) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, 50000000ull);
+}
+
 TcParams base_params(const Plan& pl, const Buffers& b) {
   TcParams p = {};
   p.d = pl.d; p.F = pl.F; p.E = pl.E; p.r_pad_max = pl.r_pad_max;
@@ -480,6 +493,11 @@ TcParams base_params(const Plan& pl, const Buffers& b) {
 }
 
 }  // namespace
+
+cudaError_t launch_wait_expiry_selftest(int32_t* status, cudaStream_t st) {
+  wait_expiry_kernel<<<1, 32, 0, st>>>(status);
+  return cudaGetLastError();
+}
 
 btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                       const Buffers& b, int save, cudaStream_t st) {

@@ -289,3 +289,12 @@ def test_capacity_factor_small_batch_and_limits(dtype):
     assert torch.equal(free["y"], wide["y"]) and torch.equal(free["routing"].perm, wide["routing"].perm)
     with pytest.raises(B.BtxError):
         gpu_forward(inp, E, B.ROUTE_SOFT, 0.01, None, capacity_factor=1.5)
+
+
+def test_bounded_wait_expires_and_the_context_stays_usable():
+    """The safety net of the tensor-core kernels: a device-side wait that nothing will satisfy gives up
+    after its limit, the status word reports it, the kernel returns, and later calls work as usual."""
+    ws = torch.empty(4096, dtype=torch.uint8, device=DEV)
+    B.btx_selftest_wait_expiry(ws)
+    assert B.btx_device_status(ws) == B.BTX_ERR_TIMEOUT
+    run_case(300, 128, 264, 4, 2, torch.bfloat16, seed=3)        # same context, fresh call: status OK inside
