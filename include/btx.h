@@ -114,7 +114,10 @@ btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, const void* 
  * `saved` is the buffer the forward call filled with the same desc and inputs.
  * Outputs: dx[T,d] (dtype); dw_router[E,d], dbias[E] (may be NULL), dw1,dw3[E,F,d], dw2[E,d,F],
  * all fp32.  accumulate = 0 overwrites the weight gradients, 1 adds to them.  With desc.skip_wgrad
- * the three expert gradients are not computed and dw1, dw3, dw2 may be NULL. */
+ * the three expert gradients are not computed and dw1, dw3, dw2 may be NULL.
+ * The memory-bound router kernels run beside the weight-gradient GEMMs on a helper stream that the
+ * library creates once per device (the only CUDA resource it keeps) and that is joined back into
+ * `stream` before the call returns: everything is complete when `stream` is. */
 btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void* w_router,
                             const float* router_bias, const float* router_noise,
                             const void* w1, const void* w3, const void* w2,

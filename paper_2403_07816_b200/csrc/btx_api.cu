@@ -139,6 +139,36 @@ static EffectiveRouting effective_routing(const btx_moe_desc* desc) {
 
 static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
 
+// One helper stream per device, created on first use and kept for the life of the process: the
+// backward pass runs its memory-bound router kernels on it beside the tensor-bound weight-gradient
+// GEMMs.  nullptr when it cannot be had; the backward then runs on the caller's stream alone.
+static cudaStream_t helper_stream() {
+  static std::mutex mu;
+  static cudaStream_t streams[64] = {};
+  static bool failed[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (streams[dev] == nullptr && !failed[dev]) {
+    if (cudaStreamCreateWithFlags(&streams[dev], cudaStreamNonBlocking) != cudaSuccess) {
+      streams[dev] = nullptr;
+      failed[dev] = true;
+      cudaGetLastError();
+    }
+  }
+  return streams[dev];
+}
+
+struct ScopedEvents {                   // destroyed on every return path; destruction waits for nothing
+  cudaEvent_t e[4] = {nullptr, nullptr, nullptr, nullptr};
+  bool create(int n) {
+    for (int i = 0; i < n; ++i)
+      if (cudaEventCreateWithFlags(&e[i], cudaEventDisableTiming) != cudaSuccess) return false;
+    return true;
+  }
+  ~ScopedEvents() { for (cudaEvent_t x : e) if (x) cudaEventDestroy(x); }
+};
+
 static btx_status check_device() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return BTX_ERR_CUDA;
@@ -262,16 +292,29 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
   BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
   BTX_CUDA_OK(launch_gather_rows(pl, dy, b.dys, b, st));
   mark_stage(1, st);
+  // The router backward (memory-bound, a few small kernels) depends on dgrad-2 and dgrad-1 only: it runs
+  // on the helper stream beside the three tensor-bound weight-gradient GEMMs and joins `stream` at the end.
+  ScopedEvents evs;
+  cudaStream_t side = skip_wgrad ? nullptr : helper_stream();
+  if (side != nullptr && !evs.create(2)) side = nullptr;
+  cudaEvent_t after_dx = side != nullptr ? evs.e[0] : nullptr;
   if (desc->dtype == BTX_F32) {
-    BTX_CUDA_OK(launch_expert_backward_f32(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, skip_wgrad, st));
+    BTX_CUDA_OK(launch_expert_backward_f32(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, skip_wgrad, after_dx, st));
   } else {
-    if ((s = launch_expert_backward_bf16(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, skip_wgrad, st)) != BTX_OK)
+    if ((s = launch_expert_backward_bf16(pl, w1, w3, w2, b, dw1, dw3, dw2, accumulate, skip_wgrad, after_dx, st)) !=
+        BTX_OK)
       return s;
   }
   const EffectiveRouting er = effective_routing(desc);
+  cudaStream_t rst = side != nullptr ? side : st;
+  if (side != nullptr) BTX_CUDA_OK(cudaStreamWaitEvent(side, after_dx, 0));
   BTX_CUDA_OK(launch_router_backward(pl, desc->dtype, er.routing, desc->lb_alpha, lb_grad_scale,
                                      desc->lb_stopgrad_u, 1, x, w_router, b, dx, dw_router, dbias, nullptr,
-                                     accumulate, er.inv_tau, st));
+                                     accumulate, er.inv_tau, rst));
+  if (side != nullptr) {
+    BTX_CUDA_OK(cudaEventRecord(evs.e[1], side));
+    BTX_CUDA_OK(cudaStreamWaitEvent(st, evs.e[1], 0));
+  }
   mark_stage(7, st);
   return BTX_OK;
 }
@@ -293,10 +336,7 @@ extern "C" btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_
   cudaStream_t cs = (cudaStream_t)copy_stream;
   const bool overlap = copy_stream != nullptr && copy_stream != stream;
   const size_t act_bytes = (size_t)pl.T * pl.d * pl.esize;
-  struct Events {                     // destroyed on every return path; destruction waits for nothing
-    cudaEvent_t e[4] = {nullptr, nullptr, nullptr, nullptr};
-    ~Events() { for (cudaEvent_t x : e) if (x) cudaEventDestroy(x); }
-  } evs;
+  ScopedEvents evs;
   cudaEvent_t &ev_start = evs.e[0], &ev_dy = evs.e[1], &ev_fwd = evs.e[2], &ev_y = evs.e[3];
   if (overlap) {
     // dy travels to the device while the forward runs, y travels back while the backward runs

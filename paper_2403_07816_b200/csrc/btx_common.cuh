@@ -90,7 +90,7 @@ cudaError_t launch_expert_forward_f32(const Plan& pl, const void* w1, const void
                                       const Buffers& b, int save, cudaStream_t st);
 cudaError_t launch_expert_backward_f32(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                        const Buffers& b, float* dw1, float* dw3, float* dw2, int accumulate,
-                                       int skip_wgrad, cudaStream_t st);
+                                       int skip_wgrad, cudaEvent_t after_dx, cudaStream_t st);
 btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                       const Buffers& b, int save, cudaStream_t st);
 int pick_decode_splits(int base_tiles, int kb_total);
@@ -98,7 +98,7 @@ btx_status launch_expert_forward_small_bf16(const Plan& pl, const void* w1, cons
                                             const Buffers& b, int save, cudaStream_t st);
 btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                        const Buffers& b, float* dw1, float* dw3, float* dw2, int accumulate,
-                                       int skip_wgrad, cudaStream_t st);
+                                       int skip_wgrad, cudaEvent_t after_dx, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
 // Device helpers

@@ -185,7 +185,7 @@ cudaError_t launch_expert_forward_f32(const Plan& pl, const void* w1, const void
 
 cudaError_t launch_expert_backward_f32(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                        const Buffers& b, float* dw1, float* dw3, float* dw2, int accumulate,
-                                       int skip_wgrad, cudaStream_t st) {
+                                       int skip_wgrad, cudaEvent_t after_dx, cudaStream_t st) {
   SimtParams p = {};
   p.d = pl.d; p.F = pl.F; p.E = pl.E; p.r_pad_max = pl.r_pad_max;
   p.tile_expert = b.tile_expert; p.pad_offsets = b.pad_offsets; p.rowmap = b.rowmap; p.gates = b.gates;
@@ -201,6 +201,7 @@ cudaError_t launch_expert_backward_f32(const Plan& pl, const void* w1, const voi
   p.o0 = b.dxp; p.N = pl.d;
   simt_gemm_kernel<S_DX><<<dim3((pl.d + TN - 1) / TN, mt), 256, 0, st>>>(p);
   mark_stage(3, st);
+  if (after_dx != nullptr) cudaEventRecord(after_dx, st);      // the router backward may start here
   if (skip_wgrad) return cudaGetLastError();
   // wgrads: contraction over the expert's (padded) token rows
   p.a0 = (const float*)b.dys; p.ldp = pl.d; p.b0 = (const float*)b.ga; p.ldq = pl.F; p.o0 = dw2; p.M = pl.d; p.N = pl.F;

@@ -524,7 +524,7 @@ btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void
 
 btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                        const Buffers& b, float* dw1, float* dw3, float* dw2, int accumulate,
-                                       int skip_wgrad, cudaStream_t st) {
+                                       int skip_wgrad, cudaEvent_t after_dx, cudaStream_t st) {
   const uint64_t d = pl.d, F = pl.F, E = pl.E, RP = pl.r_pad_max;
   CUtensorMap a0, a1, b0, b1;
   btx_status s;
@@ -545,6 +545,7 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   p.of = b.dxp; p.wide = aligned32(b.dxp);
   if ((s = launch_tc<G_DX>(a0, a1, b0, b1, p, pl.mt_max * p.n_tiles, 1, st)) != BTX_OK) return s;
   mark_stage(3, st);
+  if (after_dx != nullptr && cudaEventRecord(after_dx, st) != cudaSuccess) return BTX_ERR_CUDA;   // the router backward may start here
   if (skip_wgrad) return BTX_OK;
   // wgrads: contraction over the expert's padded token rows, both operands MN-major.  The operand
   // indexed by the gradient's contiguous (column) index goes on the M side, so that the 32 lanes of
