@@ -298,3 +298,42 @@ def test_bounded_wait_expires_and_the_context_stays_usable():
     B.btx_selftest_wait_expiry(ws)
     assert B.btx_device_status(ws) == B.BTX_ERR_TIMEOUT
     run_case(300, 128, 264, 4, 2, torch.bfloat16, seed=3)        # same context, fresh call: status OK inside
+
+
+def test_training_step_replays_from_a_cuda_graph():
+    """Forward + backward issue only stream-ordered work (kernels, memsets, event fork/join with the
+    library's helper stream), so the pair can be captured once and replayed: same bits as the direct calls."""
+    T, d, F, E, k = 1200, 256, 528, 4, 2
+    inp = synth.moe_inputs(T, d, F, E, 23, torch.bfloat16, DEV)
+    desc = B.make_desc(T, d, F, E, k, torch.bfloat16, B.ROUTE_TOPK, 0.01, False, True)
+    ws, saved = B.alloc_buffers(desc, DEV)
+    f32 = dict(dtype=torch.float32, device=DEV)
+    outs = dict(y=torch.empty_like(inp["x"]), dx=torch.empty_like(inp["x"]), dwr=torch.empty(E, d, **f32),
+                dbias=torch.empty(E, **f32), dw1=torch.empty(E, F, d, **f32), dw3=torch.empty(E, F, d, **f32),
+                dw2=torch.empty(E, d, F, **f32))
+
+    def step():
+        B.btx_moe_forward(desc, inp["x"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], outs["y"], None,
+                          saved, ws)
+        B.btx_moe_backward(desc, inp["x"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], inp["dy"], 1.0,
+                           saved, outs["dx"], outs["dwr"], outs["dbias"], outs["dw1"], outs["dw3"], outs["dw2"], 0, ws)
+
+    step()
+    torch.cuda.synchronize()
+    direct = {n: t.clone() for n, t in outs.items()}
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()                                   # warm-up on the capture stream
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for t in outs.values():
+        t.zero_()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert B.btx_device_status(ws) == B.BTX_OK
+    for n, t in outs.items():
+        assert torch.equal(t, direct[n]), n
