@@ -403,7 +403,7 @@ def run_moe(args, workload):
     if rank == 0 and world == 1 and not args.no_cpu_baseline and workload != "decode" and not args.tokens:
         del sets
         torch.cuda.empty_cache()
-        n_tok = 128 if train else 256
+        n_tok = 4096                           # about 10-30 s of host work
         fn, n = oracle_step_fn(workload, n_tok, device="cpu")
         t0 = time.perf_counter(); fn(); dt = time.perf_counter() - t0
         line["cpu_baseline"] = {"value": n / dt, "unit": "tokens/s", "cores": host_cores(), "kind": "oracle",
