@@ -222,13 +222,20 @@ def swiglu_ffn(x, w1, w3, w2, return_hidden=False):
 # MoE forward
 # --------------------------------------------------------------------------------------
 
-def route(x, w_router, k, routing=ROUTE_TOPK, router_bias=None, logits=None, noise=None, tau=1.0):
+def route(x, w_router, k, routing=ROUTE_TOPK, router_bias=None, logits=None, noise=None, tau=1.0,
+          select_fp32=False):
     """Steps 1-4: logits (or the caller's fp32 logits), selection, gates, full softmax.
 
     ROUTE_SAMPLE1 (Section 3.3, "Sample Top-1"): with Gumbel noise G (an input) the soft sample is
     SoftMax((z + G) / tau); only its largest entry is kept as the gate of that one expert.  tau = 0
     is the inference rule, hard sampling: the expert arg-max(z + G) with gate 1.  For this mode the
     returned probabilities are those of the perturbed logits (the quantity the gate is taken from).
+
+    `select_fp32`: the arg-max of Sample Top-1 is an integer decided by floating point.  When the
+    routing of an fp32 implementation is to be reproduced bit for bit (its fp32 logits and the fp32
+    noise are passed in), the perturbed logits that DECIDE the expert are formed the way that
+    implementation forms them, by one fp32 addition z + G, so that two sums that fp32 rounds to the
+    same number tie here as well (and go to the lower index).  Gate and probabilities stay fp64.
     """
     z = router_logits(x, w_router, router_bias) if logits is None else _f64(logits)
     E = z.shape[1]
@@ -239,7 +246,10 @@ def route(x, w_router, k, routing=ROUTE_TOPK, router_bias=None, logits=None, noi
         if noise is None:
             raise ValueError("Sample Top-1 routing needs the Gumbel noise")
         zp = z + _f64(noise)
-        idx = top_k_select(zp, 1)
+        if select_fp32:
+            idx = top_k_select(np.asarray(z, dtype=np.float32) + np.asarray(noise, dtype=np.float32), 1)
+        else:
+            idx = top_k_select(zp, 1)
         if tau > 0:
             zp = zp / float(tau)
             p = full_softmax(zp)
@@ -255,7 +265,8 @@ def route(x, w_router, k, routing=ROUTE_TOPK, router_bias=None, logits=None, noi
 
 
 def moe_forward(x, w_router, w1, w3, w2, k, routing=ROUTE_TOPK, alpha=0.01,
-                router_bias=None, logits=None, tokens=None, noise=None, tau=1.0, capacity_factor=0.0):
+                router_bias=None, logits=None, tokens=None, noise=None, tau=1.0, capacity_factor=0.0,
+                select_fp32=False):
     """FF_MoE(x) = sum_i g_i(W_l x) FF_i(x), skipping experts whose gate is zero.
 
     capacity_factor > 0 (Section 4.1, Switch routing): an assignment beyond its expert's capacity
@@ -269,7 +280,7 @@ def moe_forward(x, w_router, w1, w3, w2, k, routing=ROUTE_TOPK, alpha=0.01,
     x = _f64(x)
     T, d = x.shape
     E = np.asarray(w1).shape[0]
-    z, idx, g, p_tok = route(x, w_router, k, routing, router_bias, logits, noise, tau)
+    z, idx, g, p_tok = route(x, w_router, k, routing, router_bias, logits, noise, tau, select_fp32)
     gd = dense_gates(idx, g, E)
     loss, u, p = lb_loss(gd, p_tok, alpha)
     kk = idx.shape[1]
@@ -339,7 +350,7 @@ def router_backward_dz(idx, gates, probs, dgate, u, alpha, lb_grad_scale, routin
 
 def moe_backward(x, w_router, w1, w3, w2, dy, k, routing=ROUTE_TOPK, alpha=0.01,
                  lb_grad_scale=1.0, lb_stopgrad_u=False, router_bias=None, logits=None, noise=None, tau=1.0,
-                 capacity_factor=0.0):
+                 capacity_factor=0.0, select_fp32=False):
     """Gradients of  <Y, dY> + lb_grad_scale * L_LB  w.r.t. x, W_l, bias, W1, W3, W2 (all tokens).
     A dropped assignment (capacity_factor > 0) is absent from Y, so nothing flows through it; the
     keep/drop decision itself is piecewise constant."""
@@ -347,7 +358,7 @@ def moe_backward(x, w_router, w1, w3, w2, dy, k, routing=ROUTE_TOPK, alpha=0.01,
     dy = _f64(dy)
     T, d = x.shape
     E, F, _ = np.asarray(w1).shape
-    z, idx, g, p_tok = route(x, w_router, k, routing, router_bias, logits, noise, tau)
+    z, idx, g, p_tok = route(x, w_router, k, routing, router_bias, logits, noise, tau, select_fp32)
     if routing == ROUTE_SAMPLE1 and alpha != 0:
         raise ValueError("Sample Top-1 routing is defined here without the load-balancing loss (alpha = 0)")
     kk = idx.shape[1]
@@ -452,6 +463,17 @@ def moe_backward_token_slice(x, w_router, w1, w3, w2, dy, idx, gates, probs, u, 
                             routing, batch_size=T)
     dx += dz @ _f64(w_router)
     return dict(dx=dx, dlogits=dz, dgate=dgate)
+
+
+def router_wgrad_from_dz(x, dz):
+    """dW_l = sum_t dz_t (outer) x_t  and  dbias = sum_t dz_t  over all tokens, from a supplied
+    d(loss)/d(logits) array dz[T, E]: the last step of the router backward on its own, so that a
+    full-size router gradient can be checked against the dz another implementation produced."""
+    x = _f64(x)
+    dz = _f64(dz)
+    if dz.shape[0] != x.shape[0]:
+        raise ValueError("dz and x must have one row per token")
+    return dz.T @ x, dz.sum(axis=0)
 
 
 def expert_wgrad_hidden_slice(x, w1, w3, w2, dy, idx, gates, e, hidden, keep=None):

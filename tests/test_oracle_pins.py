@@ -329,6 +329,33 @@ def test_slice_modes_agree_with_full_backward():
             np.testing.assert_allclose(d2, full["dw2"][e][:, J], rtol=1e-11, atol=1e-13)
 
 
+def test_router_gradient_from_a_supplied_dz():
+    # closed form: dz nonzero at one (token, expert) entry only -> that row of dW_l is dz * x_t, dbias picks it up
+    x, wr, w1, w3, w2, dy = small_problem(31, T=9, d=5)
+    dz = np.zeros((9, 4))
+    dz[6, 2] = -1.5
+    dw, db = o.router_wgrad_from_dz(x, dz)
+    want = np.zeros((4, 5))
+    want[2] = -1.5 * x[6]
+    np.testing.assert_allclose(dw, want, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(db, [0.0, 0.0, -1.5, 0.0], rtol=0, atol=0)
+    # scalar loops on a tiny case (operand orientation: [E, d], not [d, E])
+    r = RNG(32)
+    dz = r.standard_normal((9, 4))
+    dw, db = o.router_wgrad_from_dz(x, dz)
+    for e in range(4):
+        assert abs(db[e] - sum(dz[t, e] for t in range(9))) < 1e-13
+        for c in range(5):
+            assert abs(dw[e, c] - sum(dz[t, e] * x[t, c] for t in range(9))) < 1e-13
+    # fed the full backward's own dz it reproduces that backward's router gradients (which finite differences pin)
+    full = o.moe_backward(x, wr, w1, w3, w2, dy, k=2, alpha=0.3)
+    dw, db = o.router_wgrad_from_dz(x, full["dlogits"])
+    np.testing.assert_allclose(dw, full["dw_router"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(db, full["dbias"], rtol=1e-12, atol=1e-14)
+    with pytest.raises(ValueError):
+        o.router_wgrad_from_dz(x, dz[:5])
+
+
 def test_logits_override_decides_routing():
     x, wr, w1, w3, w2, _ = small_problem(15)
     z32 = o.router_logits(x, wr).astype(np.float32)
@@ -428,6 +455,25 @@ def test_sample_top1_selection_and_temperature_limits():
     e = hard["topk_idx"][:, 0]
     want = np.stack([o.swiglu_ffn(x[t:t + 1], w1[e[t]], w3[e[t]], w2[e[t]])[0] for t in range(x.shape[0])])
     np.testing.assert_allclose(hard["y"], want, rtol=1e-12, atol=1e-13)
+
+
+def test_sample_top1_selection_in_fp32_ties_like_an_fp32_implementation():
+    # z + G differs between the experts only below fp32 resolution: 1 + 2^-25 rounds to 1 in fp32.
+    # In fp64 expert 1 wins; an fp32 implementation sees a tie, which goes to the lower index.
+    z = np.array([[0.0, 2.0 ** -25, -3.0]], dtype=np.float32)
+    G = np.array([[1.0, 1.0, 0.0]], dtype=np.float32)
+    for tau in (0.0, 0.8):
+        _, idx64, _, _ = o.route(None, None, 1, o.ROUTE_SAMPLE1, logits=z, noise=G, tau=tau)
+        _, idx32, g32, p32 = o.route(None, None, 1, o.ROUTE_SAMPLE1, logits=z, noise=G, tau=tau, select_fp32=True)
+        assert idx64.tolist() == [[1]] and idx32.tolist() == [[0]]
+        # the gate is still the fp64 softmax entry of the chosen expert (1 for hard sampling)
+        want = 1.0 if tau == 0.0 else float(o.full_softmax((z.astype(np.float64) + G) / tau)[0, 0])
+        assert abs(float(g32[0, 0]) - want) < 1e-15
+    # where fp32 resolves the two sums the flag changes nothing
+    z2 = np.array([[0.0, 2.0 ** -20, -3.0]], dtype=np.float32)
+    _, a, _, _ = o.route(None, None, 1, o.ROUTE_SAMPLE1, logits=z2, noise=G, tau=0.5)
+    _, b, _, _ = o.route(None, None, 1, o.ROUTE_SAMPLE1, logits=z2, noise=G, tau=0.5, select_fp32=True)
+    assert a.tolist() == b.tolist() == [[1]]
 
 
 def test_hard_sampling_follows_the_softmax_distribution():
