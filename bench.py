@@ -1,10 +1,16 @@
 #!/usr/bin/env python
-"""Benchmark of the MoE feed-forward hot path (forward + backward) on synthetic Llama-2-7B-shaped
-data: T=16384 tokens, d_model 4096, d_ff 11008, 4 experts, top-2, BF16 with FP32 accumulation.
+"""Benchmark of the MoE feed-forward hot path on synthetic Llama-2-7B-shaped data.
 
     python bench.py --gpus 1 --steps 20 --warmup 5            # the CUDA path, one JSON line
     python bench.py --impl reference --steps 3 --warmup 1     # the CPU oracle on host cores
-    python bench.py --workload fwd|decode|merge               # the other measured paths
+    python bench.py --workload fwd|decode|merge               # one of the other paths on its own
+
+The headline is the training step (forward + backward) of one layer: T=16384 tokens, d_model 4096,
+d_ff 11008, 4 experts, top-2, BF16 with FP32 accumulation.  On one GPU the same process then measures the
+other configurations, one after the other with the previous one's buffers freed, and adds them to the
+line under "sub": the forward alone at T=4096, the three routing variants at T=16384 (Switch top-1, soft
+routing over all experts, top-2 with a skewed router), the decode-shaped forward over 32 layers and the
+merge of four Llama-2-7B-shaped parameter sets, each with its own clock samples.
 
 Under torchrun every rank runs an independent replica on its own batch (the path has no exchange
 step), times K steps between barriers, and rank 0 prints whole-job tokens/s from the max time.
@@ -12,6 +18,8 @@ step), times K steps between barriers, and rank 0 prints whole-job tokens/s from
 from __future__ import annotations
 
 import argparse
+import gc
+import hashlib
 import json
 import os
 import statistics
@@ -23,16 +31,26 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+D_MODEL, D_FF, N_EXPERTS = 4096, 11008, 4
 WORKLOADS = {
-    # name: (T, d_model, d_ff, E, k, seed)
-    "fwd_bwd": (16384, 4096, 11008, 4, 2, 2),
-    "fwd": (4096, 4096, 11008, 4, 2, 1),
-    "decode": (32, 4096, 11008, 4, 2, 4),
+    # name: (T, k, seed, routing name, skewed router bias, forward+backward, layers)
+    "fwd_bwd": (16384, 2, 2, "topk", False, True, 1),
+    "fwd": (4096, 2, 1, "topk", False, False, 1),
+    "switch_top1": (16384, 1, 3, "switch", False, True, 1),
+    "soft_all4": (16384, 4, 3, "soft", False, True, 1),
+    "top2_skewed": (16384, 2, 3, "topk", True, True, 1),
+    "decode": (32, 2, 4, "topk", False, False, 32),
 }
 ALPHA = 0.01
-# dram__bytes_read.sum + dram__bytes_write.sum of the seven tc_gemm_kernel launches of one training step
-# at T=16384 (26.38 GB read + 7.43 GB written); the algorithmic minimum is 10.3 GB read + 7.6 GB written
-TC_GEMM_DRAM_BYTES_PER_STEP = 33.81e9
+SOAK_S = 2.0             # untimed run of the same step before the warm-up: power state and clocks settle
+E2E_STEPS = 50
+
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core GEMM launches of one training
+# step, from the ncu capture summarised under profiles/ (taken at T=4096 and scaled by 4 to T=16384: every
+# operand and output of these launches grows in proportion to T).  The figure belongs to the kernel sources
+# whose hash is recorded with it; with any other sources the bench reports traffic = null.
+TC_GEMM_TRAFFIC = {"bytes_per_step_T16384": 33.81e9, "sources_sha256_16": "unset"}
+TC_GEMM_SOURCES = ("btx_gemm_tc.cu", "btx_tc_ptx.cuh", "btx_common.cuh")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -48,6 +66,14 @@ def load_peaks():
     return p
 
 
+def kernel_sources_hash():
+    h = hashlib.sha256()
+    for name in TC_GEMM_SOURCES:
+        with open(os.path.join(ROOT, "paper_2403_07816_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -57,7 +83,6 @@ class ClockSampler:
     def __init__(self, gpu_index):
         self.proc = None
         self.gpu = gpu_index
-        self.lines = []
 
     def start(self):
         try:
@@ -97,23 +122,20 @@ class ClockSampler:
 # ----------------------------------------------------------------------------------------------
 
 def oracle_step_fn(workload, tokens, device="cpu"):
-    """Returns (fn, n_tokens): fn() runs the oracle forward + backward on the first `tokens` tokens
-    of the workload's batch with the full expert weights."""
-    import numpy as np
+    """Returns (fn, n_tokens): fn() runs the oracle (forward + backward for the training workloads) on the
+    first `tokens` tokens of the workload's batch with the full expert weights."""
     import torch
     from oracle import btx_oracle as o
     from paper_2403_07816_b200 import synth
-    T, d, F, E, k, seed = WORKLOADS[workload]
-    inp = synth.moe_inputs(T, d, F, E, seed, torch.bfloat16, device)
+    T, k, seed, _, _, train, _ = WORKLOADS[workload]
+    inp = synth.moe_inputs(T, D_MODEL, D_FF, N_EXPERTS, seed, torch.bfloat16, device)
     n = min(tokens, T)
     cpu = {name: synth.to_f64_numpy(t[:n] if name in ("x", "dy") else t) for name, t in inp.items()}
 
     def fn():
-        if workload == "fwd_bwd":
-            o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], k, alpha=ALPHA)
+        o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], k, alpha=ALPHA)
+        if train:
             o.moe_backward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], cpu["dy"], k, alpha=ALPHA)
-        else:
-            o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], k, alpha=ALPHA)
     return fn, n
 
 
@@ -129,14 +151,20 @@ def run_reference(args):
     if rank != 0:
         return
     workload = args.workload if args.workload in ("fwd_bwd", "fwd") else "fwd_bwd"
-    T, d, F, E, k, seed = WORKLOADS[workload]
-    # size the sample so that steps+warmup fit in about two minutes: calibrate on 16 tokens
-    fn, n = oracle_step_fn(workload, 16)
-    t0 = time.perf_counter(); fn(); cal = time.perf_counter() - t0
+    T, k = WORKLOADS[workload][0], WORKLOADS[workload][1]
+    # A step of the oracle costs a fixed part (every expert's fp64 weights pass through the cores once, whatever
+    # the batch) plus a part per token.  Two calibration passes give both; the sample is then sized so that
+    # steps + warm-up take about two and a half minutes.
+    fn, _ = oracle_step_fn(workload, 16)
+    t0 = time.perf_counter(); fn(); c16 = time.perf_counter() - t0
+    fn, _ = oracle_step_fn(workload, 272)
+    t0 = time.perf_counter(); fn(); c272 = time.perf_counter() - t0
+    per_token = max((c272 - c16) / 256.0, 1e-5)
+    fixed = max(c16 - 16 * per_token, 0.0)
     total = max(1, args.steps + args.warmup)
-    budget = 120.0 / total
-    tokens = int(max(16, min(T, 16 * budget / max(cal, 1e-3) * 0.6)))
-    tokens = max(16, tokens // 16 * 16)
+    budget = 150.0 / total
+    tokens = int((budget - fixed) / per_token) if budget > fixed else 16
+    tokens = max(16, min(T, tokens // 16 * 16))
     fn, n = oracle_step_fn(workload, tokens)
     for _ in range(args.warmup):
         fn()
@@ -150,8 +178,8 @@ def run_reference(args):
         "impl": "reference", "metric": "moe_ffn_%s_tokens_per_s" % workload, "value": value, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{workload}: first {n} of T={T} tokens per step, d_model={d}, d_ff={F}, E={E}, top-{k}, "
-                               "fp64 CPU oracle (numpy/OpenBLAS)"},
+        "config": {"workload": f"{workload}: first {n} of T={T} tokens per step, d_model={D_MODEL}, d_ff={D_FF}, "
+                               f"E={N_EXPERTS}, top-{k}, fp64 CPU oracle (numpy/OpenBLAS)"},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                          "sample": f"{n} tokens per step, full expert weights"},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -203,55 +231,114 @@ def aggregate_throughput(units_per_rank, ms_local, world, device):
     return units_per_rank * world / (ms * 1e-3), ms
 
 
-def run_moe(args, workload):
+def free_device_memory():
     import torch
-    from paper_2403_07816_b200 import binding as B, build as builder, synth
-    world, rank, local = dist_setup(args)
-    if rank == 0:
-        builder.build()
-    barrier(world)
-    dev = torch.device("cuda", local)
-    T, d, F, E, k, seed = WORKLOADS[workload]
-    if args.tokens:
-        T = args.tokens                      # reduced batch for profiler captures
-    train = workload == "fwd_bwd"
-    layers = (args.layers or 32) if workload == "decode" else 1
-    K, W = args.steps, max(args.warmup, 3)
-    peaks = load_peaks()
+    gc.collect()
+    torch.cuda.empty_cache()
 
-    # one independent seeded layer per decode "layer"; replicas differ by rank through the seed
-    sets = [synth.moe_inputs(T, d, F, E, seed + 1000 * rank, torch.bfloat16, dev, layer=l, with_dy=train)
-            for l in range(layers)]
-    desc = B.make_desc(T, d, F, E, k, torch.bfloat16, B.ROUTE_TOPK, ALPHA, False, train)
-    ws, saved = B.alloc_buffers(desc, dev)
-    y = torch.empty(T, d, dtype=torch.bfloat16, device=dev)
-    if train:
-        f32 = dict(dtype=torch.float32, device=dev)
-        dx = torch.empty_like(y)
-        dwr, dbias = torch.empty(E, d, **f32), torch.empty(E, **f32)
-        dw1, dw3, dw2 = torch.empty(E, F, d, **f32), torch.empty(E, F, d, **f32), torch.empty(E, d, F, **f32)
 
-    def step(i=0):
-        for inp in sets:
-            B.btx_moe_forward(desc, inp["x"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], y, None,
-                              saved if train else None, ws)
-            if train:
-                B.btx_moe_backward(desc, inp["x"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], inp["dy"],
-                                   1.0, saved, dx, dwr, dbias, dw1, dw3, dw2, 0, ws)
+# kernels launched per call (memsets and copies are not counted)
+LAUNCHES_FWD = 9          # router, loss finalise, 3 permutation kernels, gather, GEMM-1, GEMM-2, combine
+LAUNCHES_FWD_SMALL = 6    # one-launch routing, gather, pass 1, SwiGLU fix-up, pass 2, combine
+LAUNCHES_BWD = 11         # dy gather, dgrad-2, dgrad-1, 3 weight gradients, row-sum, dz, dW_l partial, dx combine, reduce
 
-    def new_events(n):
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
-        for e in evs:
-            e.record()                       # creates the handles the stage hook records into
-        return evs
 
+class MoeRun:
+    """One configuration of the layer resident on the device: inputs, buffers and the step function."""
+
+    def __init__(self, workload, dev, rank, tokens=0, layers=0):
+        import torch
+        from paper_2403_07816_b200 import binding as B, synth
+        self.B, self.torch, self.dev = B, torch, dev
+        T, k, seed, routing, skew, train, n_layers = WORKLOADS[workload]
+        self.T = tokens or T
+        self.k, self.train, self.workload = k, train, workload
+        self.layers = layers or n_layers
+        self.routing = {"topk": B.ROUTE_TOPK, "switch": B.ROUTE_SWITCH, "soft": B.ROUTE_SOFT}[routing]
+        self.k_eff = N_EXPERTS if self.routing == B.ROUTE_SOFT else k
+        d, F, E = D_MODEL, D_FF, N_EXPERTS
+        # one independent seeded layer per decode "layer"; replicas differ by rank through the seed
+        self.sets = [synth.moe_inputs(self.T, d, F, E, seed + 1000 * rank, torch.bfloat16, dev, layer=l, with_dy=train)
+                     for l in range(self.layers)]
+        self.bias = synth.skew_bias(E, dev) if skew else None
+        self.desc = B.make_desc(self.T, d, F, E, k, torch.bfloat16, self.routing, ALPHA, False, train)
+        self.ws, self.saved = B.alloc_buffers(self.desc, dev)
+        self.y = torch.empty(self.T, d, dtype=torch.bfloat16, device=dev)
+        self.routing_out = None
+        if train:
+            f32 = dict(dtype=torch.float32, device=dev)
+            self.dx = torch.empty_like(self.y)
+            self.dwr, self.dbias = torch.empty(E, d, **f32), torch.empty(E, **f32)
+            self.dw1, self.dw3, self.dw2 = torch.empty(E, F, d, **f32), torch.empty(E, F, d, **f32), torch.empty(E, d, F, **f32)
+
+    def forward(self, inp, routing_out=None):
+        self.B.btx_moe_forward(self.desc, inp["x"], inp["w_router"], self.bias, inp["w1"], inp["w3"], inp["w2"], self.y,
+                               routing_out, self.saved if self.train else None, self.ws)
+
+    def backward(self, inp):
+        self.B.btx_moe_backward(self.desc, inp["x"], inp["w_router"], self.bias, inp["w1"], inp["w3"], inp["w2"],
+                                inp["dy"], 1.0, self.saved, self.dx, self.dwr, self.dbias, self.dw1, self.dw3, self.dw2,
+                                0, self.ws)
+
+    def step(self):
+        for inp in self.sets:
+            self.forward(inp)
+            if self.train:
+                self.backward(inp)
+
+    def launches_per_step(self):
+        fwd = LAUNCHES_FWD_SMALL if self.T * self.k_eff <= 1024 else LAUNCHES_FWD
+        return (fwd + (LAUNCHES_BWD if self.train else 0)) * self.layers
+
+    def flops_per_step(self, rows):
+        return (18 if self.train else 6) * rows * D_MODEL * D_FF * self.layers
+
+    def expert_counts(self):
+        r = self.B.Routing.empty(self.desc, self.dev)
+        self.forward(self.sets[0], r)
+        self.torch.cuda.synchronize()
+        return [int(v) for v in r.counts.cpu().tolist()]
+
+
+def new_events(torch, n):
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+    for e in evs:
+        e.record()                       # creates the handles the stage hook records into
+    return evs
+
+
+STAGES_F = ["route_permute_gather", "gemm1_swiglu", "gemm2_scatter", "combine"]
+STAGES_B = ["gather_dy", "dgrad2_swiglu_bwd", "dgrad1", "wgrad_w2", "wgrad_w1", "wgrad_w3", "router_bwd"]
+
+
+def soak(run, seconds):
+    """Runs the step untimed for at least `seconds` (host clock, synchronising every few steps)."""
+    torch = run.torch
+    t0 = time.perf_counter()
+    n = 0
+    while True:
+        for _ in range(4):
+            run.step()
+        n += 4
+        torch.cuda.synchronize()
+        if time.perf_counter() - t0 >= seconds:
+            return time.perf_counter() - t0, n
+
+
+def time_moe(run, K, W, world, local, soak_s, with_stages):
+    """Soak, W warm-up steps, then exactly K timed steps between barriers with CUDA events on the launching
+    stream and clock samples taken meanwhile.  Returns (ms per step, clocks, stage times or None, soak seconds)."""
+    torch, B = run.torch, run.B
+    soaked = 0.0
+    if soak_s > 0:
+        soaked, _ = soak(run, soak_s)
     for _ in range(W):
-        step()
+        run.step()
     torch.cuda.synchronize()
-    assert B.btx_device_status(ws) == B.BTX_OK
-
-    # ---- timed region: K steps between barriers, CUDA events on the launching stream ----
-    stage_events = [(new_events(5), new_events(8)) for _ in range(K)] if layers == 1 else None
+    assert B.btx_device_status(run.ws) == B.BTX_OK
+    stage_events = None
+    if with_stages and run.layers == 1:
+        stage_events = [(new_events(torch, 5), new_events(torch, 8)) for _ in range(K)]
     sampler = ClockSampler(local)
     barrier(world)
     sampler.start()
@@ -259,155 +346,217 @@ def run_moe(args, workload):
     e0.record()
     for i in range(K):
         if stage_events is None:
-            step()
+            run.step()
             continue
-        inp = sets[0]
+        inp = run.sets[0]
         B.btx_set_stage_events(stage_events[i][0])
-        B.btx_moe_forward(desc, inp["x"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], y, None,
-                          saved if train else None, ws)
-        if train:
+        run.forward(inp)
+        if run.train:
             B.btx_set_stage_events(stage_events[i][1])
-            B.btx_moe_backward(desc, inp["x"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], inp["dy"], 1.0,
-                               saved, dx, dwr, dbias, dw1, dw3, dw2, 0, ws)
+            run.backward(inp)
     B.btx_set_stage_events(None)
     e1.record()
     barrier(world)
     clocks = sampler.stop()
-    ms = max_over_ranks(e0.elapsed_time(e1) / K, world, dev)
-    assert B.btx_device_status(ws) == B.BTX_OK
-
-    R = T * k
-    flops_step = (18 if train else 6) * R * d * F * layers
-    fwd_launches = 6 if T * k <= 1024 else 9        # small batches: routing+permutation in one launch, two passes + fix-up
-    launches_per_step = (fwd_launches + (11 if train else 0)) * layers
-    line = {
-        "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "clocks": clocks,
-        "gpu_launches": launches_per_step * K,
-    }
-    if workload == "decode":
-        w_bytes = layers * 3 * E * d * F * 2
-        gbs = w_bytes / (ms * 1e-3) / 1e9
-        line.update(metric="moe_ffn_decode_weight_stream_GBps", value=gbs * world, unit="GB/s",
-                    config={"workload": f"decode: T={T} tokens x {layers} independent layers, d_model={d}, d_ff={F}, "
-                                        f"E={E}, top-{k}, bf16; {layers} distinct weight sets (34.6 GB) exceed L2"},
-                    roofline={"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                              "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["_source"],
-                              "kernel": "tc_swapk_kernel (weight-streaming passes) over the whole step"})
-        # per-layer stage times from one extra, untimed pass
-        evs = [new_events(5) for _ in sets]
-        for inp, ev in zip(sets, evs):
-            B.btx_set_stage_events(ev)
-            B.btx_moe_forward(desc, inp["x"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], y, None, None, ws)
-        B.btx_set_stage_events(None)
-        torch.cuda.synchronize()
-        names_f = ["route_permute_gather", "gemm1_swiglu", "gemm2_scatter", "combine"]
-        line["stages_ms"] = {"fwd." + nme: round(statistics.mean(ev[i].elapsed_time(ev[i + 1]) for ev in evs), 4)
-                             for i, nme in enumerate(names_f)}
-    else:
-        tokens_s = T / (ms * 1e-3) * world
-        line.update(metric="moe_ffn_%s_tokens_per_s" % workload, value=tokens_s, unit="tokens/s",
-                    tflops=flops_step / (ms * 1e-3) / 1e12 * world,
-                    config={"workload": f"{workload}: T={T} tokens, d_model={d}, d_ff={F}, E={E}, top-{k}, bf16 with "
-                                        "fp32 accumulation, lb alpha 0.01; inputs (1.2 GB of weights and activations "
-                                        "per step) exceed the 126 MB L2, no explicit flush"})
-        # per-stage times averaged over the timed steps
-        names_f = ["route_permute_gather", "gemm1_swiglu", "gemm2_scatter", "combine"]
-        names_b = ["gather_dy", "dgrad2_swiglu_bwd", "dgrad1", "wgrad_w2", "wgrad_w1", "wgrad_w3", "router_bwd"]
+    ms = max_over_ranks(e0.elapsed_time(e1) / K, world, run.dev)
+    assert B.btx_device_status(run.ws) == B.BTX_OK
+    stages = None
+    if stage_events is not None:
         stages = {}
-        for i, nme in enumerate(names_f):
+        for i, nme in enumerate(STAGES_F):
             stages["fwd." + nme] = statistics.mean(se[0][i].elapsed_time(se[0][i + 1]) for se in stage_events)
-        if train:
-            for i, nme in enumerate(names_b):
+        if run.train:
+            for i, nme in enumerate(STAGES_B):
                 stages["bwd." + nme] = statistics.mean(se[1][i].elapsed_time(se[1][i + 1]) for se in stage_events)
-        gemm_keys = [kname for kname in stages if "gemm" in kname or "grad" in kname]
-        gemm_ms = sum(stages[kname] for kname in gemm_keys)
-        achieved = flops_step / (gemm_ms * 1e-3) / 1e12
-        # the sustained cuBLAS figure is the yardstick once the power cap has pulled the clocks down (or the
-        # timed region is long enough that it would have); a short un-capped run is compared with the burst figure
-        sustained = "sw_power_cap" in (clocks.get("reasons") or []) or ms * K >= 1000.0
-        peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-        line["stages_ms"] = {kname: round(v, 4) for kname, v in stages.items()}
-        # DRAM bytes (read + write) of the seven launches of one step, from the ncu capture summarised in
-        # profiles/tc_gemm_kernel_fwd_bwd_T16384_dram.txt; it holds for that workload only
-        traffic = TC_GEMM_DRAM_BYTES_PER_STEP if (train and (T, d, F, E, k) == (16384, 4096, 11008, 4, 2)) else None
-        line["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                            "frac": achieved / peak, "traffic": traffic, "peak_source": peaks["_source"] + (" sustained" if sustained else " burst"),
-                            "kernel": f"tc_gemm_kernel, {len(gemm_keys)} launches per step (flops of all / summed time)",
-                            "frac_of_nominal_2250": achieved / 2250.0}
+    return ms, clocks, stages, soaked
 
-    # ---- end to end through the host-buffer entry point (training workload only) ----
-    if train and not args.no_e2e:
-        # Two steps in flight, each on its own stream pair and buffer set (the weights are shared), so
-        # that the upload of step i+1 travels while step i computes: the way a training loop that keeps
-        # the GPU busy would call the entry point.  Every step still uploads its own x, dy and brings
-        # back its own y, dx and loss inside the timed region.
-        inp = sets[0]
-        hx = inp["x"].cpu().pin_memory(); hdy = inp["dy"].cpu().pin_memory()
-        Ke = max(4, min(K, 10))
-        main = torch.cuda.current_stream(dev)
-        lanes = []
-        for i in range(2):
-            ln = dict(stream=torch.cuda.Stream(device=dev), copy=torch.cuda.Stream(device=dev),
-                      hy=torch.empty_like(hx).pin_memory(), hdx=torch.empty_like(hx).pin_memory(),
-                      hloss=torch.empty(1, dtype=torch.float32).pin_memory(),
-                      xd=torch.empty_like(inp["x"]), dyd=torch.empty_like(inp["x"]))
-            if i == 0:
-                ln.update(y=y, dx=dx, saved=saved, ws=ws, dwr=dwr, dbias=dbias, dw1=dw1, dw3=dw3, dw2=dw2)
-            else:
-                ws2, saved2 = B.alloc_buffers(desc, dev)
-                ln.update(y=torch.empty_like(y), dx=torch.empty_like(dx), saved=saved2, ws=ws2,
-                          dwr=torch.empty_like(dwr), dbias=torch.empty_like(dbias), dw1=torch.empty_like(dw1),
-                          dw3=torch.empty_like(dw3), dw2=torch.empty_like(dw2))
-            lanes.append(ln)
 
-        def e2e_step(i):
-            ln = lanes[i % 2]
-            with torch.cuda.stream(ln["stream"]):
-                B.btx_moe_step_host(desc, hx, hdy, ln["hy"], ln["hdx"], ln["hloss"], ln["xd"], ln["dyd"], ln["y"],
-                                    ln["dx"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], 1.0, ln["dwr"],
-                                    ln["dbias"], ln["dw1"], ln["dw3"], ln["dw2"], 0, ln["saved"], ln["ws"],
-                                    copy_stream=ln["copy"])
+def tensor_roofline(run, rows, stages, clocks, timed_s, peaks):
+    gemm_keys = [kname for kname in stages if "gemm" in kname or "grad" in kname]
+    gemm_ms = sum(stages[kname] for kname in gemm_keys)
+    achieved = run.flops_per_step(rows) / (gemm_ms * 1e-3) / 1e12
+    # the sustained cuBLAS figure is the yardstick once the power cap has pulled the clocks down (or the
+    # run, soak included, is long enough that it would have); a short un-capped run is compared with the burst figure
+    sustained = "sw_power_cap" in (clocks.get("reasons") or []) or timed_s >= 1.0
+    peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    traffic = None
+    if (run.workload, run.T) == ("fwd_bwd", 16384) and kernel_sources_hash() == TC_GEMM_TRAFFIC["sources_sha256_16"]:
+        traffic = TC_GEMM_TRAFFIC["bytes_per_step_T16384"]
+    return {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+            "traffic": traffic, "peak_source": peaks["_source"] + (" sustained" if sustained else " burst"),
+            "kernel": f"tc_gemm_kernel, {len(gemm_keys)} launches per step (flops of all / summed time)",
+            "frac_of_nominal_2250": achieved / 2250.0}
 
-        def join():
-            for ln in lanes:
-                main.wait_stream(ln["stream"])
 
-        def fork():
-            for ln in lanes:
-                ln["stream"].wait_stream(main)
-        fork()
-        for i in range(2):
-            e2e_step(i)
-        join()
-        barrier(world)
-        e0.record()
-        fork()
-        for i in range(Ke):
-            e2e_step(i)
-        join()
-        e1.record()
-        barrier(world)
+def measure_e2e(run, world, steps):
+    """The training step through the host-buffer entry point: pinned x, dy in; y, dx and the loss out, every step.
+    Two steps are in flight, each on its own stream pair and buffer set (the weights are shared), so that the
+    upload of step i+1 travels while step i computes: the way a training loop that keeps the GPU busy would call
+    the entry point."""
+    torch, B, dev = run.torch, run.B, run.dev
+    inp = run.sets[0]
+    hx = inp["x"].cpu().pin_memory(); hdy = inp["dy"].cpu().pin_memory()
+    main = torch.cuda.current_stream(dev)
+    lanes = []
+    for i in range(2):
+        ln = dict(stream=torch.cuda.Stream(device=dev), copy=torch.cuda.Stream(device=dev),
+                  hy=torch.empty_like(hx).pin_memory(), hdx=torch.empty_like(hx).pin_memory(),
+                  hloss=torch.empty(1, dtype=torch.float32).pin_memory(),
+                  xd=torch.empty_like(inp["x"]), dyd=torch.empty_like(inp["x"]))
+        if i == 0:
+            ln.update(y=run.y, dx=run.dx, saved=run.saved, ws=run.ws, dwr=run.dwr, dbias=run.dbias, dw1=run.dw1,
+                      dw3=run.dw3, dw2=run.dw2)
+        else:
+            ws2, saved2 = B.alloc_buffers(run.desc, dev)
+            ln.update(y=torch.empty_like(run.y), dx=torch.empty_like(run.dx), saved=saved2, ws=ws2,
+                      dwr=torch.empty_like(run.dwr), dbias=torch.empty_like(run.dbias), dw1=torch.empty_like(run.dw1),
+                      dw3=torch.empty_like(run.dw3), dw2=torch.empty_like(run.dw2))
+        lanes.append(ln)
+
+    def e2e_step(i):
+        ln = lanes[i % 2]
+        with torch.cuda.stream(ln["stream"]):
+            B.btx_moe_step_host(run.desc, hx, hdy, ln["hy"], ln["hdx"], ln["hloss"], ln["xd"], ln["dyd"], ln["y"],
+                                ln["dx"], inp["w_router"], run.bias, inp["w1"], inp["w3"], inp["w2"], 1.0, ln["dwr"],
+                                ln["dbias"], ln["dw1"], ln["dw3"], ln["dw2"], 0, ln["saved"], ln["ws"],
+                                copy_stream=ln["copy"])
+
+    def join():
         for ln in lanes:
-            assert B.btx_device_status(ln["ws"]) == B.BTX_OK
-        ems = max_over_ranks(e0.elapsed_time(e1) / Ke, world, dev)
-        act = T * d * 2
-        line["e2e"] = {"value": T / (ems * 1e-3) * world, "unit": "tokens/s", "h2d_bytes_per_step": 2 * act,
-                       "d2h_bytes_per_step": 2 * act + 4, "ms_per_step": ems, "steps": Ke,
-                       "call": "btx_moe_step_host (pinned host x, dy in; y, dx, loss out), two steps in flight on two "
-                               "stream pairs"}
+            main.wait_stream(ln["stream"])
+
+    def fork():
+        for ln in lanes:
+            ln["stream"].wait_stream(main)
+    fork()
+    for i in range(4):
+        e2e_step(i)
+    join()
+    sampler = ClockSampler(dev.index or 0)
+    barrier(world)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    fork()
+    for i in range(steps):
+        e2e_step(i)
+    join()
+    e1.record()
+    barrier(world)
+    clocks = sampler.stop()
+    for ln in lanes:
+        assert B.btx_device_status(ln["ws"]) == B.BTX_OK
+    ems = max_over_ranks(e0.elapsed_time(e1) / steps, world, dev)
+    act = run.T * D_MODEL * 2
+    return {"value": run.T / (ems * 1e-3) * world, "unit": "tokens/s", "h2d_bytes_per_step": 2 * act,
+            "d2h_bytes_per_step": 2 * act + 4, "ms_per_step": ems, "steps": steps, "clocks": clocks,
+            "call": "btx_moe_step_host (pinned host x, dy in; y, dx, loss out), two steps in flight on two "
+                    "stream pairs"}
+
+
+def describe(run):
+    T, k = run.T, run.k_eff
+    if run.workload == "decode":
+        return (f"decode: T={T} tokens x {run.layers} independent layers, d_model={D_MODEL}, d_ff={D_FF}, "
+                f"E={N_EXPERTS}, top-{k}, bf16; {run.layers} distinct weight sets "
+                f"({run.layers * 3 * N_EXPERTS * D_MODEL * D_FF * 2 / 1e9:.1f} GB) exceed L2")
+    how = {"topk": f"top-{k}", "switch": "Switch top-1", "soft": f"soft routing over all {N_EXPERTS}"}[WORKLOADS[run.workload][3]]
+    if run.bias is not None:
+        how += ", router bias on expert 0 (first choice of about 70 % of the tokens)"
+    return (f"{run.workload}: T={T} tokens, d_model={D_MODEL}, d_ff={D_FF}, E={N_EXPERTS}, {how}, bf16 with fp32 "
+            f"accumulation, lb alpha {ALPHA}, {'forward+backward' if run.train else 'forward only'}; inputs (1.2 GB of "
+            "weights and activations per step) exceed the 126 MB L2, no explicit flush")
+
+
+def moe_result(run, ms, clocks, stages, soaked, K, W, world, peaks, with_counts):
+    """Result object of one MoE configuration (used for the headline and for the sub-results)."""
+    counts = run.expert_counts() if with_counts else None
+    rows = sum(counts) if counts is not None else run.T * run.k_eff
+    res = {"steps": K, "warmup": W, "soak_s": round(soaked, 2), "ms_per_step": ms, "clocks": clocks,
+           "gpu_launches": run.launches_per_step() * K, "config": {"workload": describe(run)}}
+    if counts is not None:
+        res["expert_counts"] = counts
+    if run.workload == "decode":
+        w_bytes = run.layers * 3 * N_EXPERTS * D_MODEL * D_FF * 2
+        gbs = w_bytes / (ms * 1e-3) / 1e9
+        res.update(metric="moe_ffn_decode_weight_stream_GBps", value=gbs * world, unit="GB/s",
+                   roofline={"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0, "traffic": None,
+                             "peak_source": peaks["_source"],
+                             "kernel": "tc_swapk_kernel (weight-streaming passes) over the whole step"})
     else:
-        line["e2e"] = None
+        res.update(metric="moe_ffn_%s_tokens_per_s" % run.workload, value=run.T / (ms * 1e-3) * world, unit="tokens/s",
+                   tflops=run.flops_per_step(rows) / (ms * 1e-3) / 1e12 * world)
+        res["tflops_frac_of_nominal_2250"] = res["tflops"] / world / 2250.0
+    if stages is not None:
+        res["stages_ms"] = {kname: round(v, 4) for kname, v in stages.items()}
+        if run.workload != "decode":
+            res["roofline"] = tensor_roofline(run, rows, stages, clocks, soaked + ms * K * 1e-3, peaks)
+    return res
+
+
+def decode_stage_times(run):
+    """Per-layer stage times of the decode path from one extra, untimed pass."""
+    torch, B = run.torch, run.B
+    evs = [new_events(torch, 5) for _ in run.sets]
+    for inp, ev in zip(run.sets, evs):
+        B.btx_set_stage_events(ev)
+        run.forward(inp)
+    B.btx_set_stage_events(None)
+    torch.cuda.synchronize()
+    return {"fwd." + nme: statistics.mean(ev[i].elapsed_time(ev[i + 1]) for ev in evs) for i, nme in enumerate(STAGES_F)}
+
+
+def run_moe(args, workload):
+    import torch
+    from paper_2403_07816_b200 import build as builder
+    world, rank, local = dist_setup(args)
+    if rank == 0:
+        builder.build()
+    barrier(world)
+    dev = torch.device("cuda", local)
+    peaks = load_peaks()
+    K, W = args.steps, max(args.warmup, 3)
+    soak_s = 0.0 if args.tokens or args.layers else SOAK_S        # profiler captures run few launches
+
+    run = MoeRun(workload, dev, rank, tokens=args.tokens, layers=args.layers)
+    ms, clocks, stages, soaked = time_moe(run, K, W, world, local, soak_s, with_stages=True)
+    if workload == "decode":
+        stages = decode_stage_times(run)
+    line = {"n_gpus": world, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic"}
+    line.update(moe_result(run, ms, clocks, stages, soaked, K, W, world, peaks, with_counts=False))
+    line["e2e"] = measure_e2e(run, world, E2E_STEPS) if (run.train and not args.no_e2e) else None
+
+    # ---- the other measured paths, one after the other (single GPU, default workload only) ----
+    solo = rank == 0 and world == 1 and not args.tokens and not args.layers
+    if solo and workload == "fwd_bwd" and not args.no_sub:
+        sub = {}
+        del run
+        free_device_memory()
+        for name in ("fwd", "switch_top1", "soft_all4", "top2_skewed", "decode"):
+            r = MoeRun(name, dev, rank)
+            k_sub = {"fwd": 200, "decode": 100}.get(name, 20)
+            s_ms, s_clocks, s_stages, s_soaked = time_moe(r, k_sub, 3, 1, local, 1.0 if name in ("fwd", "decode") else SOAK_S,
+                                                          with_stages=True)
+            if name == "decode":
+                s_stages = decode_stage_times(r)
+            sub[name] = moe_result(r, s_ms, s_clocks, s_stages, s_soaked, k_sub, 3, 1, peaks, with_counts=True)
+            del r
+            free_device_memory()
+        sub["merge"] = measure_merge(args, dev, local, 1, 20, 3, peaks)
+        free_device_memory()
+        line["sub"] = sub
 
     # ---- CPU oracle beside it (rank 0, single GPU only) ----
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and workload != "decode" and not args.tokens:
-        del sets
-        torch.cuda.empty_cache()
+    if solo and not args.no_cpu_baseline and workload != "decode":
+        free_device_memory()
         n_tok = 4096                           # about 10-30 s of host work
         fn, n = oracle_step_fn(workload, n_tok, device="cpu")
         t0 = time.perf_counter(); fn(); dt = time.perf_counter() - t0
         line["cpu_baseline"] = {"value": n / dt, "unit": "tokens/s", "cores": host_cores(), "kind": "oracle",
-                                "sample": f"first {n} of {T} tokens, full expert weights, one pass ({dt:.1f} s)"}
+                                "sample": f"first {n} of {WORKLOADS[workload][0]} tokens, full expert weights, one pass "
+                                          f"({dt:.1f} s)"}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -415,17 +564,11 @@ def run_moe(args, workload):
         dist.destroy_process_group()
 
 
-def run_merge(args):
+def measure_merge(args, dev, local, world, K, W, peaks):
     """btx_merge of four Llama-2-7B-shaped parameter sets, as many layers as fit (--merge-layers)."""
     import torch
-    from paper_2403_07816_b200 import binding as B, build as builder, synth
-    world, rank, local = dist_setup(args)
-    if rank == 0:
-        builder.build()
-    barrier(world)
-    dev = torch.device("cuda", local)
-    peaks = load_peaks()
-    n_models, d, F, vocab = 4, 4096, 11008, 32000
+    from paper_2403_07816_b200 import binding as B, synth
+    n_models, d, F, vocab = 4, D_MODEL, D_FF, 32000
     layers = args.merge_layers
     free, _ = torch.cuda.mem_get_info(dev)
     per_layer = (4 * d * d + 2 * d + 3 * d * F) * 2
@@ -462,7 +605,6 @@ def run_merge(args):
     ws = torch.empty(B.btx_merge_workspace_size(n_models, len(shapes)), dtype=torch.uint8, device=dev)
     read = sum(models[0][n].numel() for n, _ in shapes) * 2 * n_models
     written = sum(t.numel() for t in outputs.values()) * 2
-    K, W = args.steps, max(args.warmup, 3)
     for _ in range(W):
         B.btx_merge(models, outputs, ws)
     sampler = ClockSampler(local)
@@ -477,17 +619,32 @@ def run_merge(args):
     clocks = sampler.stop()
     ms = max_over_ranks(e0.elapsed_time(e1) / K, world, dev)
     gbs = (read + written) / (ms * 1e-3) / 1e9
-    line = {"metric": "btx_merge_GBps", "value": gbs * world, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-            "data": "synthetic", "clocks": clocks, "gpu_launches": K,
+    return {"metric": "btx_merge_GBps", "value": gbs * world, "unit": "GB/s", "steps": K, "warmup": W,
+            "ms_per_step": ms, "clocks": clocks, "gpu_launches": K,
             "config": {"workload": f"merge: 4 Llama-2-7B-shaped parameter sets, {layers} of 32 layers + embeddings/head "
                                    f"({read / 1e9:.1f} GB read, {written / 1e9:.1f} GB written per step, far beyond L2)"},
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["_source"],
-                         "kernel": "merge_kernel"},
-            "e2e": None}
+                         "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0, "traffic": None,
+                         "peak_source": peaks["_source"], "kernel": "merge_kernel"}}
+
+
+def run_merge(args):
+    import torch
+    from paper_2403_07816_b200 import build as builder
+    world, rank, local = dist_setup(args)
+    if rank == 0:
+        builder.build()
+    barrier(world)
+    dev = torch.device("cuda", local)
+    res = measure_merge(args, dev, local, world, args.steps, max(args.warmup, 3), load_peaks())
+    line = {"n_gpus": world, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "e2e": None}
+    line.update(res)
     if rank == 0:
         print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
 
 
 def main():
@@ -496,15 +653,16 @@ def main():
     ap.add_argument("--steps", type=int, default=0, help="timed steps (default 20; 100 for the short decode and merge steps)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="btx", choices=["btx", "reference"])
-    ap.add_argument("--workload", default="fwd_bwd", choices=["fwd_bwd", "fwd", "decode", "merge"])
+    ap.add_argument("--workload", default="fwd_bwd", choices=list(WORKLOADS) + ["merge"])
     ap.add_argument("--merge-layers", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sub", action="store_true", help="headline only: skip the other configurations")
     ap.add_argument("--layers", type=int, default=0, help="decode: number of layers (profiling only)")
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling only; not a bench number)")
     args = ap.parse_args()
     if args.steps <= 0:     # steps of a few ms need more repetitions for the clock sampler to see the timed region
-        short = {"decode": 100, "merge": 100, "fwd": 800}
+        short = {"decode": 100, "merge": 20, "fwd": 200}
         args.steps = short.get(args.workload, 20) if args.impl != "reference" else 20
     if args.impl == "reference":
         run_reference(args)

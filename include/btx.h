@@ -5,7 +5,11 @@
  * General conventions
  *   - Every tensor argument is a DEVICE pointer to caller-owned, row-major, contiguous memory,
  *     16-byte aligned, unless its description says "host".  The library never allocates or
- *     frees device memory and keeps no pointer after a call returns.
+ *     frees device memory and keeps no pointer after a call returns.  What it does keep, per
+ *     process: one helper stream per device (btx_moe_backward), the multiprocessor count per
+ *     device, the address of one static scratch array per device (btx_lb_loss_noalloc), and the
+ *     calling thread's stage-timing hook (btx_set_stage_events).
+ *   - The current device must be the one the buffers and `stream` belong to.
  *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and return without
  *     synchronising; arguments are validated on the host before anything is launched.
  *   - Element type of x, weights, y, dy, dx is given by btx_moe_desc.dtype (BTX_F32: float,
@@ -17,7 +21,7 @@
  *   - Errors: a btx_status is returned; nothing is launched when it is not BTX_OK.  Device-side
  *     bounded waits that expire are recorded in the workspace and read with btx_device_status.
  *
- * Notation: T tokens, d = d_model, F = d_ff, E experts, k selected experts per token
+ * Notation: T tokens, d = d_model, F = d_ff, E experts (at most 64), k selected experts per token
  * (k = E under BTX_ROUTE_SOFT), R = T*k assignments.
  */
 #ifndef BTX_H_
@@ -113,7 +117,9 @@ btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, const void* 
  * Sections 1 and 3.2; the loss is added to the training loss with weight 1, Section 3.3).
  * `saved` is the buffer the forward call filled with the same desc and inputs.
  * Outputs: dx[T,d] (dtype); dw_router[E,d], dbias[E] (may be NULL), dw1,dw3[E,F,d], dw2[E,d,F],
- * all fp32.  accumulate = 0 overwrites the weight gradients, 1 adds to them.  With desc.skip_wgrad
+ * all fp32; dlogits[T,E] fp32 (may be NULL): the gradient with respect to the router logits W_l x that
+ * dw_router, dbias and the router's share of dx are formed from (never accumulated into).
+ * accumulate = 0 overwrites the weight gradients, 1 adds to them.  With desc.skip_wgrad
  * the three expert gradients are not computed and dw1, dw3, dw2 may be NULL.
  * The memory-bound router kernels run beside the weight-gradient GEMMs on a helper stream that the
  * library creates once per device (the only CUDA resource it keeps) and that is joined back into
@@ -122,7 +128,7 @@ btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, const void*
                             const float* router_bias, const float* router_noise,
                             const void* w1, const void* w3, const void* w2,
                             const void* dy, float lb_grad_scale, const void* saved,
-                            void* dx, float* dw_router, float* dbias,
+                            void* dx, float* dw_router, float* dbias, float* dlogits,
                             float* dw1, float* dw3, float* dw2, int32_t accumulate,
                             void* workspace, size_t workspace_bytes, void* stream);
 
@@ -145,12 +151,13 @@ btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_host, const
                              void* stream, void* copy_stream);
 
 /* L_LB = alpha * E * sum_i u_i p_i with u_i the batch mean of the gate of expert i and p_i the
- * batch mean of SoftMax_i (Section 3.3), from given fp32 logits[T,E] (bias, if any, already
- * added).  Outputs loss[1], u[E], p[E]; dlogits[T,E] (d loss / d logits) unless NULL.
- * Uses desc.T, E, k, routing, lb_alpha, lb_stopgrad_u.  Workspace: btx_lb_loss_workspace_size. */
+ * batch mean of SoftMax_i (Section 3.3), from given fp32 logits[T,E]; router_bias[E] fp32 is added
+ * to every row first (NULL: none, as in the paper).  Outputs loss[1], u[E], p[E]; dlogits[T,E]
+ * (d loss / d logits) unless NULL.  Uses desc.T, E, k, routing (not SAMPLE1), lb_alpha,
+ * lb_stopgrad_u.  Workspace: btx_lb_loss_workspace_size. */
 btx_status btx_lb_loss_workspace_size(const btx_moe_desc* desc, size_t* workspace_bytes);
-btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits, float* loss, float* u, float* p,
-                       float* dlogits, void* workspace, size_t workspace_bytes, void* stream);
+btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits, const float* router_bias, float* loss,
+                       float* u, float* p, float* dlogits, void* workspace, size_t workspace_bytes, void* stream);
 
 /* btx_lb_loss without a caller-supplied workspace (the paper has no counterpart; this is a
  * packaging variant of the call above).  It is meant for callers that hold no allocator: plug-in
@@ -159,24 +166,29 @@ btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits, float* los
  * scratch lives in a 4 MiB (BTX_LB_NOALLOC_SCRATCH_BYTES) static device array inside the library,
  * which every GPU that loads the library holds until the process exits.  Same arguments and
  * results as btx_lb_loss; inputs and outputs are still the caller's.
- *   - Requests whose btx_lb_loss_workspace_size exceeds the array return BTX_ERR_WORKSPACE and
- *     launch nothing (4 MiB covers e.g. T = 32768 tokens with E = 4).
+ *   - A request is refused with BTX_ERR_WORKSPACE, before anything is enqueued, exactly when
+ *     btx_lb_loss_workspace_size(desc) exceeds the array (4 MiB covers e.g. T = 32768 tokens with
+ *     E = 4, top-2, which needs 3.05 MiB).
  *   - The first call on each device looks up the array's device address (once per device, with that
  *     device current); make that first call before starting any stream capture.
  *   - The call allocates and frees nothing.  All calls on one device share the array, which keeps
  *     whatever the previous call left in it (the call itself clears the part that must start at
  *     zero): two calls whose kernels may overlap on the GPU, e.g. on different streams, race. */
 #define BTX_LB_NOALLOC_SCRATCH_BYTES (4u << 20)
-btx_status btx_lb_loss_noalloc(const btx_moe_desc* desc, const float* logits, float* loss, float* u, float* p,
-                               float* dlogits, void* stream);
+btx_status btx_lb_loss_noalloc(const btx_moe_desc* desc, const float* logits, const float* router_bias, float* loss,
+                               float* u, float* p, float* dlogits, void* stream);
 
 /* MiX merge (Section 3.2): the feed-forward matrices of the N expert LLMs become the experts of
  * one MoE layer (kind FFN: dst[e*numel .. ] = src[e], bit for bit); every other parameter is the
  * uniform mean over the N models (kind AVERAGE: fp32 sum in model order, divided by N, rounded
  * once to dtype).  `items` is a HOST array; each item's `src` is a HOST array of N device
  * pointers.  Sources and destinations must not overlap.  numel*sizeof(element) need not be a
- * multiple of 16 for AVERAGE items; the pointers must be 16-byte aligned. */
-typedef enum { BTX_PARAM_AVERAGE = 0, BTX_PARAM_FFN = 1 } btx_param_kind;
+ * multiple of 16 for AVERAGE items; the pointers must be 16-byte aligned.  The three FFN_W* kinds
+ * name which matrix an item is and are all stacked like BTX_PARAM_FFN.
+ * The item table is staged through pageable host memory inside the call: the call blocks the host
+ * for that copy and must not be recorded into a CUDA graph. */
+typedef enum { BTX_PARAM_AVERAGE = 0, BTX_PARAM_FFN = 1, BTX_PARAM_FFN_W1 = 1, BTX_PARAM_FFN_W3 = 2,
+               BTX_PARAM_FFN_W2 = 3 } btx_param_kind;
 typedef struct {
   int32_t kind;               /* btx_param_kind */
   int32_t layer;              /* informational  */

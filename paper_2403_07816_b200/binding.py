@@ -63,13 +63,13 @@ def lib():
         L.btx_moe_forward.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, vp, C.POINTER(RoutingOut), vp, vp,
                                       sz, vp]
         L.btx_moe_backward.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp, vp,
-                                       vp, i32, vp, sz, vp]
+                                       vp, vp, i32, vp, sz, vp]
         L.btx_moe_step_host.argtypes = [C.POINTER(MoeDesc)] + [vp] * 15 + [f32] + [vp] * 5 + [i32, vp, vp, sz, vp, vp]
         L.btx_set_stage_events.argtypes = [C.POINTER(vp), i32]
         L.btx_selftest_wait_expiry.argtypes = [vp, sz, vp]
         L.btx_lb_loss_workspace_size.argtypes = [C.POINTER(MoeDesc), C.POINTER(sz)]
-        L.btx_lb_loss.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, sz, vp]
-        L.btx_lb_loss_noalloc.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp]
+        L.btx_lb_loss.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.btx_lb_loss_noalloc.argtypes = [C.POINTER(MoeDesc), vp, vp, vp, vp, vp, vp, vp]
         L.btx_merge_workspace_size.argtypes = [i32, C.c_uint64, C.POINTER(sz)]
         L.btx_merge.argtypes = [i32, i32, C.POINTER(MergeItem), C.c_uint64, vp, sz, vp]
         L.btx_merge_ffn_workspace_size.argtypes = [i32, i32, C.POINTER(sz)]
@@ -106,6 +106,14 @@ def _ptr(t):
 
 def _stream(device):
     return C.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def _on(device):
+    """The library works on the current device (its helper stream, multiprocessor count and static scratch
+    are looked up per current device): every call runs with the tensors' device made current."""
+    if torch.device(device).type != "cuda":
+        raise RuntimeError("btx: tensors must live on a CUDA device (there is no CPU path)")
+    return torch.cuda.device(device)
 
 
 def make_desc(T, d_model, d_ff, E, k, dtype, routing=ROUTE_TOPK, lb_alpha=0.01, lb_stopgrad_u=False,
@@ -162,21 +170,23 @@ def alloc_buffers(desc: MoeDesc, device):
 
 def btx_moe_forward(desc, x, w_router, router_bias, w1, w3, w2, y, routing, saved, workspace, router_noise=None):
     ro = routing.as_struct() if routing is not None else None
-    s = lib().btx_moe_forward(C.byref(desc), _ptr(x), _ptr(w_router), _ptr(router_bias), _ptr(router_noise), _ptr(w1),
-                              _ptr(w3), _ptr(w2),
-                              _ptr(y), C.byref(ro) if ro is not None else None, _ptr(saved), _ptr(workspace),
-                              workspace.numel(), _stream(x.device))
+    with _on(x.device):
+        s = lib().btx_moe_forward(C.byref(desc), _ptr(x), _ptr(w_router), _ptr(router_bias), _ptr(router_noise),
+                                  _ptr(w1), _ptr(w3), _ptr(w2),
+                                  _ptr(y), C.byref(ro) if ro is not None else None, _ptr(saved), _ptr(workspace),
+                                  workspace.numel(), _stream(x.device))
     if s != BTX_OK:
         raise BtxError(s, "btx_moe_forward")
 
 
 def btx_moe_backward(desc, x, w_router, router_bias, w1, w3, w2, dy, lb_grad_scale, saved, dx, dw_router, dbias,
-                     dw1, dw3, dw2, accumulate, workspace, router_noise=None):
-    s = lib().btx_moe_backward(C.byref(desc), _ptr(x), _ptr(w_router), _ptr(router_bias), _ptr(router_noise), _ptr(w1),
-                               _ptr(w3), _ptr(w2),
-                               _ptr(dy), float(lb_grad_scale), _ptr(saved), _ptr(dx), _ptr(dw_router), _ptr(dbias),
-                               _ptr(dw1), _ptr(dw3), _ptr(dw2), int(accumulate), _ptr(workspace), workspace.numel(),
-                               _stream(x.device))
+                     dw1, dw3, dw2, accumulate, workspace, router_noise=None, dlogits=None):
+    with _on(x.device):
+        s = lib().btx_moe_backward(C.byref(desc), _ptr(x), _ptr(w_router), _ptr(router_bias), _ptr(router_noise),
+                                   _ptr(w1), _ptr(w3), _ptr(w2),
+                                   _ptr(dy), float(lb_grad_scale), _ptr(saved), _ptr(dx), _ptr(dw_router), _ptr(dbias),
+                                   _ptr(dlogits), _ptr(dw1), _ptr(dw3), _ptr(dw2), int(accumulate), _ptr(workspace),
+                                   workspace.numel(), _stream(x.device))
     if s != BTX_OK:
         raise BtxError(s, "btx_moe_backward")
 
@@ -190,13 +200,14 @@ def btx_moe_step_host(desc, x_host, dy_host, y_host, dx_host, loss_host, x_dev, 
         if t.is_cuda or not t.is_contiguous():
             raise RuntimeError("btx_moe_step_host: host tensors must be contiguous CPU tensors")
     hp = lambda t: C.c_void_p(t.data_ptr())
-    s = lib().btx_moe_step_host(C.byref(desc), hp(x_host), hp(dy_host), hp(y_host), hp(dx_host), hp(loss_host),
-                                _ptr(x_dev), _ptr(dy_dev), _ptr(y_dev), _ptr(dx_dev), _ptr(w_router),
-                                _ptr(router_bias), _ptr(router_noise), _ptr(w1), _ptr(w3), _ptr(w2),
-                                float(lb_grad_scale),
-                                _ptr(dw_router), _ptr(dbias), _ptr(dw1), _ptr(dw3), _ptr(dw2), int(accumulate),
-                                _ptr(saved), _ptr(workspace), workspace.numel(), _stream(x_dev.device),
-                                C.c_void_p(copy_stream.cuda_stream) if copy_stream is not None else None)
+    with _on(x_dev.device):
+        s = lib().btx_moe_step_host(C.byref(desc), hp(x_host), hp(dy_host), hp(y_host), hp(dx_host), hp(loss_host),
+                                    _ptr(x_dev), _ptr(dy_dev), _ptr(y_dev), _ptr(dx_dev), _ptr(w_router),
+                                    _ptr(router_bias), _ptr(router_noise), _ptr(w1), _ptr(w3), _ptr(w2),
+                                    float(lb_grad_scale),
+                                    _ptr(dw_router), _ptr(dbias), _ptr(dw1), _ptr(dw3), _ptr(dw2), int(accumulate),
+                                    _ptr(saved), _ptr(workspace), workspace.numel(), _stream(x_dev.device),
+                                    C.c_void_p(copy_stream.cuda_stream) if copy_stream is not None else None)
     if s != BTX_OK:
         raise BtxError(s, "btx_moe_step_host")
 
@@ -227,17 +238,19 @@ def btx_lb_loss_workspace_size(desc):
     return sz.value
 
 
-def btx_lb_loss(desc, logits, loss, u, p, dlogits, workspace):
-    s = lib().btx_lb_loss(C.byref(desc), _ptr(logits), _ptr(loss), _ptr(u), _ptr(p), _ptr(dlogits), _ptr(workspace),
-                          workspace.numel(), _stream(logits.device))
+def btx_lb_loss(desc, logits, loss, u, p, dlogits, workspace, router_bias=None):
+    with _on(logits.device):
+        s = lib().btx_lb_loss(C.byref(desc), _ptr(logits), _ptr(router_bias), _ptr(loss), _ptr(u), _ptr(p),
+                              _ptr(dlogits), _ptr(workspace), workspace.numel(), _stream(logits.device))
     if s != BTX_OK:
         raise BtxError(s, "btx_lb_loss")
 
 
-def btx_lb_loss_noalloc(desc, logits, loss, u, p, dlogits):
+def btx_lb_loss_noalloc(desc, logits, loss, u, p, dlogits, router_bias=None):
     """btx_lb_loss on the library's own static scratch: no workspace argument, nothing allocated."""
-    s = lib().btx_lb_loss_noalloc(C.byref(desc), _ptr(logits), _ptr(loss), _ptr(u), _ptr(p), _ptr(dlogits),
-                                  _stream(logits.device))
+    with _on(logits.device):
+        s = lib().btx_lb_loss_noalloc(C.byref(desc), _ptr(logits), _ptr(router_bias), _ptr(loss), _ptr(u), _ptr(p),
+                                      _ptr(dlogits), _stream(logits.device))
     if s != BTX_OK:
         raise BtxError(s, "btx_lb_loss_noalloc")
 
@@ -272,7 +285,9 @@ def btx_merge(models, outputs, workspace=None):
     device = models[0][names[0]].device
     if workspace is None:
         workspace = torch.empty(btx_merge_workspace_size(n, len(names)), dtype=torch.uint8, device=device)
-    s = lib().btx_merge(n, _dtype_code(dtype), items, len(names), _ptr(workspace), workspace.numel(), _stream(device))
+    with _on(device):
+        s = lib().btx_merge(n, _dtype_code(dtype), items, len(names), _ptr(workspace), workspace.numel(),
+                            _stream(device))
     if s != BTX_OK:
         raise BtxError(s, "btx_merge")
     return workspace
@@ -292,8 +307,9 @@ def btx_merge_ffn(w1s, w3s, w2s, layout, chunks, w1_dst, w3_dst, w2_dst, workspa
         if s != BTX_OK:
             raise BtxError(s, "btx_merge_ffn_workspace_size")
         workspace = torch.empty(sz.value, dtype=torch.uint8, device=device)
-    s = lib().btx_merge_ffn(n, _dtype_code(w1s[0].dtype), layout, chunks, d, F, a1, a3, a2, _ptr(w1_dst), _ptr(w3_dst),
-                            _ptr(w2_dst), _ptr(workspace), workspace.numel(), _stream(device))
+    with _on(device):
+        s = lib().btx_merge_ffn(n, _dtype_code(w1s[0].dtype), layout, chunks, d, F, a1, a3, a2, _ptr(w1_dst),
+                                _ptr(w3_dst), _ptr(w2_dst), _ptr(workspace), workspace.numel(), _stream(device))
     if s != BTX_OK:
         raise BtxError(s, "btx_merge_ffn")
     return workspace
@@ -301,15 +317,17 @@ def btx_merge_ffn(w1s, w3s, w2s, layout, chunks, w1_dst, w3_dst, w2_dst, workspa
 
 def btx_selftest_wait_expiry(workspace):
     """Makes one bounded device-side wait run out on purpose; see btx.h."""
-    s = lib().btx_selftest_wait_expiry(_ptr(workspace), workspace.numel() * workspace.element_size(),
-                                       _stream(workspace.device))
+    with _on(workspace.device):
+        s = lib().btx_selftest_wait_expiry(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                           _stream(workspace.device))
     if s != BTX_OK:
         raise BtxError(s, "btx_selftest_wait_expiry")
 
 
 def btx_device_status(workspace):
     st = C.c_int32(0)
-    s = lib().btx_device_status(_ptr(workspace), _stream(workspace.device), C.byref(st))
+    with _on(workspace.device):
+        s = lib().btx_device_status(_ptr(workspace), _stream(workspace.device), C.byref(st))
     if s != BTX_OK:
         raise BtxError(s, "btx_device_status")
     return st.value

@@ -44,7 +44,7 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   p.mt_max = p.r_pad_max / kRowTile;
   p.nt_dact = desc->dtype == BTX_BF16 ? 2 * ((p.F + 255) / 256) : (p.F + 63) / 64;   // row-dot partials per row
   p.route_blocks = (p.T + 7) / 8;
-  if (p.route_blocks > 148 * 8) p.route_blocks = 148 * 8;
+  if (p.route_blocks > kMaxRouteBlocks) p.route_blocks = kMaxRouteBlocks;
   p.perm_blocks = (p.R + 1023) / 1024;
   p.wr_chunks = (p.T + 127) / 128;
   // Small BF16 batches stream the expert weights through the swap-AB kernels (weights on the M side,
@@ -62,7 +62,7 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   const size_t rp = (size_t)p.r_pad_max;
   p.s_topk = take((size_t)p.R * 4);       p.s_gates = take((size_t)p.R * 4);
   p.s_probs = take((size_t)p.T * p.E * 4); p.s_logits = take((size_t)p.T * p.E * 4);
-  p.s_u = take(p.E * 4);  p.s_p = take(p.E * 4);  p.s_loss = take(4);
+  p.s_u = take(p.E * 4);  p.s_p = take(p.E * 4);  p.s_up64 = take(2 * p.E * 8);  p.s_loss = take(4);
   p.s_counts = take(p.E * 4);  p.s_offsets = take((p.E + 1) * 4);  p.s_pad_offsets = take((p.E + 1) * 4);
   p.s_tile_expert = take((size_t)p.mt_max * 4);
   p.s_rowmap = take(rp * 4);  p.s_flat2row = take((size_t)p.R * 4);
@@ -106,6 +106,7 @@ static void resolve(const Plan& p, char* saved, char* ws, Buffers* b) {
   b->topk = (int32_t*)(saved + p.s_topk);   b->gates = (float*)(saved + p.s_gates);
   b->probs = (float*)(saved + p.s_probs);   b->logits = (float*)(saved + p.s_logits);
   b->u = (float*)(saved + p.s_u);  b->p = (float*)(saved + p.s_p);  b->loss = (float*)(saved + p.s_loss);
+  b->up64 = (double*)(saved + p.s_up64);
   b->counts = (int32_t*)(saved + p.s_counts);  b->offsets = (int32_t*)(saved + p.s_offsets);
   b->pad_offsets = (int32_t*)(saved + p.s_pad_offsets);  b->tile_expert = (int32_t*)(saved + p.s_tile_expert);
   b->rowmap = (int32_t*)(saved + p.s_rowmap);  b->flat2row = (int32_t*)(saved + p.s_flat2row);
@@ -168,6 +169,30 @@ struct ScopedEvents {                   // destroyed on every return path; destr
   }
   ~ScopedEvents() { for (cudaEvent_t x : e) if (x) cudaEventDestroy(x); }
 };
+
+}  // namespace btx
+
+int btx::sm_count() {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static int count[kMaxDevices] = {};
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return 148;                        // no usable device (size queries on a host without a GPU)
+  }
+  std::lock_guard<std::mutex> lock(mu);
+  if (count[dev] == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      return 148;
+    }
+    count[dev] = n;
+  }
+  return count[dev];
+}
+
+namespace btx {
 
 static btx_status check_device() {
   int dev = 0;
@@ -267,8 +292,9 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
                                        const float* router_bias, const float* router_noise, const void* w1,
                                        const void* w3, const void* w2,
                                        const void* dy, float lb_grad_scale, const void* saved, void* dx,
-                                       float* dw_router, float* dbias, float* dw1, float* dw3, float* dw2,
-                                       int32_t accumulate, void* workspace, size_t workspace_bytes, void* stream) {
+                                       float* dw_router, float* dbias, float* dlogits, float* dw1, float* dw3,
+                                       float* dw2, int32_t accumulate, void* workspace, size_t workspace_bytes,
+                                       void* stream) {
   (void)router_bias;   // the bias only shifts the logits; its gradient needs dz alone
   (void)router_noise;  // likewise: the forward saved the perturbed probabilities
   Plan pl;
@@ -279,7 +305,8 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
     return BTX_ERR_INVALID_ARG;
   if (!skip_wgrad && (!dw1 || !dw3 || !dw2)) return BTX_ERR_INVALID_ARG;
   if (misaligned(x) || misaligned(w_router) || misaligned(w1) || misaligned(w3) || misaligned(w2) ||
-      misaligned(dy) || misaligned(saved) || misaligned(dx) || misaligned(dw_router) || misaligned(dw1) ||
+      misaligned(dy) || misaligned(saved) || misaligned(dx) || misaligned(dw_router) || misaligned(dlogits) ||
+      misaligned(dw1) ||
       misaligned(dw3) || misaligned(dw2) || misaligned(workspace))
     return BTX_ERR_INVALID_ARG;
   if (workspace_bytes < pl.workspace_bytes) return BTX_ERR_WORKSPACE;
@@ -309,8 +336,8 @@ extern "C" btx_status btx_moe_backward(const btx_moe_desc* desc, const void* x, 
   cudaStream_t rst = side != nullptr ? side : st;
   if (side != nullptr) BTX_CUDA_OK(cudaStreamWaitEvent(side, after_dx, 0));
   BTX_CUDA_OK(launch_router_backward(pl, desc->dtype, er.routing, desc->lb_alpha, lb_grad_scale,
-                                     desc->lb_stopgrad_u, 1, x, w_router, b, dx, dw_router, dbias, nullptr,
-                                     accumulate, er.inv_tau, rst));
+                                     desc->lb_stopgrad_u, 1, x, w_router, b, dx, dw_router, dbias, dlogits,
+                                     accumulate, er.inv_tau, desc->routing == BTX_ROUTE_SAMPLE1, rst));
   if (side != nullptr) {
     BTX_CUDA_OK(cudaEventRecord(evs.e[1], side));
     BTX_CUDA_OK(cudaStreamWaitEvent(st, evs.e[1], 0));
@@ -364,7 +391,8 @@ extern "C" btx_status btx_moe_step_host(const btx_moe_desc* desc, const void* x_
     BTX_CUDA_OK(cudaStreamWaitEvent(st, ev_dy, 0));
   }
   if ((s = btx_moe_backward(desc, x_dev, w_router, router_bias, router_noise, w1, w3, w2, dy_dev, lb_grad_scale, saved,
-                            dx_dev, dw_router, dbias, dw1, dw3, dw2, accumulate, workspace, workspace_bytes, stream)) !=
+                            dx_dev, dw_router, dbias, nullptr, dw1, dw3, dw2, accumulate, workspace, workspace_bytes,
+                            stream)) !=
       BTX_OK)
     return s;
   if (!overlap) BTX_CUDA_OK(cudaMemcpyAsync(y_host, y_dev, act_bytes, cudaMemcpyDeviceToHost, st));
@@ -392,28 +420,39 @@ extern "C" btx_status btx_lb_loss_workspace_size(const btx_moe_desc* desc, size_
   return BTX_OK;
 }
 
-extern "C" btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits, float* loss, float* u, float* p,
-                                  float* dlogits, void* workspace, size_t workspace_bytes, void* stream) {
-  Plan pl;
-  btx_status s = make_plan(desc, &pl, true);
+// Host-side checks shared by the two loss entry points (everything except the workspace).
+static btx_status lb_loss_validate(const btx_moe_desc* desc, const float* logits, float* loss, float* u, float* p,
+                                   Plan* pl) {
+  btx_status s = make_plan(desc, pl, true);
   if (s != BTX_OK) return s;
-  if (!logits || !loss || !u || !p || !workspace) return BTX_ERR_INVALID_ARG;
-  if (misaligned(workspace)) return BTX_ERR_INVALID_ARG;
+  if (desc->routing == BTX_ROUTE_SAMPLE1) return BTX_ERR_UNSUPPORTED;
+  if (!logits || !loss || !u || !p) return BTX_ERR_INVALID_ARG;
+  return BTX_OK;
+}
+
+extern "C" btx_status btx_lb_loss(const btx_moe_desc* desc, const float* logits, const float* router_bias, float* loss,
+                                  float* u, float* p, float* dlogits, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+  // every check comes before the first enqueue: a refused call leaves the stream and the workspace alone
+  Plan pl;
+  btx_status s = lb_loss_validate(desc, logits, loss, u, p, &pl);
+  if (s != BTX_OK) return s;
+  if (!workspace || misaligned(workspace)) return BTX_ERR_INVALID_ARG;
   if (workspace_bytes < pl.workspace_bytes) return BTX_ERR_WORKSPACE;
+  if ((s = check_device()) != BTX_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
   char* ws = (char*)workspace;
   Buffers b;
   resolve(pl, ws + pl.w_saved_fallback, ws, &b);
   BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
-  if (desc->routing == BTX_ROUTE_SAMPLE1) return BTX_ERR_UNSUPPORTED;
-  BTX_CUDA_OK(launch_router(pl, BTX_F32, desc->routing, desc->lb_alpha, nullptr, nullptr, nullptr, logits, nullptr, 1.0f,
-                            b, st));
+  BTX_CUDA_OK(launch_router(pl, BTX_F32, desc->routing, desc->lb_alpha, nullptr, nullptr, router_bias, logits, nullptr,
+                            1.0f, b, st));
   BTX_CUDA_OK(cudaMemcpyAsync(loss, b.loss, 4, cudaMemcpyDeviceToDevice, st));
   BTX_CUDA_OK(cudaMemcpyAsync(u, b.u, pl.E * 4, cudaMemcpyDeviceToDevice, st));
   BTX_CUDA_OK(cudaMemcpyAsync(p, b.p, pl.E * 4, cudaMemcpyDeviceToDevice, st));
   if (dlogits) {
     BTX_CUDA_OK(launch_router_backward(pl, BTX_F32, desc->routing, desc->lb_alpha, 1.0f, desc->lb_stopgrad_u, 0,
-                                       nullptr, nullptr, b, nullptr, nullptr, nullptr, dlogits, 0, 1.0f, st));
+                                       nullptr, nullptr, b, nullptr, nullptr, nullptr, dlogits, 0, 1.0f, 0, st));
   }
   return BTX_OK;
 }
@@ -439,17 +478,17 @@ static btx_status lb_noalloc_scratch(void** out) {
   return BTX_OK;
 }
 
-extern "C" btx_status btx_lb_loss_noalloc(const btx_moe_desc* desc, const float* logits, float* loss, float* u,
-                                          float* p, float* dlogits, void* stream) {
-  size_t need = 0;
-  btx_status s = btx_lb_loss_workspace_size(desc, &need);
+extern "C" btx_status btx_lb_loss_noalloc(const btx_moe_desc* desc, const float* logits, const float* router_bias,
+                                          float* loss, float* u, float* p, float* dlogits, void* stream) {
+  Plan pl;
+  btx_status s = lb_loss_validate(desc, logits, loss, u, p, &pl);
   if (s != BTX_OK) return s;
-  if (need > (size_t)BTX_LB_NOALLOC_SCRATCH_BYTES) return BTX_ERR_WORKSPACE;   // beyond the static array
+  if (pl.workspace_bytes > (size_t)BTX_LB_NOALLOC_SCRATCH_BYTES) return BTX_ERR_WORKSPACE;   // beyond the static array
   void* scratch = nullptr;
   if ((s = lb_noalloc_scratch(&scratch)) != BTX_OK) return s;
   // btx_lb_loss clears the status block at the head of the scratch and overwrites every other
   // region before reading it, so stale contents of an earlier call are harmless.
-  return btx_lb_loss(desc, logits, loss, u, p, dlogits, scratch, BTX_LB_NOALLOC_SCRATCH_BYTES, stream);
+  return btx_lb_loss(desc, logits, router_bias, loss, u, p, dlogits, scratch, BTX_LB_NOALLOC_SCRATCH_BYTES, stream);
 }
 
 extern "C" btx_status btx_device_status(const void* workspace, void* stream, int32_t* device_status) {

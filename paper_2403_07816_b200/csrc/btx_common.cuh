@@ -11,7 +11,8 @@
 namespace btx {
 
 constexpr int kRowTile = 256;        // expert segments of the sorted buffers are padded to this many rows
-constexpr int kMaxExperts = 32;
+constexpr int kMaxExperts = 64;
+constexpr int kMaxRouteBlocks = 1184; // bound of the router kernel's grid (sizes its partial-sum buffer)
 constexpr int kStatusWords = 64;     // first 256 bytes of every workspace: device status block
                                      // (word 0: error code; word 8: ticket of the one-launch routing;
 constexpr int kTileCounterWord = 16; //  words 16..23: tile counters of a call's tensor-core launches)
@@ -22,8 +23,8 @@ constexpr int kTileCounterWord = 16; //  words 16..23: tile counters of a call's
 struct Plan {
   int T, d, F, E, k, R;              // k = effective number of selected experts
   int esize;                         // bytes per element of dtype
-  int r_pad_max;                     // upper bound of the padded sorted row count (multiple of 128)
-  int mt_max;                        // r_pad_max / 128
+  int r_pad_max;                     // upper bound of the padded sorted row count (multiple of kRowTile)
+  int mt_max;                        // r_pad_max / kRowTile
   int nt_dact;                       // column tiles of the dgrad-2 GEMM (row-dot partials)
   int route_blocks;                  // blocks of the router kernel (partial sums for u, p)
   int perm_blocks;                   // blocks of the permutation kernels
@@ -33,7 +34,7 @@ struct Plan {
   int capacity;                      // rows one expert accepts (R when there is no limit)
   int capped;                        // a capacity limit is set: assignments may be dropped
   // saved
-  size_t s_topk, s_gates, s_probs, s_logits, s_u, s_p, s_loss, s_counts, s_offsets, s_pad_offsets,
+  size_t s_topk, s_gates, s_probs, s_logits, s_u, s_p, s_up64, s_loss, s_counts, s_offsets, s_pad_offsets,
       s_tile_expert, s_rowmap, s_flat2row, s_perm, s_inv_perm, s_xs, s_h1, s_h3, saved_bytes;
   // workspace
   size_t w_status, w_route_part, w_perm_counts, w_perm_base, w_act, w_yp, w_dys, w_dh1, w_dh3, w_ga,
@@ -47,6 +48,7 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* plan, bool routing_only);
 struct Buffers {
   int32_t* topk;      float* gates;   float* probs;   float* logits;
   float* u;           float* p;       float* loss;
+  double* up64;       // the batch means u[E] then p[E] as computed (double), for the backward
   int32_t* counts;    int32_t* offsets;   int32_t* pad_offsets;   int32_t* tile_expert;
   int32_t* rowmap;    // padded sorted row -> flat assignment id (t*k+slot), -1 for padding rows
   int32_t* flat2row;  // flat assignment id -> padded sorted row (-1: dropped by the capacity limit)
@@ -60,6 +62,9 @@ struct Buffers {
 
 // Records stage event i of the calling thread's timing hook (no-op when the hook is off).
 void mark_stage(int i, cudaStream_t st);
+
+// Multiprocessor count of the current device (looked up once per device).
+int sm_count();
 
 // ---------------------------------------------------------------------------------------------
 // Launchers (defined in the .cu files).
@@ -83,7 +88,7 @@ cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int spl
 cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float alpha, float lb_scale,
                                    int stopgrad_u, int have_dg, const void* x, const void* w_router, const Buffers& b,
                                    void* dx, float* dw_router, float* dbias, float* dlogits_out, int accumulate,
-                                   float dz_scale, cudaStream_t st);
+                                   float dz_scale, int perturbed, cudaStream_t st);
 
 // Expert GEMMs: SIMT fp32 kernels for BTX_F32, tcgen05 kernels for BTX_BF16.
 cudaError_t launch_expert_forward_f32(const Plan& pl, const void* w1, const void* w3, const void* w2,

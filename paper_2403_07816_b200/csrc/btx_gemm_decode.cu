@@ -29,7 +29,7 @@ constexpr int DA_BYTES = WM * BK * 2;                    // weights per CTA and 
 constexpr int D_RING_BYTES = 192 * 1024;                 // stages = min(9, ring / (DA_BYTES + token box))
 constexpr int D_EPI_WARPS = 8;
 constexpr int D_THREADS = 64 + D_EPI_WARPS * 32;
-constexpr int D_MAX_CHUNKS = 64;                         // (1024 + 32 * 255) / 256 rounded up, with room
+constexpr int D_MAX_CHUNKS = 72;                         // row tiles that can hold tokens: at most R/256 + E = 4 + 64
 constexpr int D_SMEM_BYTES = D_RING_BYTES + 1024 + 256 + (D_MAX_CHUNKS + 2) * 4;
 
 struct SwapParams {
@@ -277,7 +277,7 @@ btx_status launch_swapk(const CUtensorMap& w0, const CUtensorMap& w1, const CUte
 // un-split round of 64 items on 74 pairs streams W2 as fast as 512 items in seven rounds did, and
 // fewer splits mean fewer partial products to write and to sum.
 int pick_decode_splits(int base_tiles, int kb_total) {
-  const int pairs = 74;                                   // 148 SMs; only a balance heuristic
+  const int pairs = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
   int best = 1;
   double best_eff = 0.0;
   for (int S = 1; S <= 8 && S <= kb_total; ++S) {

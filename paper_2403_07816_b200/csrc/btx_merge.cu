@@ -187,16 +187,15 @@ static btx_status launch_merge_items(std::vector<DevItem>& dev, std::vector<uint
   char* w = (char*)workspace + kStatusWords * 4;
   DevItem* d_items = (DevItem*)w;
   uint64_t* d_start = (uint64_t*)(w + dev.size() * sizeof(DevItem));
-  // pageable sources are staged before cudaMemcpyAsync returns, so the vectors may go out of scope
+  // The tables are pageable host memory: cudaMemcpyAsync stages them before it returns (the vectors may
+  // then go out of scope), which also means that these two copies block the host for a moment and that a
+  // merge call must not be recorded into a CUDA graph (a replay would read the freed vectors).
   if (cudaMemcpyAsync(d_items, dev.data(), dev.size() * sizeof(DevItem), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return BTX_ERR_CUDA;
   if (cudaMemcpyAsync(d_start, start.data(), start.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, st) !=
       cudaSuccess)
     return BTX_ERR_CUDA;
-  int sms = 148, dev_id = 0;
-  cudaGetDevice(&dev_id);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_id);
-  uint64_t grid = (uint64_t)sms * 8;
+  uint64_t grid = (uint64_t)sm_count() * 8;
   if (grid > total) grid = total;
   if (dtype == BTX_BF16)
     merge_kernel<__nv_bfloat16><<<(unsigned)grid, kMergeThreads, 0, st>>>(d_items, d_start, (int)dev.size(), total);
@@ -231,7 +230,7 @@ extern "C" btx_status btx_merge(int32_t n_models, int32_t dtype, const btx_merge
   for (uint64_t i = 0; i < n_items; ++i) {
     const btx_merge_item& it = items[i];
     if (!it.src || !it.dst || ((uintptr_t)it.dst & 15)) return BTX_ERR_INVALID_ARG;
-    if (it.kind != BTX_PARAM_AVERAGE && it.kind != BTX_PARAM_FFN) return BTX_ERR_INVALID_ARG;
+    if (it.kind < BTX_PARAM_AVERAGE || it.kind > BTX_PARAM_FFN_W2) return BTX_ERR_INVALID_ARG;
     for (int m = 0; m < n_models; ++m)
       if (!it.src[m] || ((uintptr_t)it.src[m] & 15)) return BTX_ERR_INVALID_ARG;
     if (it.numel == 0) continue;

@@ -6,7 +6,7 @@
 //               the batch means u and p of Section 3.3
 //   finalize    u, p, L_LB = alpha E sum_i u_i p_i
 //   permutation histogram -> exclusive scan -> stable scatter of the R assignments into
-//               (expert ascending, token ascending) order; expert segments padded to 128 rows
+//               (expert ascending, token ascending) order; expert segments padded to whole 256-row tiles
 //   gather      rows of x (or dy) copied into the padded expert-sorted layout
 //   combine     y_t = sum over slots of the gate-scaled expert rows
 //   router bwd  d logits from d gates and the two L_LB terms; dW_l = dz^T x; dx += W_l^T dz
@@ -46,12 +46,15 @@ template <> struct Vec<__nv_bfloat16> {
 // Router
 // ---------------------------------------------------------------------------------------------
 // Selection, gates and softmax for one token from the logits z[0..E) in shared memory (all lanes of
-// the calling warp take part).  On return lane e (< E) holds the dense gate and probability of expert e.
-__device__ __forceinline__ void route_select(int t, int E, int k, int routing, const float* z, int lane,
+// the calling warp take part).  The experts are chosen on z as it stands; the softmaxes are those of
+// z * scale (scale = 1 except for Sample Top-1, whose temperature must not touch the arg-max: a
+// rounded product could merge two distinct perturbed logits into a tie).  On return lane l holds the
+// dense gate and probability of experts l (index 0) and l + 32 (index 1).
+__device__ __forceinline__ void route_select(int t, int E, int k, int routing, float scale, const float* z, int lane,
                                              int32_t* __restrict__ topk,
-                                             float* __restrict__ gates, float* __restrict__ probs, float& my_g,
-                                             float& my_p) {
-  uint32_t taken = 0;
+                                             float* __restrict__ gates, float* __restrict__ probs, float (&my_g)[2],
+                                             float (&my_p)[2]) {
+  unsigned long long taken = 0;
   int sel[kMaxExperts];
   int first = 0;
   // repeated arg-max: strict '>' keeps the lower index on ties
@@ -59,50 +62,56 @@ __device__ __forceinline__ void route_select(int t, int E, int k, int routing, c
     int best = -1;
     float zb = 0.f;
     for (int e = 0; e < E; ++e) {
-      if ((taken >> e) & 1u) continue;
+      if ((taken >> e) & 1ull) continue;
       float ze = z[e];
       if (best < 0 || ze > zb) { best = e; zb = ze; }
     }
-    taken |= 1u << best;
+    taken |= 1ull << best;
     sel[j] = best;
     if (j == 0) first = best;
   }
   const float zmax = z[first];
   float psum = 0.f;
-  for (int e = 0; e < E; ++e) psum += expf(z[e] - zmax);
-  my_p = (lane < E) ? expf(z[lane] - zmax) / psum : 0.f;
-  my_g = 0.f;
+  for (int e = 0; e < E; ++e) psum += expf((z[e] - zmax) * scale);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int e = lane + 32 * h;
+    my_p[h] = (e < E) ? expf((z[e] - zmax) * scale) / psum : 0.f;
+    my_g[h] = 0.f;
+  }
   if (routing == BTX_ROUTE_SWITCH) {
-    float g0 = expf(z[first] - zmax) / psum;
-    if (lane == first) my_g = g0;
+    float g0 = expf((z[first] - zmax) * scale) / psum;
+    if ((first & 31) == lane) my_g[first >> 5] = g0;
     if (lane == 0) { topk[t] = first; gates[t] = g0; }
   } else {
     float gsum = 0.f;
-    for (int j = 0; j < k; ++j) gsum += expf(z[sel[j]] - zmax);
+    for (int j = 0; j < k; ++j) gsum += expf((z[sel[j]] - zmax) * scale);
     for (int j = 0; j < k; ++j) {
-      float gj = expf(z[sel[j]] - zmax) / gsum;
-      if (sel[j] == lane) my_g = gj;
+      float gj = expf((z[sel[j]] - zmax) * scale) / gsum;
+      if ((sel[j] & 31) == lane) my_g[sel[j] >> 5] = gj;
       if (lane == 0) { topk[(size_t)t * k + j] = sel[j]; gates[(size_t)t * k + j] = gj; }
     }
   }
-  if (lane < E) probs[(size_t)t * E + lane] = my_p;
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+    if (lane + 32 * h < E) probs[(size_t)t * E + lane + 32 * h] = my_p[h];
   __syncwarp();
 }
 
 // Routing of one token by one warp: logits (or the given ones), top-k by repeated arg-max with
 // ties to the lower index, gates, full softmax.  `z` is this warp's shared scratch of kMaxExperts
-// floats.  On return lane e (< E) holds the dense gate and the probability of expert e.
+// floats.  On return lane l holds the dense gate and the probability of experts l and l + 32.
 template <typename T>
 __device__ __forceinline__ void route_token(int t, int d, int E, int k, int routing, const T* __restrict__ x,
                                             const T* __restrict__ wr, const float* __restrict__ bias,
                                             const float* __restrict__ given_logits,
                                             const float* __restrict__ noise, float inv_tau, float* z, int lane,
                                             float* __restrict__ logits, int32_t* __restrict__ topk,
-                                            float* __restrict__ gates, float* __restrict__ probs, float& my_g,
-                                            float& my_p) {
+                                            float* __restrict__ gates, float* __restrict__ probs, float (&my_g)[2],
+                                            float (&my_p)[2]) {
   constexpr int VN = Vec<T>::N;
   if (given_logits != nullptr) {
-    if (lane < E) z[lane] = given_logits[(size_t)t * E + lane];
+    for (int e = lane; e < E; e += 32) z[e] = given_logits[(size_t)t * E + e] + (bias ? bias[e] : 0.f);
   } else {
     const T* xr = x + (size_t)t * d;
     for (int eb = 0; eb < E; eb += 8) {
@@ -133,12 +142,12 @@ __device__ __forceinline__ void route_token(int t, int d, int E, int k, int rout
     }
   }
   __syncwarp();
-  if (lane < E) {
-    logits[(size_t)t * E + lane] = z[lane];                       // reported logits are unperturbed
-    if (noise != nullptr) z[lane] = (z[lane] + noise[(size_t)t * E + lane]) * inv_tau;
+  for (int e = lane; e < E; e += 32) {
+    logits[(size_t)t * E + e] = z[e];                             // reported logits are unperturbed
+    if (noise != nullptr) z[e] = z[e] + noise[(size_t)t * E + e]; // one fp32 addition decides the expert
   }
   __syncwarp();
-  route_select(t, E, k, routing, z, lane, topk, gates, probs, my_g, my_p);
+  route_select(t, E, k, routing, noise != nullptr ? inv_tau : 1.0f, z, lane, topk, gates, probs, my_g, my_p);
 }
 
 template <typename T>
@@ -151,15 +160,17 @@ router_kernel(int Tn, int d, int E, int k, int routing, const T* __restrict__ x,
   __shared__ float zs[kRouterWarps][kMaxExperts];
   __shared__ float red[kRouterWarps][kMaxExperts][2];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  float u_acc = 0.f, p_acc = 0.f;      // lane e accumulates expert e over this warp's tokens
+  float u_acc[2] = {0.f, 0.f}, p_acc[2] = {0.f, 0.f};   // lane l accumulates experts l and l + 32 over this warp's tokens
   for (int t = blockIdx.x * kRouterWarps + warp; t < Tn; t += gridDim.x * kRouterWarps) {
-    float my_g, my_p;
+    float my_g[2], my_p[2];
     route_token<T>(t, d, E, k, routing, x, wr, bias, given_logits, noise, inv_tau, zs[warp], lane, logits, topk, gates,
                    probs, my_g, my_p);
-    u_acc += my_g;
-    p_acc += my_p;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
   }
-  if (lane < E) { red[warp][lane][0] = u_acc; red[warp][lane][1] = p_acc; }
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+    if (lane + 32 * h < E) { red[warp][lane + 32 * h][0] = u_acc[h]; red[warp][lane + 32 * h][1] = p_acc[h]; }
   __syncthreads();
   if (threadIdx.x < 2 * E) {
     int e = threadIdx.x >> 1, which = threadIdx.x & 1;
@@ -173,7 +184,7 @@ router_kernel(int Tn, int d, int E, int k, int routing, const T* __restrict__ x,
 // shuffle tree, so the result does not depend on scheduling.
 __global__ void __launch_bounds__(256)
 lb_finalize_kernel(int Tn, int E, int nblocks, float alpha, const float* __restrict__ route_part,
-                   float* __restrict__ u, float* __restrict__ p, float* __restrict__ loss) {
+                   float* __restrict__ u, float* __restrict__ p, float* __restrict__ loss, double* __restrict__ up64) {
   __shared__ double su[kMaxExperts], sp[kMaxExperts];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int pair = warp; pair < 2 * E; pair += 8) {
@@ -183,8 +194,8 @@ lb_finalize_kernel(int Tn, int E, int nblocks, float alpha, const float* __restr
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     s /= (double)Tn;
     if (lane == 0) {
-      if (pair & 1) { sp[pair >> 1] = s; p[pair >> 1] = (float)s; }
-      else { su[pair >> 1] = s; u[pair >> 1] = (float)s; }
+      if (pair & 1) { sp[pair >> 1] = s; p[pair >> 1] = (float)s; up64[E + (pair >> 1)] = s; }
+      else { su[pair >> 1] = s; u[pair >> 1] = (float)s; up64[pair >> 1] = s; }
     }
   }
   __syncthreads();
@@ -310,7 +321,8 @@ __global__ void __launch_bounds__(kSmallThreads)
 route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha, int mt_max, int r_pad_max, int cap,
                            const T* __restrict__ x, const T* __restrict__ wr, const float* __restrict__ bias,
                            const float* __restrict__ noise, float inv_tau, float* logits, int32_t* topk, float* gates, float* probs, float* __restrict__ u,
-                           float* __restrict__ p, float* __restrict__ loss, int32_t* __restrict__ counts,
+                           float* __restrict__ p, double* __restrict__ up64, float* __restrict__ loss,
+                           int32_t* __restrict__ counts,
                            int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
                            int32_t* __restrict__ tile_expert, int32_t* __restrict__ perm,
                            int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
@@ -361,13 +373,13 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
     for (int w = 0; w < NW; ++w) a += part[w][threadIdx.x];
     a += bias ? bias[threadIdx.x] : 0.f;
     logits[(size_t)t * E + threadIdx.x] = a;                      // reported logits are unperturbed
-    if (noise != nullptr) a = (a + noise[(size_t)t * E + threadIdx.x]) * inv_tau;
+    if (noise != nullptr) a = a + noise[(size_t)t * E + threadIdx.x];   // one fp32 addition decides the expert
     z[threadIdx.x] = a;
   }
   __syncthreads();
   if (warp == 0) {
-    float my_g, my_p;
-    route_select(t, E, k, routing, z, lane, topk, gates, probs, my_g, my_p);
+    float my_g[2], my_p[2];
+    route_select(t, E, k, routing, noise != nullptr ? inv_tau : 1.0f, z, lane, topk, gates, probs, my_g, my_p);
   }
   __threadfence();
   __syncthreads();
@@ -391,7 +403,7 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
     }
     if (lane == 0) {
       du /= (double)Tn; dp /= (double)Tn;
-      su[e] = du; sp[e] = dp; u[e] = (float)du; p[e] = (float)dp;
+      su[e] = du; sp[e] = dp; u[e] = (float)du; p[e] = (float)dp; up64[e] = du; up64[E + e] = dp;
     }
   }
   // ---- permutation: histogram, scan, stable scatter in rounds of one block ----
@@ -536,43 +548,68 @@ dg_rowsum_kernel(int nt, int r_pad_max, int E, const int32_t* __restrict__ pad_o
 }
 
 // One thread per token: d gate of every slot (the summed row-dot of its row plus the u-term of L_LB),
-// then the softmax Jacobians and the p-term of L_LB.
+// then the softmax Jacobians and the p-term of L_LB.  The L_LB terms are differences of nearly equal
+// numbers when the load is balanced (c_i - sum_j p_j c_j with all c_i close to one another, and
+// g_a (dg_a - sum_j g_j dg_j) with all dg_j close), which multiplies any error in sum_j p_j = 1 and
+// sum_j g_j = 1 a hundredfold: the thread therefore forms the two softmaxes again, in double, from the
+// saved fp32 logits (`logits` non-null; for Sample Top-1, whose softmax is that of the perturbed logits
+// and which has no L_LB terms, it takes the stored fp32 values), uses the batch means kept in double,
+// and rounds the result to fp32 once.
 __global__ void __launch_bounds__(64)
 router_dz_kernel(int Tn, int E, int k, int routing, float alpha, float lb_scale, int stopgrad_u,
                  const int32_t* __restrict__ topk, const float* __restrict__ gates,
-                 const float* __restrict__ probs, const float* __restrict__ u, const float* __restrict__ p,
+                 const float* __restrict__ probs, const float* __restrict__ logits,
+                 const double* __restrict__ up64,
                  const int32_t* __restrict__ flat2row, const float* __restrict__ dg_part, float dz_scale,
                  float* __restrict__ dz_out, float* __restrict__ dz_out2) {
   int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= Tn) return;
-  float dzv[kMaxExperts];
-  for (int e = 0; e < E; ++e) dzv[e] = 0.f;
-  const float lbc = lb_scale * alpha * (float)E / (float)Tn;
-  float dg[kMaxExperts];
+  const double* u = up64;
+  const double* p = up64 + E;
+  double pt[kMaxExperts], dzv[kMaxExperts], gt[kMaxExperts], dg[kMaxExperts];
+  if (logits != nullptr) {
+    const float* z = logits + (size_t)t * E;
+    double zmax = (double)z[0];
+    for (int e = 1; e < E; ++e) zmax = fmax(zmax, (double)z[e]);
+    double sum = 0.0;
+    for (int e = 0; e < E; ++e) { pt[e] = exp((double)z[e] - zmax); sum += pt[e]; }
+    for (int e = 0; e < E; ++e) pt[e] /= sum;
+    if (routing == BTX_ROUTE_SWITCH) {
+      gt[0] = pt[topk[t]];
+    } else {
+      double gsum = 0.0;
+      for (int s = 0; s < k; ++s) { gt[s] = exp((double)z[topk[(size_t)t * k + s]] - zmax); gsum += gt[s]; }
+      for (int s = 0; s < k; ++s) gt[s] /= gsum;
+    }
+  } else {
+    for (int e = 0; e < E; ++e) pt[e] = (double)probs[(size_t)t * E + e];
+    for (int s = 0; s < k; ++s) gt[s] = (double)gates[(size_t)t * k + s];
+  }
+  for (int e = 0; e < E; ++e) dzv[e] = 0.0;
+  const double lbc = (double)lb_scale * (double)alpha * (double)E / (double)Tn;
   for (int s = 0; s < k; ++s) {
-    float a = 0.f;
+    double a = 0.0;
     if (dg_part != nullptr) {
       int rp = flat2row[(size_t)t * k + s];
-      if (rp >= 0) a = dg_part[rp];                  // a dropped assignment has no path into y
+      if (rp >= 0) a = (double)dg_part[rp];          // a dropped assignment has no path into y
     }
     if (!stopgrad_u) a += lbc * p[topk[(size_t)t * k + s]];
     dg[s] = a;
   }
-  const float* pt = probs + (size_t)t * E;
   if (routing == BTX_ROUTE_SWITCH) {
     int sel = topk[t];
-    float ps = pt[sel];
+    double ps = pt[sel];
     for (int e = 0; e < E; ++e) dzv[e] = -dg[0] * ps * pt[e];
     dzv[sel] += dg[0] * ps;
   } else {
-    float inner = 0.f;
-    for (int s = 0; s < k; ++s) inner += gates[(size_t)t * k + s] * dg[s];
-    for (int s = 0; s < k; ++s) dzv[topk[(size_t)t * k + s]] = gates[(size_t)t * k + s] * (dg[s] - inner);
+    double inner = 0.0;
+    for (int s = 0; s < k; ++s) inner += gt[s] * dg[s];
+    for (int s = 0; s < k; ++s) dzv[topk[(size_t)t * k + s]] = gt[s] * (dg[s] - inner);
   }
-  float pc = 0.f;
+  double pc = 0.0;
   for (int e = 0; e < E; ++e) pc += pt[e] * (lbc * u[e]);
   for (int e = 0; e < E; ++e) {
-    float v = (dzv[e] + pt[e] * (lbc * u[e] - pc)) * dz_scale;
+    float v = (float)((dzv[e] + pt[e] * (lbc * u[e] - pc)) * (double)dz_scale);
     dz_out[(size_t)t * E + e] = v;
     if (dz_out2 != nullptr) dz_out2[(size_t)t * E + e] = v;
   }
@@ -663,7 +700,7 @@ cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, c
         pl.T, pl.d, pl.E, pl.k, routing, (const float*)x, (const float*)w_router, bias, given_logits, noise, inv_tau,
         b.logits, b.topk, b.gates, b.probs, b.route_part);
   }
-  lb_finalize_kernel<<<1, 256, 0, st>>>(pl.T, pl.E, pl.route_blocks, alpha, b.route_part, b.u, b.p, b.loss);
+  lb_finalize_kernel<<<1, 256, 0, st>>>(pl.T, pl.E, pl.route_blocks, alpha, b.route_part, b.u, b.p, b.loss, b.up64);
   return cudaGetLastError();
 }
 
@@ -675,13 +712,13 @@ cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, f
   if (dtype == BTX_BF16)
     route_permute_small_kernel<__nv_bfloat16><<<pl.T, kSmallThreads, 0, st>>>(
         pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, pl.capacity, (const __nv_bfloat16*)x,
-        (const __nv_bfloat16*)w_router, bias, noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets,
+        (const __nv_bfloat16*)w_router, bias, noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.up64, b.loss, b.counts, b.offsets,
         b.pad_offsets, b.tile_expert, b.perm, b.inv_perm, b.rowmap, b.flat2row, b.status + 8);
   else
     route_permute_small_kernel<float><<<pl.T, kSmallThreads, 0, st>>>(
         pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, pl.capacity, (const float*)x,
         (const float*)w_router, bias,
-        noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.loss, b.counts, b.offsets, b.pad_offsets, b.tile_expert, b.perm,
+        noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.up64, b.loss, b.counts, b.offsets, b.pad_offsets, b.tile_expert, b.perm,
         b.inv_perm, b.rowmap, b.flat2row, b.status + 8);
   return cudaGetLastError();
 }
@@ -704,7 +741,7 @@ cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st) {
 
 cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st) {
   int row_vecs = pl.d * pl.esize / 16;
-  int blocks = min(pl.r_pad_max / 8, 148 * 16);
+  int blocks = min(pl.r_pad_max / 8, sm_count() * 16);
   // small batches: the gather's launch overlaps the routing kernel's run
   return launch_after_predecessor(gather_rows_kernel, dim3(blocks), dim3(256), 0, st, pl.small != 0, pl.k, row_vecs,
                                   (const uint4*)src, (uint4*)dst_sorted, (const int32_t*)b.rowmap,
@@ -714,7 +751,7 @@ cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted
 cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, const Buffers& b,
                            cudaStream_t st) {
   size_t n = (size_t)pl.T * (pl.d / 4);
-  int blocks = (int)min((n + 255) / 256, (size_t)148 * 32);
+  int blocks = (int)min((n + 255) / 256, (size_t)sm_count() * 32);
   const int32_t* kept = pl.capped ? b.flat2row : nullptr;
   if (dtype == BTX_BF16)
     return launch_after_predecessor(combine_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, pl.small != 0, pl.T,
@@ -727,18 +764,18 @@ cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int spl
 cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float alpha, float lb_scale,
                                    int stopgrad_u, int have_dg, const void* x, const void* w_router, const Buffers& b,
                                    void* dx, float* dw_router, float* dbias, float* dlogits_out, int accumulate,
-                                   float dz_scale, cudaStream_t st) {
+                                   float dz_scale, int perturbed, cudaStream_t st) {
   if (have_dg)
     dg_rowsum_kernel<<<(pl.r_pad_max + 255) / 256, 256, 0, st>>>(pl.nt_dact, pl.r_pad_max, pl.E, b.pad_offsets, b.dg_part);
   router_dz_kernel<<<(pl.T + 63) / 64, 64, 0, st>>>(pl.T, pl.E, pl.k, routing, alpha, lb_scale, stopgrad_u, b.topk,
-                                                    b.gates, b.probs, b.u, b.p, b.flat2row,
+                                                    b.gates, b.probs, perturbed ? nullptr : b.logits, b.up64, b.flat2row,
                                                     have_dg ? b.dg_part : nullptr, dz_scale, b.dz, dlogits_out);
   if (x == nullptr) return cudaGetLastError();     // loss-only gradient (btx_lb_loss)
   const int vn = dtype == BTX_BF16 ? 8 : 4;
   dim3 grid(pl.wr_chunks, (pl.d / vn + 127) / 128);
   float* bias_part = b.dwr_part + (size_t)pl.wr_chunks * pl.E * pl.d;
   size_t n = (size_t)pl.T * (pl.d / 4);
-  int cblocks = (int)min((n + 255) / 256, (size_t)148 * 32);
+  int cblocks = (int)min((n + 255) / 256, (size_t)sm_count() * 32);
   const int32_t* kept = pl.capped ? b.flat2row : nullptr;
   if (dtype == BTX_BF16) {
     router_dw_partial_kernel<__nv_bfloat16><<<grid, 128, 0, st>>>(pl.T, pl.d, pl.E, (const __nv_bfloat16*)x, b.dz,

@@ -228,17 +228,6 @@ inline bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t r
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-inline int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
-}
-
 inline bool aligned32(const void* p) { return ((uintptr_t)p & 31) == 0; }
 
 }  // namespace tcx

@@ -1,8 +1,10 @@
 """Parity at the benchmark's full sizes (Llama-2-7B-shaped layer: d_model 4096, d_ff 11008, 4 experts),
 in the launch configuration bench.py times.  Routing, counts and the permutation are compared in full
 and bit-exactly (oracle fed the GPU's fp32 logits); floating-point outputs are compared on sampled
-tokens (y, dx) and sampled hidden units (dW1, dW3, dW2), which the oracle computes one by one, plus
-properties that hold at any size (router-gradient rows sum to zero)."""
+tokens (y, dx) and sampled hidden units (dW1, dW3, dW2), which the oracle computes one by one; the router
+gradient is compared in full (all E x d entries) through the oracle's sum over the GPU's d(loss)/d(logits),
+which itself is compared on the sampled tokens; plus properties that hold at any size (router-gradient
+rows sum to zero)."""
 import numpy as np
 import pytest
 import torch
@@ -76,6 +78,19 @@ def full_size_case(T, k, seed, routing=B.ROUTE_TOPK, bias=None, backward=True, n
                 continue
             err = rel_err(np64(have), want)
             assert err <= TOL, f"{name}[{e}] {err}"
+    # router gradient at full size.  d(loss)/d(logits) on the sampled tokens against the oracle; then dW_l and
+    # dbias over ALL tokens against the oracle's sums of the GPU's own dz (x and dz are the same numbers on both
+    # sides, so only the order of the fp32 additions differs: a far tighter bar than the layer's tolerance).
+    dz_gpu = got["dlogits"].cpu().numpy()
+    assert np.all(np.isfinite(dz_gpu))
+    e_dz = np.max(np.abs(dz_gpu[tok] - sl["dlogits"])) / np.max(np.abs(sl["dlogits"]))
+    assert e_dz <= TOL, f"dlogits {e_dz}"
+    dwr_ref, db_ref = o.router_wgrad_from_dz(cpu["x"], dz_gpu)
+    e_dwr = rel_err(np64(got["dw_router"]), dwr_ref)
+    assert e_dwr <= 1e-4, f"dw_router {e_dwr}"
+    summed = float(np.max(np.sum(np.abs(dz_gpu.astype(np.float64)), axis=0)))
+    e_db = float(np.max(np.abs(np64(got["dbias"]) - db_ref))) / summed
+    assert e_db <= 1e-4, f"dbias {e_db}"
     # properties at full size: every softmax Jacobian is shift invariant
     dwr = np64(got["dw_router"])
     assert np.all(np.isfinite(dwr))

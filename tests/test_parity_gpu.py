@@ -46,12 +46,15 @@ def test_ragged_shapes(dtype, T, d, F, E, k):
 
 
 @pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
-@pytest.mark.parametrize("T,d,F,routing,k", [(200, 72, 40, B.ROUTE_TOPK, 8), (150, 64, 72, B.ROUTE_SOFT, 32),
-                                             (40, 8, 8, B.ROUTE_TOPK, 32), (2500, 64, 64, B.ROUTE_SWITCH, 1)])
-def test_maximum_expert_count_and_smallest_widths(dtype, T, d, F, routing, k):
-    """E = 32 (the library's limit): sparse loads with experts that receive nothing, every expert
-    selected (k = E), rows of a single 16-byte vector, and more padded row tiles than tokens."""
-    run_case(T, d, F, 32, k, dtype, seed=17, routing=routing, alpha=0.05, lb_scale=0.7)
+@pytest.mark.parametrize("E", [32, 64])
+@pytest.mark.parametrize("T,d,F,routing,k", [(200, 72, 40, B.ROUTE_TOPK, 8), (150, 64, 72, B.ROUTE_SOFT, 0),
+                                             (40, 8, 8, B.ROUTE_TOPK, 0), (2500, 64, 64, B.ROUTE_SWITCH, 1),
+                                             (300, 64, 72, B.ROUTE_TOPK, 3), (12, 64, 72, B.ROUTE_TOPK, 3)])
+def test_maximum_expert_count_and_smallest_widths(dtype, E, T, d, F, routing, k):
+    """E = 64 (the library's limit) and E = 32 (one warp lane per expert exactly): sparse loads with experts
+    that receive nothing, every expert selected (k = 0 stands for k = E), rows of a single 16-byte vector,
+    more padded row tiles than tokens, and the small-batch path with more row tiles than its usual handful."""
+    run_case(T, d, F, E, k if k else E, dtype, seed=17, routing=routing, alpha=0.05, lb_scale=0.7)
 
 
 @pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
@@ -133,6 +136,30 @@ def test_sample_top1_routing(dtype, tau):
             assert float(got["dw_router"].abs().max()) == 0.0
 
 
+@pytest.mark.parametrize("dtype", DTYPES, ids=IDS)
+@pytest.mark.parametrize("tau", [0.7, 0.0], ids=["soft", "hard"])
+def test_sample_top1_perturbed_logits_that_tie_in_fp32(dtype, tau):
+    """The expert of Sample Top-1 is decided on z + G formed by one fp32 addition: where two sums differ only
+    below fp32 resolution they tie and the lower index wins, whatever the temperature (which scales only the
+    softmax).  Tokens are unit vectors, so the logits are router weights exactly."""
+    for T in (64, 700):                                   # one-launch and multi-block routing kernels
+        inp = synth.moe_inputs(T, 64, 72, 4, 14, dtype, DEV)
+        inp["x"].zero_()
+        inp["x"][:, 0] = 1.0
+        inp["w_router"].zero_()
+        inp["w_router"][:, 0] = torch.tensor([0.0, 2.0 ** -25, -3.0, -3.0], dtype=dtype, device=DEV)
+        noise = torch.zeros(T, 4, dtype=torch.float32, device=DEV)
+        noise[:, 0] = 1.0
+        noise[:, 1] = 1.0                                  # fp64: expert 1 leads by 2^-25; fp32: 1 + 2^-25 == 1
+        noise[T // 2:, 1] = 1.0 + 2.0 ** -20               # second half: expert 1 leads in fp32 as well
+        fwd = gpu_forward(inp, 1, B.ROUTE_SAMPLE1, alpha=0.0, noise=noise, tau=tau)
+        idx = fwd["routing"].topk_idx.cpu().numpy()[:, 0]
+        assert (idx[:T // 2] == 0).all() and (idx[T // 2:] == 1).all()
+        cpu, b64, z_gpu, ref = check_forward(inp, fwd, 1, B.ROUTE_SAMPLE1, 0.0, None, TOL[dtype], noise=noise, tau=tau)
+        got = gpu_backward(inp, fwd)
+        check_backward(cpu, b64, z_gpu, got, 1, B.ROUTE_SAMPLE1, 0.0, 1.0, False, TOL[dtype], noise=noise, tau=tau)
+
+
 def test_results_are_deterministic_across_runs():
     inp = synth.moe_inputs(256, 256, 688, 4, 0, torch.float32, DEV)
     a = gpu_forward(inp, 2)
@@ -144,17 +171,19 @@ def test_results_are_deterministic_across_runs():
         assert torch.equal(ga[n], gb[n]), n
 
 
+@pytest.mark.parametrize("with_bias", [False, True], ids=["nobias", "bias"])
 @pytest.mark.parametrize("routing,k", [(B.ROUTE_TOPK, 2), (B.ROUTE_SWITCH, 1), (B.ROUTE_SOFT, 4)])
-def test_lb_loss_entry_point(routing, k):
+def test_lb_loss_entry_point(routing, k, with_bias):
     T, E, alpha = 333, 4, 0.01
     g = torch.Generator(device="cpu").manual_seed(4)
     logits = (torch.randn(T, E, generator=g) * 1.3).to(DEV)
+    bias = torch.tensor([0.75, -0.5, 0.0, 1.25], device=DEV) if with_bias else None
     desc = B.make_desc(T, 0, 0, E, k, torch.float32, routing, alpha)
     ws = torch.empty(B.btx_lb_loss_workspace_size(desc), dtype=torch.uint8, device=DEV)
     loss = torch.empty(1, device=DEV); u = torch.empty(E, device=DEV); p = torch.empty(E, device=DEV)
     dz = torch.empty(T, E, device=DEV)
-    B.btx_lb_loss(desc, logits, loss, u, p, dz, ws)
-    z = logits.cpu().numpy()
+    B.btx_lb_loss(desc, logits, loss, u, p, dz, ws, router_bias=bias)
+    z = (logits + bias).cpu().numpy() if with_bias else logits.cpu().numpy()    # the same fp32 sum the kernel forms
     kk = E if routing == B.ROUTE_SOFT else k
     want, wu, wp = o.lb_loss_from_logits(z, kk, routing, alpha)
     assert abs(loss.item() - want) <= 1e-5 * want

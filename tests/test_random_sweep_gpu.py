@@ -14,6 +14,12 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
+def draw_T(r):
+    """Batch sizes from a single token up: a third of the cases below 96 tokens (the one-launch routing
+    and weight-streaming kernels, single-tile experts), the rest up to 1400."""
+    return int(r.integers(1, 96)) if r.integers(0, 3) == 0 else int(r.integers(96, 1400))
+
+
 def make_cases(n, seed):
     r = np.random.default_rng(seed)
     cases = []
@@ -21,7 +27,7 @@ def make_cases(n, seed):
         E = int(r.integers(1, 13))
         routing = [B.ROUTE_TOPK, B.ROUTE_TOPK, B.ROUTE_SWITCH, B.ROUTE_SOFT, B.ROUTE_SAMPLE1][int(r.integers(0, 5))]
         k = int(r.integers(1, E + 1)) if routing == B.ROUTE_TOPK else (E if routing == B.ROUTE_SOFT else 1)
-        c = dict(T=int(r.integers(96, 1400)), d=8 * int(r.integers(2, 33)), F=8 * int(r.integers(2, 49)), E=E, k=k,
+        c = dict(T=draw_T(r), d=8 * int(r.integers(2, 33)), F=8 * int(r.integers(2, 49)), E=E, k=k,
                  routing=routing, seed=1000 + i,
                  alpha=0.0 if routing == B.ROUTE_SAMPLE1 else float(r.choice([0.0, 0.01, 0.3])),
                  tau=float(r.choice([0.0, 0.6, 1.4])) if routing == B.ROUTE_SAMPLE1 else 0.0,
@@ -32,11 +38,23 @@ def make_cases(n, seed):
     return cases
 
 
-CASES = make_cases(14, 20240311)
+CASES = make_cases(24, 20240311)
+
+# Two small batches with two experts and Switch routing, kept by name: there the two entries of dbias are +s
+# and -s with s a sum of mixed-sign terms that nearly cancels, and the plain max-norm figure of dbias reads
+# 1.6e-2 and 2.2e-2 in BF16 while every other tensor sits at 2-4e-3.  dbias is held to the tolerance relative
+# to the size of what was summed (see check_backward); everything else to the max-norm bar.
+NAMED = {
+    "two_experts_switch_T89": dict(T=89, d=128, F=336, E=2, k=1, routing=B.ROUTE_SWITCH, seed=1012, alpha=0.0, tau=0.0,
+                                   bias=True, stopgrad=True, frozen=True, accumulate=False, lb_scale=1.0, cf=0.0),
+    "two_experts_switch_T17": dict(T=17, d=256, F=288, E=2, k=1, routing=B.ROUTE_SWITCH, seed=1103, alpha=0.01, tau=0.0,
+                                   bias=True, stopgrad=False, frozen=False, accumulate=False, lb_scale=0.4, cf=0.6),
+}
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
-@pytest.mark.parametrize("c", CASES, ids=[f"case{i}" for i in range(len(CASES))])
+@pytest.mark.parametrize("c", CASES + list(NAMED.values()),
+                         ids=[f"case{i}" for i in range(len(CASES))] + list(NAMED.keys()))
 def test_option_combinations(c, dtype):
     inp = synth.moe_inputs(c["T"], c["d"], c["F"], c["E"], c["seed"], dtype, DEV)
     tol = TOL[dtype]
