@@ -240,6 +240,7 @@ def free_device_memory():
 # kernels launched per call (memsets and copies are not counted)
 LAUNCHES_FWD = 9          # router, loss finalise, 3 permutation kernels, gather, GEMM-1, GEMM-2, combine
 LAUNCHES_FWD_SMALL = 6    # one-launch routing, gather, pass 1, SwiGLU fix-up, pass 2, combine
+LAUNCHES_FWD_DENSE = 4    # inference with at most 64 tokens: pass 1 (+SwiGLU), routing beside it, pass 2, combine
 LAUNCHES_BWD = 11         # dy gather, dgrad-2, dgrad-1, 3 weight gradients, row-sum, dz, dW_l partial, dx combine, reduce
 
 
@@ -288,6 +289,8 @@ class MoeRun:
 
     def launches_per_step(self):
         fwd = LAUNCHES_FWD_SMALL if self.T * self.k_eff <= 1024 else LAUNCHES_FWD
+        if not self.train and self.T <= 64:
+            fwd = LAUNCHES_FWD_DENSE
         return (fwd + (LAUNCHES_BWD if self.train else 0)) * self.layers
 
     def flops_per_step(self, rows):
@@ -483,7 +486,7 @@ def moe_result(run, ms, clocks, stages, soaked, K, W, world, peaks, with_counts)
                    roofline={"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                              "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0, "traffic": None,
                              "peak_source": peaks["_source"],
-                             "kernel": "tc_swapk_kernel (weight-streaming passes) over the whole step"})
+                             "kernel": "tc_dense_kernel (the two weight-streaming passes) over the whole step"})
     else:
         res.update(metric="moe_ffn_%s_tokens_per_s" % run.workload, value=run.T / (ms * 1e-3) * world, unit="tokens/s",
                    tflops=run.flops_per_step(rows) / (ms * 1e-3) / 1e12 * world)

@@ -55,6 +55,8 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
     const int chunks = p.E < p.R ? p.E : p.R;             // typical: every expert holds one token chunk
     p.dec_s1 = pick_decode_splits(2 * chunks * ((p.F + 255) / 256), (p.d + 63) / 64);
     p.dec_s2 = pick_decode_splits(chunks * ((p.d + 255) / 256), (p.F + 63) / 64);
+    p.dense = dense_small_fits(p, desc->save_for_backward) ? 1 : 0;
+    p.dense_n = (p.T + 15) & ~15;
   }
 
   size_t o = 0;
@@ -243,27 +245,36 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
   resolve(pl, sv, ws, &b);
 
   mark_stage(0, st);
-  BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
-  if (route_permute_small_fits(pl)) {
-    BTX_CUDA_OK(launch_route_permute_small(pl, desc->dtype, er.routing, desc->lb_alpha, x, w_router, router_bias, noise,
-                                           er.inv_tau, b, st));
-  } else {
-    BTX_CUDA_OK(launch_router(pl, desc->dtype, er.routing, desc->lb_alpha, x, w_router, router_bias, nullptr, noise,
-                              er.inv_tau, b, st));
-    BTX_CUDA_OK(launch_permute(pl, b, st));
-  }
-  BTX_CUDA_OK(launch_gather_rows(pl, x, b.xs, b, st));
-  mark_stage(1, st);
   const float* expert_rows = b.yp;
   int splits = 1;
-  if (desc->dtype == BTX_F32) {
-    BTX_CUDA_OK(launch_expert_forward_f32(pl, w1, w3, w2, b, desc->save_for_backward, st));
-  } else if (pl.small) {
-    if ((s = launch_expert_forward_small_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
-    expert_rows = b.part;
-    splits = pl.dec_s2;
+  if (pl.dense) {
+    // a handful of tokens, nothing kept: the first expert kernel clears the status word and starts at once,
+    // the routing runs beside it, no gather
+    mark_stage(1, st);
+    if ((s = launch_expert_forward_dense_bf16(pl, er.routing, desc->lb_alpha, x, w_router, router_bias, noise, er.inv_tau,
+                                              w1, w3, w2, b, st)) != BTX_OK)
+      return s;
   } else {
-    if ((s = launch_expert_forward_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
+    BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
+    if (route_permute_small_fits(pl)) {
+      BTX_CUDA_OK(launch_route_permute_small(pl, desc->dtype, er.routing, desc->lb_alpha, x, w_router, router_bias, noise,
+                                             er.inv_tau, b, st));
+    } else {
+      BTX_CUDA_OK(launch_router(pl, desc->dtype, er.routing, desc->lb_alpha, x, w_router, router_bias, nullptr, noise,
+                                er.inv_tau, b, st));
+      BTX_CUDA_OK(launch_permute(pl, b, st));
+    }
+    BTX_CUDA_OK(launch_gather_rows(pl, x, b.xs, b, st));
+    mark_stage(1, st);
+    if (desc->dtype == BTX_F32) {
+      BTX_CUDA_OK(launch_expert_forward_f32(pl, w1, w3, w2, b, desc->save_for_backward, st));
+    } else if (pl.small) {
+      if ((s = launch_expert_forward_small_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
+      expert_rows = b.part;
+      splits = pl.dec_s2;
+    } else {
+      if ((s = launch_expert_forward_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
+    }
   }
   mark_stage(3, st);
   BTX_CUDA_OK(launch_combine(pl, desc->dtype, expert_rows, splits, y, b, st));

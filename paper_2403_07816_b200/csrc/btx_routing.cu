@@ -313,81 +313,24 @@ perm_scatter_kernel(int R, int E, int nblocks, int cap, const int32_t* __restric
 constexpr int kSmallThreads = 256;
 constexpr int kSmallMaxR = 1024;
 
-// One block per token computes its logits (eight warps share the row) and routes it; the block that
-// finishes last (a ticket counter in the workspace status block) then forms u, p, the loss and the
-// permutation.  Every sum runs in a fixed order, so results do not depend on which block is last.
-template <typename T>
-__global__ void __launch_bounds__(kSmallThreads)
-route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha, int mt_max, int r_pad_max, int cap,
-                           const T* __restrict__ x, const T* __restrict__ wr, const float* __restrict__ bias,
-                           const float* __restrict__ noise, float inv_tau, float* logits, int32_t* topk, float* gates, float* probs, float* __restrict__ u,
-                           float* __restrict__ p, double* __restrict__ up64, float* __restrict__ loss,
-                           int32_t* __restrict__ counts,
-                           int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
-                           int32_t* __restrict__ tile_expert, int32_t* __restrict__ perm,
-                           int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
-                           int32_t* __restrict__ flat2row, int32_t* ticket) {
-  constexpr int NW = kSmallThreads / 32;
-  constexpr int VN = Vec<T>::N;
-  __shared__ float part[NW][kMaxExperts];
-  __shared__ float z[kMaxExperts];
+// Batch means u and p, the loss, and the permutation of a small batch (R <= 1024) by ONE block of THREADS
+// threads, from the per-token routing results already in global memory.  Every sum runs in a fixed
+// order, so the result does not depend on which block runs this or on how many threads it has.
+template <int THREADS>
+__device__ __forceinline__ void small_batch_finish(int Tn, int E, int k, float alpha, int mt_max, int r_pad_max, int cap,
+                                                   const int32_t* topk, const float* gates, const float* probs,
+                                                   float* __restrict__ u, float* __restrict__ p,
+                                                   double* __restrict__ up64, float* __restrict__ loss,
+                                                   int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+                                                   int32_t* __restrict__ pad_offsets, int32_t* __restrict__ tile_expert,
+                                                   int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
+                                                   int32_t* __restrict__ rowmap, int32_t* __restrict__ flat2row) {
+  constexpr int NW = THREADS / 32;
   __shared__ double su[kMaxExperts], sp[kMaxExperts];
   __shared__ int hist[kMaxExperts + 1], running[kMaxExperts + 1], soff[kMaxExperts + 1], spad[kMaxExperts + 1];
   __shared__ int wcnt[NW][kMaxExperts + 1];
-  __shared__ int is_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t = blockIdx.x;
   const int R = Tn * k;
-  allow_dependents();
-
-  const T* xr = x + (size_t)t * d;
-  for (int eb = 0; eb < E; eb += 8) {
-    float acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-#pragma unroll 2
-    for (int c = (warp * 32 + lane) * VN; c < d; c += NW * 32 * VN) {
-      float xv[VN];
-      Vec<T>::load(xr + c, xv);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (eb + j < E) {
-          float wv[VN];
-          Vec<T>::load(wr + (size_t)(eb + j) * d + c, wv);
-#pragma unroll
-          for (int v = 0; v < VN; ++v) acc[j] = fmaf(xv[v], wv[v], acc[j]);
-        }
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      float a = acc[j];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-      if (lane == 0 && eb + j < E) part[warp][eb + j] = a;
-    }
-  }
-  __syncthreads();
-  if (threadIdx.x < E) {
-    float a = 0.f;
-    for (int w = 0; w < NW; ++w) a += part[w][threadIdx.x];
-    a += bias ? bias[threadIdx.x] : 0.f;
-    logits[(size_t)t * E + threadIdx.x] = a;                      // reported logits are unperturbed
-    if (noise != nullptr) a = a + noise[(size_t)t * E + threadIdx.x];   // one fp32 addition decides the expert
-    z[threadIdx.x] = a;
-  }
-  __syncthreads();
-  if (warp == 0) {
-    float my_g[2], my_p[2];
-    route_select(t, E, k, routing, noise != nullptr ? inv_tau : 1.0f, z, lane, topk, gates, probs, my_g, my_p);
-  }
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-
   // ---- last block: batch means, loss ----
   for (int e = warp; e < E; e += NW) {
     double du = 0.0, dp = 0.0;
@@ -408,11 +351,11 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
   }
   // ---- permutation: histogram, scan, stable scatter in rounds of one block ----
   if (threadIdx.x <= kMaxExperts) hist[threadIdx.x] = 0;
-  for (int j = threadIdx.x; j < r_pad_max; j += kSmallThreads) rowmap[j] = -1;
+  for (int j = threadIdx.x; j < r_pad_max; j += THREADS) rowmap[j] = -1;
   if (cap < R)
-    for (int j = threadIdx.x; j < R; j += kSmallThreads) perm[j] = -1;
+    for (int j = threadIdx.x; j < R; j += THREADS) perm[j] = -1;
   __syncthreads();
-  for (int i = threadIdx.x; i < R; i += kSmallThreads) atomicAdd(&hist[__ldcg(topk + i)], 1);
+  for (int i = threadIdx.x; i < R; i += THREADS) atomicAdd(&hist[__ldcg(topk + i)], 1);
   __syncthreads();
   if (threadIdx.x == 0) {
     double acc = 0.0;
@@ -428,15 +371,15 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
     offsets[E] = o; pad_offsets[E] = po; soff[E] = o; spad[E] = po;
   }
   __syncthreads();
-  for (int mt = threadIdx.x; mt < mt_max; mt += kSmallThreads) {
+  for (int mt = threadIdx.x; mt < mt_max; mt += THREADS) {
     const int row = mt * kRowTile;
     int ex = -1;
     for (int q = 0; q < E; ++q)
       if (row >= spad[q] && row < spad[q + 1]) ex = q;
     tile_expert[mt] = ex;
   }
-  for (int r0 = 0; r0 < R; r0 += kSmallThreads) {
-    for (int j = threadIdx.x; j < NW * (kMaxExperts + 1); j += kSmallThreads) (&wcnt[0][0])[j] = 0;
+  for (int r0 = 0; r0 < R; r0 += THREADS) {
+    for (int j = threadIdx.x; j < NW * (kMaxExperts + 1); j += THREADS) (&wcnt[0][0])[j] = 0;
     __syncthreads();
     const int i = r0 + threadIdx.x;
     const int e = (i < R) ? __ldcg(topk + i) : E;       // E = dummy bucket for idle lanes
@@ -463,6 +406,144 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
     }
     __syncthreads();
   }
+}
+
+
+// Logits of one token by eight warps that share its row: warp w takes every eighth 16-byte vector,
+// part[w][e] receives its share of <x_t, W_l[e]>; the caller adds the eight parts in warp order.
+template <typename T>
+__device__ __forceinline__ void token_logit_parts(const T* __restrict__ xr, const T* __restrict__ wr, int d, int E,
+                                                  int warp, int lane, float (*part)[kMaxExperts]) {
+  constexpr int NW = kSmallThreads / 32;
+  constexpr int VN = Vec<T>::N;
+  for (int eb = 0; eb < E; eb += 8) {
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+#pragma unroll 2
+    for (int c = (warp * 32 + lane) * VN; c < d; c += NW * 32 * VN) {
+      float xv[VN];
+      Vec<T>::load(xr + c, xv);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (eb + j < E) {
+          float wv[VN];
+          Vec<T>::load(wr + (size_t)(eb + j) * d + c, wv);
+#pragma unroll
+          for (int v = 0; v < VN; ++v) acc[j] = fmaf(xv[v], wv[v], acc[j]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      float a = acc[j];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+      if (lane == 0 && eb + j < E) part[warp][eb + j] = a;
+    }
+  }
+}
+
+// One block per token computes its logits (eight warps share the row) and routes it; the block that
+// finishes last (a ticket counter in the workspace status block) then forms u, p, the loss and the
+// permutation.  Every sum runs in a fixed order, so results do not depend on which block is last.
+template <typename T>
+__global__ void __launch_bounds__(kSmallThreads)
+route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha, int mt_max, int r_pad_max, int cap,
+                           const T* __restrict__ x, const T* __restrict__ wr, const float* __restrict__ bias,
+                           const float* __restrict__ noise, float inv_tau, float* logits, int32_t* topk, float* gates, float* probs, float* __restrict__ u,
+                           float* __restrict__ p, double* __restrict__ up64, float* __restrict__ loss,
+                           int32_t* __restrict__ counts,
+                           int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
+                           int32_t* __restrict__ tile_expert, int32_t* __restrict__ perm,
+                           int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
+                           int32_t* __restrict__ flat2row, int32_t* ticket) {
+  constexpr int NW = kSmallThreads / 32;
+  __shared__ float part[NW][kMaxExperts];
+  __shared__ float z[kMaxExperts];
+  __shared__ int is_last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x;
+  allow_dependents();
+
+  token_logit_parts<T>(x + (size_t)t * d, wr, d, E, warp, lane, part);
+  __syncthreads();
+  if (threadIdx.x < E) {
+    float a = 0.f;
+    for (int w = 0; w < NW; ++w) a += part[w][threadIdx.x];
+    a += bias ? bias[threadIdx.x] : 0.f;
+    logits[(size_t)t * E + threadIdx.x] = a;                      // reported logits are unperturbed
+    if (noise != nullptr) a = a + noise[(size_t)t * E + threadIdx.x];   // one fp32 addition decides the expert
+    z[threadIdx.x] = a;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    float my_g[2], my_p[2];
+    route_select(t, E, k, routing, noise != nullptr ? inv_tau : 1.0f, z, lane, topk, gates, probs, my_g, my_p);
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+
+  small_batch_finish<kSmallThreads>(Tn, E, k, alpha, mt_max, r_pad_max, cap, topk, gates, probs, u, p, up64, loss, counts,
+                                    offsets, pad_offsets, tile_expert, perm, inv_perm, rowmap, flat2row);
+}
+
+// The same routing for a handful of tokens whose expert kernels do not wait for it (they multiply every
+// expert's weights with all tokens and look the routing up in their epilogues): one cluster of eight
+// blocks, each taking every eighth token with the arithmetic of the kernel above; after a cluster
+// barrier the first block forms the batch means, the loss and the permutation.  No ticket is needed.
+// The kernel is launched as a programmatic dependent of the first expert kernel, which lets it start only
+// after everything earlier in the stream is complete; it runs beside that kernel (256 threads of at most
+// 64 registers fit next to one of its blocks) and, its work done, stays parked until that kernel has
+// completed, so that whoever waits for this kernel has waited for both.
+constexpr int kRouteCluster = 8;
+
+template <typename T>
+__global__ void __cluster_dims__(kRouteCluster, 1, 1) __launch_bounds__(kSmallThreads, 4)
+route_permute_cluster_kernel(int Tn, int d, int E, int k, int routing, float alpha, int mt_max, int r_pad_max, int cap,
+                             const T* __restrict__ x, const T* __restrict__ wr, const float* __restrict__ bias,
+                             const float* __restrict__ noise, float inv_tau, float* logits, int32_t* topk, float* gates,
+                             float* probs, float* __restrict__ u, float* __restrict__ p, double* __restrict__ up64,
+                             float* __restrict__ loss, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+                             int32_t* __restrict__ pad_offsets, int32_t* __restrict__ tile_expert,
+                             int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
+                             int32_t* __restrict__ flat2row) {
+  constexpr int NW = kSmallThreads / 32;
+  __shared__ float part[NW][kMaxExperts];
+  __shared__ float z[kMaxExperts];
+  allow_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int t = blockIdx.x; t < Tn; t += kRouteCluster) {
+    token_logit_parts<T>(x + (size_t)t * d, wr, d, E, warp, lane, part);
+    __syncthreads();
+    if (threadIdx.x < E) {
+      float a = 0.f;
+      for (int w = 0; w < NW; ++w) a += part[w][threadIdx.x];
+      a += bias ? bias[threadIdx.x] : 0.f;
+      logits[(size_t)t * E + threadIdx.x] = a;
+      if (noise != nullptr) a = a + noise[(size_t)t * E + threadIdx.x];
+      z[threadIdx.x] = a;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      float my_g[2], my_p[2];
+      route_select(t, E, k, routing, noise != nullptr ? inv_tau : 1.0f, z, lane, topk, gates, probs, my_g, my_p);
+    }
+    __syncthreads();
+  }
+  // every block's routing results are visible to the first block after the cluster barrier
+  __threadfence();
+  __syncthreads();
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (blockIdx.x == 0)
+    small_batch_finish<kSmallThreads>(Tn, E, k, alpha, mt_max, r_pad_max, cap, topk, gates, probs, u, p, up64, loss, counts,
+                                      offsets, pad_offsets, tile_expert, perm, inv_perm, rowmap, flat2row);
+  grid_dependency_wait();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -721,6 +802,16 @@ cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, f
         noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.u, b.p, b.up64, b.loss, b.counts, b.offsets, b.pad_offsets, b.tile_expert, b.perm,
         b.inv_perm, b.rowmap, b.flat2row, b.status + 8);
   return cudaGetLastError();
+}
+
+cudaError_t launch_route_permute_cluster(const Plan& pl, int routing, float alpha, const void* x, const void* w_router,
+                                       const float* bias, const float* noise, float inv_tau, const Buffers& b,
+                                       cudaStream_t st) {
+  return launch_after_predecessor(route_permute_cluster_kernel<__nv_bfloat16>, dim3(kRouteCluster), dim3(kSmallThreads), 0, st, true,
+                                  pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, pl.capacity,
+                                  (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, noise, inv_tau, b.logits,
+                                  b.topk, b.gates, b.probs, b.u, b.p, b.up64, b.loss, b.counts, b.offsets, b.pad_offsets,
+                                  b.tile_expert, b.perm, b.inv_perm, b.rowmap, b.flat2row);
 }
 
 cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st) {

@@ -320,6 +320,41 @@ def test_capacity_factor_small_batch_and_limits(dtype):
         gpu_forward(inp, E, B.ROUTE_SOFT, 0.01, None, capacity_factor=1.5)
 
 
+@pytest.mark.parametrize("T,d,F,E,k,routing,cf", [
+    (32, 256, 688, 4, 2, B.ROUTE_TOPK, 0.0),      # the decode shape in small: F = 5*128 + 48, one 32-column group
+    (5, 128, 136, 4, 2, B.ROUTE_TOPK, 0.0),       # N = 16 with 5 real tokens; the second CTA's token rows are all padding
+    (64, 264, 392, 4, 2, B.ROUTE_TOPK, 0.0),      # N = 64: both column groups; contraction tails in both passes
+    (33, 128, 256, 8, 8, B.ROUTE_SOFT, 0.0),      # every expert for every token; N = 48
+    (17, 192, 328, 2, 1, B.ROUTE_SWITCH, 0.0),
+    (1, 128, 128, 1, 1, B.ROUTE_TOPK, 0.0),       # a single token, a single expert
+    (40, 128, 264, 4, 2, B.ROUTE_TOPK, 0.5),      # capacity limit: dropped assignments are skipped in pass 2
+    (48, 64, 72, 3, 1, B.ROUTE_SAMPLE1, 0.0),
+])
+def test_inference_forward_of_a_few_tokens(T, d, F, E, k, routing, cf):
+    """BF16 forward that keeps nothing for backward, at most 64 tokens: every expert's weights meet all tokens
+    (no gather, SwiGLU formed in the first kernel's epilogue, routing beside it).  Compared with the oracle in
+    full, with the forward that saves for backward (other kernels: same routing bits, y within tolerance), and
+    run twice on one workspace (the second call finds the first call's scratch and status word)."""
+    dtype = torch.bfloat16
+    inp = synth.moe_inputs(T, d, F, E, 61, dtype, DEV)
+    bias = synth.normal((E,), 0.3, 61, 77, torch.float32, DEV)
+    noise = synth.gumbel_noise(T, E, 61, DEV) if routing == B.ROUTE_SAMPLE1 else None
+    alpha = 0.0 if routing == B.ROUTE_SAMPLE1 else 0.02
+    kk = E if routing == B.ROUTE_SOFT else k
+    fwd = gpu_forward(inp, k, routing, alpha, bias, save=False, noise=noise, tau=0.8, capacity_factor=cf)
+    check_forward(inp, fwd, kk, routing, alpha, bias, TOL[dtype], noise=noise, tau=0.8, capacity_factor=cf)
+    kept = gpu_forward(inp, k, routing, alpha, bias, save=True, noise=noise, tau=0.8, capacity_factor=cf)
+    for name in ("logits", "topk_idx", "gates", "probs", "perm", "inv_perm", "counts", "u", "p", "lb_loss"):
+        assert torch.equal(getattr(fwd["routing"], name), getattr(kept["routing"], name)), name
+    assert rel_err(np64(fwd["y"]), np64(kept["y"])) <= TOL[dtype]
+    y1 = fwd["y"].clone()
+    r = fwd["routing"]
+    B.btx_moe_forward(fwd["desc"], inp["x"], inp["w_router"], bias, inp["w1"], inp["w3"], inp["w2"], fwd["y"], r, None,
+                      fwd["ws"], router_noise=noise)
+    assert B.btx_device_status(fwd["ws"]) == B.BTX_OK
+    assert torch.equal(fwd["y"], y1)
+
+
 def test_bounded_wait_expires_and_the_context_stays_usable():
     """The safety net of the tensor-core kernels: a device-side wait that nothing will satisfy gives up
     after its limit, the status word reports it, the kernel returns, and later calls work as usual."""
