@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbtx.so")
 SOURCES = ["btx_api.cu", "btx_routing.cu", "btx_merge.cu", "btx_gemm_simt.cu", "btx_gemm_tc.cu", "btx_gemm_decode.cu",
-           "btx_gemm_dense.cu"]
+           "btx_gemm_fused.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

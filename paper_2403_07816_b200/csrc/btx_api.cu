@@ -43,7 +43,7 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   p.r_pad_max = (int)align_up((size_t)p.R + (size_t)p.E * (kRowTile - 1), kRowTile);
   p.mt_max = p.r_pad_max / kRowTile;
   p.nt_dact = desc->dtype == BTX_BF16 ? 2 * ((p.F + 255) / 256) : (p.F + 63) / 64;   // row-dot partials per row
-  p.route_blocks = (p.T + 7) / 8;
+  p.route_blocks = (p.T + 15) / 16;                       // a router block routes 16 tokens at a time
   if (p.route_blocks > kMaxRouteBlocks) p.route_blocks = kMaxRouteBlocks;
   p.perm_blocks = (p.R + 1023) / 1024;
   p.wr_chunks = (p.T + 127) / 128;
@@ -245,17 +245,18 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
   resolve(pl, sv, ws, &b);
 
   mark_stage(0, st);
-  const float* expert_rows = b.yp;
-  int splits = 1;
   if (pl.dense) {
-    // a handful of tokens, nothing kept: the first expert kernel clears the status word and starts at once,
-    // the routing runs beside it, no gather
-    mark_stage(1, st);
-    if ((s = launch_expert_forward_dense_bf16(pl, er.routing, desc->lb_alpha, x, w_router, router_bias, noise, er.inv_tau,
-                                              w1, w3, w2, b, st)) != BTX_OK)
+    // a handful of tokens, nothing kept: the whole layer is one kernel (it clears the status word itself)
+    if ((s = launch_forward_small_fused_bf16(pl, er.routing, desc->lb_alpha, x, w_router, router_bias, noise, er.inv_tau,
+                                             w1, w3, w2, y, b, st)) != BTX_OK)
       return s;
+    mark_stage(4, st);
   } else {
+    const float* expert_rows = b.yp;
+    int splits = 1;
     BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));
+    if (!route_permute_small_fits(pl) && pl.capacity < pl.R)       // the tail of perm past the kept rows reads -1
+      BTX_CUDA_OK(cudaMemsetAsync(b.perm, 0xFF, (size_t)pl.R * sizeof(int32_t), st));
     if (route_permute_small_fits(pl)) {
       BTX_CUDA_OK(launch_route_permute_small(pl, desc->dtype, er.routing, desc->lb_alpha, x, w_router, router_bias, noise,
                                              er.inv_tau, b, st));
@@ -275,10 +276,10 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
     } else {
       if ((s = launch_expert_forward_bf16(pl, w1, w3, w2, b, desc->save_for_backward, st)) != BTX_OK) return s;
     }
+    mark_stage(3, st);
+    BTX_CUDA_OK(launch_combine(pl, desc->dtype, expert_rows, splits, y, b, st));
+    mark_stage(4, st);
   }
-  mark_stage(3, st);
-  BTX_CUDA_OK(launch_combine(pl, desc->dtype, expert_rows, splits, y, b, st));
-  mark_stage(4, st);
 
   if (routing) {
     auto out = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {

@@ -83,11 +83,6 @@ bool route_permute_small_fits(const Plan& pl);
 cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, float alpha, const void* x,
                                        const void* w_router, const float* bias, const float* noise, float inv_tau,
                                        const Buffers& b, cudaStream_t st);
-// The same by one cluster of blocks, launched as a programmatic dependent of the first kernel of the dense
-// small-batch forward, beside which it runs (BF16).
-cudaError_t launch_route_permute_cluster(const Plan& pl, int routing, float alpha, const void* x, const void* w_router,
-                                       const float* bias, const float* noise, float inv_tau, const Buffers& b,
-                                       cudaStream_t st);
 cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st);
 // y[t] = sum over slots and over `splits` partial copies ([split][R][d]) of the expert rows
 cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, const Buffers& b,
@@ -108,13 +103,13 @@ btx_status launch_expert_forward_bf16(const Plan& pl, const void* w1, const void
 int pick_decode_splits(int base_tiles, int kb_total);
 btx_status launch_expert_forward_small_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                             const Buffers& b, int save, cudaStream_t st);
-// Forward for at most 64 tokens when nothing is kept for backward: act[e] = SwiGLU(x W1_e^T, x W3_e^T) for every
-// expert and all tokens, the routing beside it, then the gate-scaled rows W2_e act[e][t] of the selected
-// (token, expert) pairs.
+// Whole forward for at most 64 tokens when nothing is kept for backward, as one cooperative kernel: routing,
+// act[e] = SwiGLU(x W1_e^T, x W3_e^T) for every expert and all tokens, the gate-scaled rows W2_e act[e][t] of the
+// selected (token, expert) pairs, and their sum y.  Clears the status word itself.
 bool dense_small_fits(const Plan& pl, int save_for_backward);
-btx_status launch_expert_forward_dense_bf16(const Plan& pl, int routing, float alpha, const void* x, const void* w_router,
-                                            const float* bias, const float* noise, float inv_tau, const void* w1,
-                                            const void* w3, const void* w2, const Buffers& b, cudaStream_t st);
+btx_status launch_forward_small_fused_bf16(const Plan& pl, int routing, float alpha, const void* x, const void* w_router,
+                                           const float* bias, const float* noise, float inv_tau, const void* w1,
+                                           const void* w3, const void* w2, void* y, const Buffers& b, cudaStream_t st);
 btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const void* w3, const void* w2,
                                        const Buffers& b, float* dw1, float* dw3, float* dw2, int accumulate,
                                        int skip_wgrad, cudaEvent_t after_dx, cudaStream_t st);

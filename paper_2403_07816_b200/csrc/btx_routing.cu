@@ -10,138 +10,85 @@
 //   gather      rows of x (or dy) copied into the padded expert-sorted layout
 //   combine     y_t = sum over slots of the gate-scaled expert rows
 //   router bwd  d logits from d gates and the two L_LB terms; dW_l = dz^T x; dx += W_l^T dz
-#include "btx_common.cuh"
+#include "btx_route_dev.cuh"
 
 namespace btx {
 
 namespace {
+
+using namespace routedev;
 
 constexpr int kRouterThreads = 256;
 constexpr int kRouterWarps = kRouterThreads / 32;
 constexpr int kPermThreads = 256;
 constexpr int kPermChunk = 1024;      // assignments per block of the permutation kernels
 
-template <typename T> struct Vec;     // 16-byte vectors of the element type
-template <> struct Vec<float> {
-  static constexpr int N = 4;
-  static __device__ __forceinline__ void load(const float* p, float (&v)[4]) {
-    float4 q = *reinterpret_cast<const float4*>(p);
-    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
-  }
-};
-template <> struct Vec<__nv_bfloat16> {
-  static constexpr int N = 8;
-  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8]) {
-    uint4 q = *reinterpret_cast<const uint4*>(p);
-    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&q);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float2 f = __bfloat1622float2(h[i]);
-      v[2 * i] = f.x; v[2 * i + 1] = f.y;
-    }
-  }
-};
-
 // ---------------------------------------------------------------------------------------------
 // Router
 // ---------------------------------------------------------------------------------------------
-// Selection, gates and softmax for one token from the logits z[0..E) in shared memory (all lanes of
-// the calling warp take part).  The experts are chosen on z as it stands; the softmaxes are those of
-// z * scale (scale = 1 except for Sample Top-1, whose temperature must not touch the arg-max: a
-// rounded product could merge two distinct perturbed logits into a tie).  On return lane l holds the
-// dense gate and probability of experts l (index 0) and l + 32 (index 1).
-__device__ __forceinline__ void route_select(int t, int E, int k, int routing, float scale, const float* z, int lane,
-                                             int32_t* __restrict__ topk,
-                                             float* __restrict__ gates, float* __restrict__ probs, float (&my_g)[2],
-                                             float (&my_p)[2]) {
-  unsigned long long taken = 0;
-  int sel[kMaxExperts];
-  int first = 0;
-  // repeated arg-max: strict '>' keeps the lower index on ties
-  for (int j = 0; j < k; ++j) {
-    int best = -1;
-    float zb = 0.f;
-    for (int e = 0; e < E; ++e) {
-      if ((taken >> e) & 1ull) continue;
-      float ze = z[e];
-      if (best < 0 || ze > zb) { best = e; zb = ze; }
-    }
-    taken |= 1ull << best;
-    sel[j] = best;
-    if (j == 0) first = best;
-  }
-  const float zmax = z[first];
-  float psum = 0.f;
-  for (int e = 0; e < E; ++e) psum += expf((z[e] - zmax) * scale);
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    const int e = lane + 32 * h;
-    my_p[h] = (e < E) ? expf((z[e] - zmax) * scale) / psum : 0.f;
-    my_g[h] = 0.f;
-  }
-  if (routing == BTX_ROUTE_SWITCH) {
-    float g0 = expf((z[first] - zmax) * scale) / psum;
-    if ((first & 31) == lane) my_g[first >> 5] = g0;
-    if (lane == 0) { topk[t] = first; gates[t] = g0; }
-  } else {
-    float gsum = 0.f;
-    for (int j = 0; j < k; ++j) gsum += expf((z[sel[j]] - zmax) * scale);
-    for (int j = 0; j < k; ++j) {
-      float gj = expf((z[sel[j]] - zmax) * scale) / gsum;
-      if ((sel[j] & 31) == lane) my_g[sel[j] >> 5] = gj;
-      if (lane == 0) { topk[(size_t)t * k + j] = sel[j]; gates[(size_t)t * k + j] = gj; }
-    }
-  }
-#pragma unroll
-  for (int h = 0; h < 2; ++h)
-    if (lane + 32 * h < E) probs[(size_t)t * E + lane + 32 * h] = my_p[h];
-  __syncwarp();
-}
-
-// Routing of one token by one warp: logits (or the given ones), top-k by repeated arg-max with
-// ties to the lower index, gates, full softmax.  `z` is this warp's shared scratch of kMaxExperts
-// floats.  On return lane l holds the dense gate and the probability of experts l and l + 32.
+// Logits of two tokens by one warp (the second may be absent: t1 >= Tn): every lane takes each 32nd
+// 16-byte vector of both rows, so a router row vector fetched from L1 serves two tokens and twice as many
+// loads of x are in flight per warp.  z0/z1: the warp's shared scratch of kMaxExperts floats each.
 template <typename T>
-__device__ __forceinline__ void route_token(int t, int d, int E, int k, int routing, const T* __restrict__ x,
-                                            const T* __restrict__ wr, const float* __restrict__ bias,
-                                            const float* __restrict__ given_logits,
-                                            const float* __restrict__ noise, float inv_tau, float* z, int lane,
-                                            float* __restrict__ logits, int32_t* __restrict__ topk,
-                                            float* __restrict__ gates, float* __restrict__ probs, float (&my_g)[2],
-                                            float (&my_p)[2]) {
+__device__ __forceinline__ void route_logits2(int t0, bool two, int d, int E, const T* __restrict__ x,
+                                              const T* __restrict__ wr, const float* __restrict__ bias,
+                                              const float* __restrict__ given_logits, float* z0, float* z1, int lane) {
   constexpr int VN = Vec<T>::N;
   if (given_logits != nullptr) {
-    for (int e = lane; e < E; e += 32) z[e] = given_logits[(size_t)t * E + e] + (bias ? bias[e] : 0.f);
-  } else {
-    const T* xr = x + (size_t)t * d;
-    for (int eb = 0; eb < E; eb += 8) {
-      float acc[8];
+    for (int e = lane; e < E; e += 32) {
+      const float b = bias ? bias[e] : 0.f;
+      z0[e] = given_logits[(size_t)t0 * E + e] + b;
+      if (two) z1[e] = given_logits[(size_t)(t0 + 1) * E + e] + b;
+    }
+    return;
+  }
+  const T* x0 = x + (size_t)t0 * d;
+  const T* x1 = two ? x0 + d : x0;
+  for (int eb = 0; eb < E; eb += 8) {
+    float a0[8], a1[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    for (int j = 0; j < 8; ++j) { a0[j] = 0.f; a1[j] = 0.f; }
 #pragma unroll 2
-      for (int c = lane * VN; c < d; c += 32 * VN) {
-        float xv[VN];
-        Vec<T>::load(xr + c, xv);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (eb + j < E) {
-            float wv[VN];
-            Vec<T>::load(wr + (size_t)(eb + j) * d + c, wv);
-#pragma unroll
-            for (int v = 0; v < VN; ++v) acc[j] = fmaf(xv[v], wv[v], acc[j]);
-          }
-        }
-      }
+    for (int c = lane * VN; c < d; c += 32 * VN) {
+      float u0[VN], u1[VN];
+      Vec<T>::load(x0 + c, u0);
+      Vec<T>::load(x1 + c, u1);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        float a = acc[j];
+        if (eb + j < E) {
+          float wv[VN];
+          Vec<T>::load(wr + (size_t)(eb + j) * d + c, wv);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-        if (lane == 0 && eb + j < E) z[eb + j] = a + (bias ? bias[eb + j] : 0.f);
+          for (int v = 0; v < VN; ++v) { a0[j] = fmaf(u0[v], wv[v], a0[j]); a1[j] = fmaf(u1[v], wv[v], a1[j]); }
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (eb + j < E) {
+        float s0 = a0[j], s1 = a1[j];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          s0 += __shfl_xor_sync(0xffffffffu, s0, o);
+          s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+        }
+        if (lane == 0) {
+          const float b = bias ? bias[eb + j] : 0.f;
+          z0[eb + j] = s0 + b;
+          z1[eb + j] = s1 + b;
+        }
       }
     }
   }
-  __syncwarp();
+}
+
+// Stores the (unperturbed) logits of token t, adds the Sample Top-1 noise, and routes: top-k by repeated
+// arg-max with ties to the lower index, gates, full softmax.  On return lane l holds the dense gate and the
+// probability of experts l and l + 32.
+__device__ __forceinline__ void route_finish_token(int t, int E, int k, int routing, const float* __restrict__ noise,
+                                                   float inv_tau, float* z, int lane, float* __restrict__ logits,
+                                                   int32_t* __restrict__ topk, float* __restrict__ gates,
+                                                   float* __restrict__ probs, float (&my_g)[2], float (&my_p)[2]) {
   for (int e = lane; e < E; e += 32) {
     logits[(size_t)t * E + e] = z[e];                             // reported logits are unperturbed
     if (noise != nullptr) z[e] = z[e] + noise[(size_t)t * E + e]; // one fp32 addition decides the expert
@@ -150,46 +97,17 @@ __device__ __forceinline__ void route_token(int t, int d, int E, int k, int rout
   route_select(t, E, k, routing, noise != nullptr ? inv_tau : 1.0f, z, lane, topk, gates, probs, my_g, my_p);
 }
 
-template <typename T>
-__global__ void __launch_bounds__(kRouterThreads, 4)      // at most 64 registers: the x stream needs the occupancy
-router_kernel(int Tn, int d, int E, int k, int routing, const T* __restrict__ x, const T* __restrict__ wr,
-              const float* __restrict__ bias, const float* __restrict__ given_logits,
-              const float* __restrict__ noise, float inv_tau,
-              float* __restrict__ logits, int32_t* __restrict__ topk, float* __restrict__ gates,
-              float* __restrict__ probs, float* __restrict__ route_part) {
-  __shared__ float zs[kRouterWarps][kMaxExperts];
-  __shared__ float red[kRouterWarps][kMaxExperts][2];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  float u_acc[2] = {0.f, 0.f}, p_acc[2] = {0.f, 0.f};   // lane l accumulates experts l and l + 32 over this warp's tokens
-  for (int t = blockIdx.x * kRouterWarps + warp; t < Tn; t += gridDim.x * kRouterWarps) {
-    float my_g[2], my_p[2];
-    route_token<T>(t, d, E, k, routing, x, wr, bias, given_logits, noise, inv_tau, zs[warp], lane, logits, topk, gates,
-                   probs, my_g, my_p);
-#pragma unroll
-    for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
-  }
-#pragma unroll
-  for (int h = 0; h < 2; ++h)
-    if (lane + 32 * h < E) { red[warp][lane + 32 * h][0] = u_acc[h]; red[warp][lane + 32 * h][1] = p_acc[h]; }
-  __syncthreads();
-  if (threadIdx.x < 2 * E) {
-    int e = threadIdx.x >> 1, which = threadIdx.x & 1;
-    float s = 0.f;
-    for (int w = 0; w < kRouterWarps; ++w) s += red[w][e][which];
-    route_part[(size_t)blockIdx.x * 2 * E + threadIdx.x] = s;
-  }
-}
-
-// One warp per (expert, u|p) pair: lanes sum strided block partials in double, then a fixed-order
-// shuffle tree, so the result does not depend on scheduling.
-__global__ void __launch_bounds__(256)
-lb_finalize_kernel(int Tn, int E, int nblocks, float alpha, const float* __restrict__ route_part,
-                   float* __restrict__ u, float* __restrict__ p, float* __restrict__ loss, double* __restrict__ up64) {
+// u, p and L_LB = alpha E sum_i u_i p_i from the per-block partial sums, by one block of 256 threads: one warp
+// per (expert, u|p) pair, lanes sum strided block partials in double, then a fixed-order shuffle tree, so the
+// result does not depend on scheduling.
+__device__ __forceinline__ void lb_finalize(int Tn, int E, int nblocks, float alpha, const float* route_part,
+                                            float* __restrict__ u, float* __restrict__ p, float* __restrict__ loss,
+                                            double* __restrict__ up64) {
   __shared__ double su[kMaxExperts], sp[kMaxExperts];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int pair = warp; pair < 2 * E; pair += 8) {
+  for (int pair = warp; pair < 2 * E; pair += kRouterWarps) {
     double s = 0.0;
-    for (int b = lane; b < nblocks; b += 32) s += (double)route_part[(size_t)b * 2 * E + pair];
+    for (int b = lane; b < nblocks; b += 32) s += (double)__ldcg(route_part + (size_t)b * 2 * E + pair);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     s /= (double)Tn;
@@ -206,14 +124,66 @@ lb_finalize_kernel(int Tn, int E, int nblocks, float alpha, const float* __restr
   }
 }
 
+// One warp per pair of tokens.  Every block leaves its partial sums of the gates and probabilities; the block
+// that finishes last (a ticket in the workspace status block, zero when the kernel starts) forms the batch
+// means and the loss from all of them.
+template <typename T>
+__global__ void __launch_bounds__(kRouterThreads, 4)      // at most 64 registers: the x stream needs the occupancy
+router_kernel(int Tn, int d, int E, int k, int routing, float alpha, const T* __restrict__ x, const T* __restrict__ wr,
+              const float* __restrict__ bias, const float* __restrict__ given_logits,
+              const float* __restrict__ noise, float inv_tau,
+              float* __restrict__ logits, int32_t* __restrict__ topk, float* __restrict__ gates,
+              float* __restrict__ probs, float* route_part, float* __restrict__ u, float* __restrict__ p,
+              float* __restrict__ loss, double* __restrict__ up64, int32_t* ticket) {
+  __shared__ float zs[kRouterWarps][2][kMaxExperts];
+  __shared__ float red[kRouterWarps][kMaxExperts][2];
+  __shared__ int is_last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  allow_dependents();
+  float u_acc[2] = {0.f, 0.f}, p_acc[2] = {0.f, 0.f};   // lane l accumulates experts l and l + 32 over this warp's tokens
+  for (int t = (blockIdx.x * kRouterWarps + warp) * 2; t < Tn; t += gridDim.x * kRouterWarps * 2) {
+    const bool two = t + 1 < Tn;
+    route_logits2<T>(t, two, d, E, x, wr, bias, given_logits, zs[warp][0], zs[warp][1], lane);
+    __syncwarp();
+    float my_g[2], my_p[2];
+    route_finish_token(t, E, k, routing, noise, inv_tau, zs[warp][0], lane, logits, topk, gates, probs, my_g, my_p);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
+    if (two) {
+      route_finish_token(t + 1, E, k, routing, noise, inv_tau, zs[warp][1], lane, logits, topk, gates, probs, my_g, my_p);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
+    }
+  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+    if (lane + 32 * h < E) { red[warp][lane + 32 * h][0] = u_acc[h]; red[warp][lane + 32 * h][1] = p_acc[h]; }
+  __syncthreads();
+  if (threadIdx.x < 2 * E) {
+    int e = threadIdx.x >> 1, which = threadIdx.x & 1;
+    float s = 0.f;
+    for (int w = 0; w < kRouterWarps; ++w) s += red[w][e][which];
+    route_part[(size_t)blockIdx.x * 2 * E + threadIdx.x] = s;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  lb_finalize(Tn, E, (int)gridDim.x, alpha, route_part, u, p, loss, up64);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Permutation
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kPermThreads)
 perm_count_kernel(int R, int E, int nblocks, const int32_t* __restrict__ topk, int32_t* __restrict__ perm_counts) {
   __shared__ int hist[kMaxExperts];
+  allow_dependents();
   if (threadIdx.x < kMaxExperts) hist[threadIdx.x] = 0;
   __syncthreads();
+  grid_dependency_wait();
   int base = blockIdx.x * kPermChunk;
   int end = min(R, base + kPermChunk);
   for (int i = base + threadIdx.x; i < end; i += kPermThreads) atomicAdd(&hist[topk[i]], 1);
@@ -228,6 +198,8 @@ __global__ void perm_scan_kernel(int E, int nblocks, int mt_max, int cap, const 
   __shared__ int scnt[kMaxExperts];
   __shared__ int spad[kMaxExperts + 1];
   int tid = threadIdx.x;
+  allow_dependents();
+  grid_dependency_wait();
   if (tid < E) {
     int run = 0;
     for (int b = 0; b < nblocks; ++b) {
@@ -258,16 +230,30 @@ __global__ void perm_scan_kernel(int E, int nblocks, int mt_max, int cap, const 
 }
 
 __global__ void __launch_bounds__(kPermThreads)
-perm_scatter_kernel(int R, int E, int nblocks, int cap, const int32_t* __restrict__ topk,
-                    const int32_t* __restrict__ perm_base,
+perm_scatter_kernel(int R, int E, int nblocks, int cap, int r_pad_max, const int32_t* __restrict__ topk,
+                    const int32_t* __restrict__ perm_base, const int32_t* __restrict__ counts,
                     const int32_t* __restrict__ offsets, const int32_t* __restrict__ pad_offsets,
                     int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
                     int32_t* __restrict__ flat2row) {
   constexpr int NW = kPermThreads / 32;
   __shared__ int running[kMaxExperts + 1];
   __shared__ int wcnt[NW][kMaxExperts + 1];
+  __shared__ int spad[kMaxExperts + 1], scnt[kMaxExperts];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  allow_dependents();
+  grid_dependency_wait();
   if (threadIdx.x < E) running[threadIdx.x] = perm_base[threadIdx.x * nblocks + blockIdx.x];
+  if (threadIdx.x <= E) spad[threadIdx.x] = pad_offsets[threadIdx.x];
+  if (threadIdx.x < E) scnt[threadIdx.x] = counts[threadIdx.x];
+  __syncthreads();
+  // padding rows (behind an expert's last real row, and behind the last expert) map to no assignment;
+  // the real rows are written below, by whichever block holds their assignment
+  for (int rp = blockIdx.x * kPermThreads + threadIdx.x; rp < r_pad_max; rp += gridDim.x * kPermThreads) {
+    bool real = false;
+    for (int e = 0; e < E; ++e)
+      if (rp >= spad[e] && rp < spad[e] + scnt[e]) real = true;
+    if (!real) rowmap[rp] = -1;
+  }
   const int base = blockIdx.x * kPermChunk;
   const int end = min(R, base + kPermChunk);
   for (int r0 = base; r0 < end; r0 += kPermThreads) {
@@ -310,140 +296,6 @@ perm_scatter_kernel(int R, int E, int nblocks, int cap, const int32_t* __restric
 // instead of six.  (The workspace status block is zeroed at the start of every forward call; its
 // word 8 is the ticket counter.)
 // ---------------------------------------------------------------------------------------------
-constexpr int kSmallThreads = 256;
-constexpr int kSmallMaxR = 1024;
-
-// Batch means u and p, the loss, and the permutation of a small batch (R <= 1024) by ONE block of THREADS
-// threads, from the per-token routing results already in global memory.  Every sum runs in a fixed
-// order, so the result does not depend on which block runs this or on how many threads it has.
-template <int THREADS>
-__device__ __forceinline__ void small_batch_finish(int Tn, int E, int k, float alpha, int mt_max, int r_pad_max, int cap,
-                                                   const int32_t* topk, const float* gates, const float* probs,
-                                                   float* __restrict__ u, float* __restrict__ p,
-                                                   double* __restrict__ up64, float* __restrict__ loss,
-                                                   int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
-                                                   int32_t* __restrict__ pad_offsets, int32_t* __restrict__ tile_expert,
-                                                   int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
-                                                   int32_t* __restrict__ rowmap, int32_t* __restrict__ flat2row) {
-  constexpr int NW = THREADS / 32;
-  __shared__ double su[kMaxExperts], sp[kMaxExperts];
-  __shared__ int hist[kMaxExperts + 1], running[kMaxExperts + 1], soff[kMaxExperts + 1], spad[kMaxExperts + 1];
-  __shared__ int wcnt[NW][kMaxExperts + 1];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int R = Tn * k;
-  // ---- last block: batch means, loss ----
-  for (int e = warp; e < E; e += NW) {
-    double du = 0.0, dp = 0.0;
-    for (int tt = lane; tt < Tn; tt += 32) {
-      dp += (double)__ldcg(probs + (size_t)tt * E + e);
-      for (int sl = 0; sl < k; ++sl)
-        if (__ldcg(topk + (size_t)tt * k + sl) == e) du += (double)__ldcg(gates + (size_t)tt * k + sl);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      du += __shfl_xor_sync(0xffffffffu, du, o);
-      dp += __shfl_xor_sync(0xffffffffu, dp, o);
-    }
-    if (lane == 0) {
-      du /= (double)Tn; dp /= (double)Tn;
-      su[e] = du; sp[e] = dp; u[e] = (float)du; p[e] = (float)dp; up64[e] = du; up64[E + e] = dp;
-    }
-  }
-  // ---- permutation: histogram, scan, stable scatter in rounds of one block ----
-  if (threadIdx.x <= kMaxExperts) hist[threadIdx.x] = 0;
-  for (int j = threadIdx.x; j < r_pad_max; j += THREADS) rowmap[j] = -1;
-  if (cap < R)
-    for (int j = threadIdx.x; j < R; j += THREADS) perm[j] = -1;
-  __syncthreads();
-  for (int i = threadIdx.x; i < R; i += THREADS) atomicAdd(&hist[__ldcg(topk + i)], 1);
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double acc = 0.0;
-    for (int q = 0; q < E; ++q) acc += su[q] * sp[q];
-    loss[0] = (float)((double)alpha * (double)E * acc);
-    int o = 0, po = 0;
-    for (int q = 0; q < E; ++q) {
-      const int c = min(hist[q], cap);
-      counts[q] = c; offsets[q] = o; pad_offsets[q] = po; soff[q] = o; spad[q] = po; running[q] = 0;
-      o += c;
-      po += (c + kRowTile - 1) / kRowTile * kRowTile;
-    }
-    offsets[E] = o; pad_offsets[E] = po; soff[E] = o; spad[E] = po;
-  }
-  __syncthreads();
-  for (int mt = threadIdx.x; mt < mt_max; mt += THREADS) {
-    const int row = mt * kRowTile;
-    int ex = -1;
-    for (int q = 0; q < E; ++q)
-      if (row >= spad[q] && row < spad[q + 1]) ex = q;
-    tile_expert[mt] = ex;
-  }
-  for (int r0 = 0; r0 < R; r0 += THREADS) {
-    for (int j = threadIdx.x; j < NW * (kMaxExperts + 1); j += THREADS) (&wcnt[0][0])[j] = 0;
-    __syncthreads();
-    const int i = r0 + threadIdx.x;
-    const int e = (i < R) ? __ldcg(topk + i) : E;       // E = dummy bucket for idle lanes
-    const unsigned same = __match_any_sync(0xffffffffu, e);
-    const int rank = __popc(same & ((1u << lane) - 1u));
-    if (rank == 0) wcnt[warp][e] = __popc(same);
-    __syncthreads();
-    if (i < R) {
-      int before = 0;
-      for (int w = 0; w < warp; ++w) before += wcnt[w][e];
-      const int within = running[e] + before + rank;
-      if (within < cap) {
-        const int r = soff[e] + within, rp = spad[e] + within;
-        perm[r] = i; inv_perm[i] = r; rowmap[rp] = i; flat2row[i] = rp;
-      } else {
-        inv_perm[i] = -1; flat2row[i] = -1;
-      }
-    }
-    __syncthreads();
-    if (threadIdx.x < E) {
-      int sum = 0;
-      for (int w = 0; w < NW; ++w) sum += wcnt[w][threadIdx.x];
-      running[threadIdx.x] += sum;
-    }
-    __syncthreads();
-  }
-}
-
-
-// Logits of one token by eight warps that share its row: warp w takes every eighth 16-byte vector,
-// part[w][e] receives its share of <x_t, W_l[e]>; the caller adds the eight parts in warp order.
-template <typename T>
-__device__ __forceinline__ void token_logit_parts(const T* __restrict__ xr, const T* __restrict__ wr, int d, int E,
-                                                  int warp, int lane, float (*part)[kMaxExperts]) {
-  constexpr int NW = kSmallThreads / 32;
-  constexpr int VN = Vec<T>::N;
-  for (int eb = 0; eb < E; eb += 8) {
-    float acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-#pragma unroll 2
-    for (int c = (warp * 32 + lane) * VN; c < d; c += NW * 32 * VN) {
-      float xv[VN];
-      Vec<T>::load(xr + c, xv);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (eb + j < E) {
-          float wv[VN];
-          Vec<T>::load(wr + (size_t)(eb + j) * d + c, wv);
-#pragma unroll
-          for (int v = 0; v < VN; ++v) acc[j] = fmaf(xv[v], wv[v], acc[j]);
-        }
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      float a = acc[j];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-      if (lane == 0 && eb + j < E) part[warp][eb + j] = a;
-    }
-  }
-}
-
 // One block per token computes its logits (eight warps share the row) and routes it; the block that
 // finishes last (a ticket counter in the workspace status block) then forms u, p, the loss and the
 // permutation.  Every sum runs in a fixed order, so results do not depend on which block is last.
@@ -488,62 +340,9 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
   if (!is_last) return;
   __threadfence();
 
-  small_batch_finish<kSmallThreads>(Tn, E, k, alpha, mt_max, r_pad_max, cap, topk, gates, probs, u, p, up64, loss, counts,
-                                    offsets, pad_offsets, tile_expert, perm, inv_perm, rowmap, flat2row);
-}
-
-// The same routing for a handful of tokens whose expert kernels do not wait for it (they multiply every
-// expert's weights with all tokens and look the routing up in their epilogues): one cluster of eight
-// blocks, each taking every eighth token with the arithmetic of the kernel above; after a cluster
-// barrier the first block forms the batch means, the loss and the permutation.  No ticket is needed.
-// The kernel is launched as a programmatic dependent of the first expert kernel, which lets it start only
-// after everything earlier in the stream is complete; it runs beside that kernel (256 threads of at most
-// 64 registers fit next to one of its blocks) and, its work done, stays parked until that kernel has
-// completed, so that whoever waits for this kernel has waited for both.
-constexpr int kRouteCluster = 8;
-
-template <typename T>
-__global__ void __cluster_dims__(kRouteCluster, 1, 1) __launch_bounds__(kSmallThreads, 4)
-route_permute_cluster_kernel(int Tn, int d, int E, int k, int routing, float alpha, int mt_max, int r_pad_max, int cap,
-                             const T* __restrict__ x, const T* __restrict__ wr, const float* __restrict__ bias,
-                             const float* __restrict__ noise, float inv_tau, float* logits, int32_t* topk, float* gates,
-                             float* probs, float* __restrict__ u, float* __restrict__ p, double* __restrict__ up64,
-                             float* __restrict__ loss, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
-                             int32_t* __restrict__ pad_offsets, int32_t* __restrict__ tile_expert,
-                             int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, int32_t* __restrict__ rowmap,
-                             int32_t* __restrict__ flat2row) {
-  constexpr int NW = kSmallThreads / 32;
-  __shared__ float part[NW][kMaxExperts];
-  __shared__ float z[kMaxExperts];
-  allow_dependents();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int t = blockIdx.x; t < Tn; t += kRouteCluster) {
-    token_logit_parts<T>(x + (size_t)t * d, wr, d, E, warp, lane, part);
-    __syncthreads();
-    if (threadIdx.x < E) {
-      float a = 0.f;
-      for (int w = 0; w < NW; ++w) a += part[w][threadIdx.x];
-      a += bias ? bias[threadIdx.x] : 0.f;
-      logits[(size_t)t * E + threadIdx.x] = a;
-      if (noise != nullptr) a = a + noise[(size_t)t * E + threadIdx.x];
-      z[threadIdx.x] = a;
-    }
-    __syncthreads();
-    if (warp == 0) {
-      float my_g[2], my_p[2];
-      route_select(t, E, k, routing, noise != nullptr ? inv_tau : 1.0f, z, lane, topk, gates, probs, my_g, my_p);
-    }
-    __syncthreads();
-  }
-  // every block's routing results are visible to the first block after the cluster barrier
-  __threadfence();
-  __syncthreads();
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-  if (blockIdx.x == 0)
-    small_batch_finish<kSmallThreads>(Tn, E, k, alpha, mt_max, r_pad_max, cap, topk, gates, probs, u, p, up64, loss, counts,
-                                      offsets, pad_offsets, tile_expert, perm, inv_perm, rowmap, flat2row);
-  grid_dependency_wait();
+  small_batch_finish<kSmallThreads>((int)threadIdx.x, [] { __syncthreads(); }, Tn, E, k, alpha, mt_max, r_pad_max, cap, topk,
+                                    gates, probs, u, p, up64, loss, counts, offsets, pad_offsets, tile_expert, perm,
+                                    inv_perm, rowmap, flat2row);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -581,35 +380,55 @@ template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16*
 
 // y[t, :] = sum_slot sum_split rows[split][t*k + slot, :]   (+ sum_e dz[t,e] * wr[e, :] when dz != nullptr)
 // `kept` (optional): flat assignment -> sorted row; a negative entry is a dropped assignment, whose
-// row was never written and counts as zero.
+// row was never written and counts as zero.  A thread owns 16 bytes of the output row (8 columns in BF16,
+// 4 in FP32), so in BF16 it has two 16-byte loads in flight per slot and stores one whole vector.
 template <typename T>
 __global__ void __launch_bounds__(256)
 combine_kernel(int Tn, int d, int k, int E, int splits, const float* __restrict__ rows, const float* __restrict__ dz,
                const T* __restrict__ wr, const int32_t* __restrict__ kept, T* __restrict__ y) {
+  constexpr int G = Vec<T>::N / 4;                        // float4 groups per thread
   const size_t split_stride = (size_t)Tn * k * d;
-  const int vecs = d >> 2;
+  const int vecs = d / Vec<T>::N;
   allow_dependents();
   grid_dependency_wait();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)Tn * vecs;
        i += (size_t)gridDim.x * blockDim.x) {
-    int t = (int)(i / vecs), c = (int)(i % vecs) * 4;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int t = (int)(i / vecs), c = (int)(i % vecs) * Vec<T>::N;
+    float4 acc[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < k; ++s) {
       if (kept != nullptr && kept[(size_t)t * k + s] < 0) continue;
       for (int sp = 0; sp < splits; ++sp) {
-        float4 v = *reinterpret_cast<const float4*>(rows + sp * split_stride + ((size_t)t * k + s) * d + c);
-        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        const float* r = rows + sp * split_stride + ((size_t)t * k + s) * d + c;
+        float4 v[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) v[g] = *reinterpret_cast<const float4*>(r + 4 * g);
+#pragma unroll
+        for (int g = 0; g < G; ++g) { acc[g].x += v[g].x; acc[g].y += v[g].y; acc[g].z += v[g].z; acc[g].w += v[g].w; }
       }
     }
     if (dz != nullptr) {
       for (int e = 0; e < E; ++e) {
-        float g = dz[(size_t)t * E + e];
-        const T* w = wr + (size_t)e * d + c;
-        acc.x = fmaf(g, to_f32(w[0]), acc.x); acc.y = fmaf(g, to_f32(w[1]), acc.y);
-        acc.z = fmaf(g, to_f32(w[2]), acc.z); acc.w = fmaf(g, to_f32(w[3]), acc.w);
+        const float gz = dz[(size_t)t * E + e];
+        float wv[Vec<T>::N];
+        Vec<T>::load(wr + (size_t)e * d + c, wv);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          acc[g].x = fmaf(gz, wv[4 * g], acc[g].x); acc[g].y = fmaf(gz, wv[4 * g + 1], acc[g].y);
+          acc[g].z = fmaf(gz, wv[4 * g + 2], acc[g].z); acc[g].w = fmaf(gz, wv[4 * g + 3], acc[g].w);
+        }
       }
     }
-    store4<T>(y + (size_t)t * d + c, acc);
+    if (G == 1) {
+      store4<T>(y + (size_t)t * d + c, acc[0]);
+    } else {
+      float f[8] = {acc[0].x, acc[0].y, acc[0].z, acc[0].w, acc[G - 1].x, acc[G - 1].y, acc[G - 1].z, acc[G - 1].w};
+      __nv_bfloat162 h[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) h[j] = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
+      *reinterpret_cast<uint4*>(y + (size_t)t * d + c) = *reinterpret_cast<uint4*>(h);
+    }
   }
 }
 
@@ -772,16 +591,17 @@ router_dw_reduce_kernel(int d, int E, int chunks, const float* __restrict__ part
 cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, const void* x, const void* w_router,
                           const float* bias, const float* given_logits, const float* noise, float inv_tau,
                           const Buffers& b, cudaStream_t st) {
+  // the ticket of the last-block finalisation is word 8 of the status block, zeroed by the caller
   if (dtype == BTX_BF16) {
     router_kernel<__nv_bfloat16><<<pl.route_blocks, kRouterThreads, 0, st>>>(
-        pl.T, pl.d, pl.E, pl.k, routing, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, given_logits,
-        noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.route_part);
+        pl.T, pl.d, pl.E, pl.k, routing, alpha, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias,
+        given_logits, noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.route_part, b.u, b.p, b.loss, b.up64,
+        b.status + 8);
   } else {
     router_kernel<float><<<pl.route_blocks, kRouterThreads, 0, st>>>(
-        pl.T, pl.d, pl.E, pl.k, routing, (const float*)x, (const float*)w_router, bias, given_logits, noise, inv_tau,
-        b.logits, b.topk, b.gates, b.probs, b.route_part);
+        pl.T, pl.d, pl.E, pl.k, routing, alpha, (const float*)x, (const float*)w_router, bias, given_logits, noise,
+        inv_tau, b.logits, b.topk, b.gates, b.probs, b.route_part, b.u, b.p, b.loss, b.up64, b.status + 8);
   }
-  lb_finalize_kernel<<<1, 256, 0, st>>>(pl.T, pl.E, pl.route_blocks, alpha, b.route_part, b.u, b.p, b.loss, b.up64);
   return cudaGetLastError();
 }
 
@@ -804,44 +624,34 @@ cudaError_t launch_route_permute_small(const Plan& pl, int dtype, int routing, f
   return cudaGetLastError();
 }
 
-cudaError_t launch_route_permute_cluster(const Plan& pl, int routing, float alpha, const void* x, const void* w_router,
-                                       const float* bias, const float* noise, float inv_tau, const Buffers& b,
-                                       cudaStream_t st) {
-  return launch_after_predecessor(route_permute_cluster_kernel<__nv_bfloat16>, dim3(kRouteCluster), dim3(kSmallThreads), 0, st, true,
-                                  pl.T, pl.d, pl.E, pl.k, routing, alpha, pl.mt_max, pl.r_pad_max, pl.capacity,
-                                  (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias, noise, inv_tau, b.logits,
-                                  b.topk, b.gates, b.probs, b.u, b.p, b.up64, b.loss, b.counts, b.offsets, b.pad_offsets,
-                                  b.tile_expert, b.perm, b.inv_perm, b.rowmap, b.flat2row);
-}
-
+// The three kernels follow the router kernel as programmatic dependents of one another (each waits for the one
+// before it prior to reading).  Under a capacity limit the caller has filled perm with -1 beforehand.
 cudaError_t launch_permute(const Plan& pl, const Buffers& b, cudaStream_t st) {
-  cudaError_t e = cudaMemsetAsync(b.rowmap, 0xFF, (size_t)pl.r_pad_max * sizeof(int32_t), st);
+  cudaError_t e = launch_after_predecessor(perm_count_kernel, dim3(pl.perm_blocks), dim3(kPermThreads), 0, st, true, pl.R,
+                                           pl.E, pl.perm_blocks, (const int32_t*)b.topk, b.perm_counts);
   if (e != cudaSuccess) return e;
-  if (pl.capacity < pl.R) {      // the tail of perm past the kept rows reads -1
-    e = cudaMemsetAsync(b.perm, 0xFF, (size_t)pl.R * sizeof(int32_t), st);
-    if (e != cudaSuccess) return e;
-  }
-  perm_count_kernel<<<pl.perm_blocks, kPermThreads, 0, st>>>(pl.R, pl.E, pl.perm_blocks, b.topk, b.perm_counts);
-  perm_scan_kernel<<<1, 256, 0, st>>>(pl.E, pl.perm_blocks, pl.mt_max, pl.capacity, b.perm_counts, b.perm_base, b.counts,
-                                      b.offsets, b.pad_offsets, b.tile_expert);
-  perm_scatter_kernel<<<pl.perm_blocks, kPermThreads, 0, st>>>(pl.R, pl.E, pl.perm_blocks, pl.capacity, b.topk, b.perm_base,
-                                                               b.offsets, b.pad_offsets, b.perm, b.inv_perm, b.rowmap,
-                                                               b.flat2row);
-  return cudaGetLastError();
+  e = launch_after_predecessor(perm_scan_kernel, dim3(1), dim3(256), 0, st, true, pl.E, pl.perm_blocks, pl.mt_max,
+                               pl.capacity, (const int32_t*)b.perm_counts, b.perm_base, b.counts, b.offsets,
+                               b.pad_offsets, b.tile_expert);
+  if (e != cudaSuccess) return e;
+  return launch_after_predecessor(perm_scatter_kernel, dim3(pl.perm_blocks), dim3(kPermThreads), 0, st, true, pl.R, pl.E,
+                                  pl.perm_blocks, pl.capacity, pl.r_pad_max, (const int32_t*)b.topk,
+                                  (const int32_t*)b.perm_base, (const int32_t*)b.counts, (const int32_t*)b.offsets,
+                                  (const int32_t*)b.pad_offsets, b.perm, b.inv_perm, b.rowmap, b.flat2row);
 }
 
 cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted, const Buffers& b, cudaStream_t st) {
   int row_vecs = pl.d * pl.esize / 16;
   int blocks = min(pl.r_pad_max / 8, sm_count() * 16);
-  // small batches: the gather's launch overlaps the routing kernel's run
-  return launch_after_predecessor(gather_rows_kernel, dim3(blocks), dim3(256), 0, st, pl.small != 0, pl.k, row_vecs,
+  // the gather's launch overlaps the run of the kernel before it
+  return launch_after_predecessor(gather_rows_kernel, dim3(blocks), dim3(256), 0, st, true, pl.k, row_vecs,
                                   (const uint4*)src, (uint4*)dst_sorted, (const int32_t*)b.rowmap,
                                   (const int32_t*)b.pad_offsets, pl.E);
 }
 
 cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, const Buffers& b,
                            cudaStream_t st) {
-  size_t n = (size_t)pl.T * (pl.d / 4);
+  size_t n = (size_t)pl.T * (pl.d / (dtype == BTX_BF16 ? 8 : 4));
   int blocks = (int)min((n + 255) / 256, (size_t)sm_count() * 32);
   const int32_t* kept = pl.capped ? b.flat2row : nullptr;
   if (dtype == BTX_BF16)
@@ -865,7 +675,7 @@ cudaError_t launch_router_backward(const Plan& pl, int dtype, int routing, float
   const int vn = dtype == BTX_BF16 ? 8 : 4;
   dim3 grid(pl.wr_chunks, (pl.d / vn + 127) / 128);
   float* bias_part = b.dwr_part + (size_t)pl.wr_chunks * pl.E * pl.d;
-  size_t n = (size_t)pl.T * (pl.d / 4);
+  size_t n = (size_t)pl.T * (pl.d / vn);
   int cblocks = (int)min((n + 255) / 256, (size_t)sm_count() * 32);
   const int32_t* kept = pl.capped ? b.flat2row : nullptr;
   if (dtype == BTX_BF16) {

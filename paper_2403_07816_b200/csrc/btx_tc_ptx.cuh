@@ -77,9 +77,11 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out of time).
+// Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out of time).  The first
+// wait of a call that runs out also leaves `site` (which wait, where: the caller's code) in status word 1,
+// which the kernel that clears the status word clears as well.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                          unsigned long long limit_ns = kWaitLimitNs) {
+                                          unsigned long long limit_ns = kWaitLimitNs, int site = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
@@ -88,6 +90,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       if (global_ns() - t0 > limit_ns) {
         *abort_flag = 1;
+        if (site != 0) atomicCAS(status + 1, 0, site);
         atomicExch(status, (int32_t)BTX_ERR_TIMEOUT);
         return false;
       }
