@@ -521,7 +521,7 @@ def run_moe(args, workload):
     dev = torch.device("cuda", local)
     peaks = load_peaks()
     K, W = args.steps, max(args.warmup, 3)
-    soak_s = 0.0 if args.tokens or args.layers else SOAK_S        # profiler captures run few launches
+    soak_s = 0.0 if args.tokens or args.layers else args.soak_s    # profiler captures run few launches
 
     run = MoeRun(workload, dev, rank, tokens=args.tokens, layers=args.layers)
     ms, clocks, stages, soaked = time_moe(run, K, W, world, local, soak_s, with_stages=True)
@@ -662,6 +662,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sub", action="store_true", help="headline only: skip the other configurations")
+    ap.add_argument("--soak-s", type=float, default=SOAK_S, help="untimed run of the step before the warm-up, seconds")
     ap.add_argument("--layers", type=int, default=0, help="decode: number of layers (profiling only)")
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling only; not a bench number)")
     args = ap.parse_args()

@@ -68,6 +68,7 @@ struct TcParams {
   float* of;
   float* dg_part;
   int save, accumulate;
+  int a_one, b_one;             // the MN-major A / B tile of a stage is one TMA box (chunked tensor map)
   int wide;                     // all epilogue rows start on 32-byte boundaries
   int32_t* status;
   int32_t* next_tile;           // tile counter of this launch (zero when the kernel starts)
@@ -232,24 +233,40 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             tma_load_3d(sB, &tmB0, kb * BK, tl.nt * BN + (int)rank * 128, tl.e, full);
           } else if (MODE == G_DACT) {
             tma_load_2d(sA, &tmA0, kb * BK, m0, full);
+            if (p.b_one) {
+              tma_load_4d(sB, &tmB0, 0, kb * BK, tl.nt * (BN / 64) + (int)rank * 2, tl.e, full);
+            } else {
 #pragma unroll
-            for (int j = 0; j < 2; ++j)
-              tma_load_3d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + ((int)rank * 2 + j) * 64, kb * BK, tl.e, full);
+              for (int j = 0; j < 2; ++j)
+                tma_load_3d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + ((int)rank * 2 + j) * 64, kb * BK, tl.e, full);
+            }
           } else if (MODE == G_DX) {
             const bool second = kb >= p.kb_half;
             const int kk = (second ? kb - p.kb_half : kb) * BK;
             tma_load_2d(sA, second ? &tmA1 : &tmA0, kk, m0, full);
+            if (p.b_one) {
+              tma_load_4d(sB, second ? &tmB1 : &tmB0, 0, kk, tl.nt * (BN / 64) + (int)rank * 2, tl.e, full);
+            } else {
 #pragma unroll
-            for (int j = 0; j < 2; ++j)
-              tma_load_3d(sB + j * CHUNK_BYTES, second ? &tmB1 : &tmB0, tl.nt * BN + ((int)rank * 2 + j) * 64, kk, tl.e,
-                          full);
+              for (int j = 0; j < 2; ++j)
+                tma_load_3d(sB + j * CHUNK_BYTES, second ? &tmB1 : &tmB0, tl.nt * BN + ((int)rank * 2 + j) * 64, kk, tl.e,
+                            full);
+            }
           } else {
             const int row = tl.k_base + kb * BK;
+            if (p.a_one) {
+              tma_load_3d(sA, &tmA0, 0, row, m0 / 64, full);
+            } else {
 #pragma unroll
-            for (int j = 0; j < 2; ++j) tma_load_2d(sA + j * CHUNK_BYTES, &tmA0, m0 + j * 64, row, full);
+              for (int j = 0; j < 2; ++j) tma_load_2d(sA + j * CHUNK_BYTES, &tmA0, m0 + j * 64, row, full);
+            }
+            if (p.b_one) {
+              tma_load_3d(sB, &tmB0, 0, row, tl.nt * (BN / 64) + (int)rank * 2, full);
+            } else {
 #pragma unroll
-            for (int j = 0; j < 2; ++j)
-              tma_load_2d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + ((int)rank * 2 + j) * 64, row, full);
+              for (int j = 0; j < 2; ++j)
+                tma_load_2d(sB + j * CHUNK_BYTES, &tmB0, tl.nt * BN + ((int)rank * 2 + j) * 64, row, full);
+            }
           }
           ++uses;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -530,7 +547,9 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   btx_status s;
   TcParams p = base_params(pl, b);
   // dgrad-2: dA' = dYs W2 (W2[d,F] read N-major), SwiGLU backward epilogue
-  if (!make_map(&a0, b.dys, d, RP, 0, 64, 128) || !make_map(&b0, w2, F, d, E, 64, 64)) return BTX_ERR_CUDA;
+  if (!make_map(&a0, b.dys, d, RP, 0, 64, 128)) return BTX_ERR_CUDA;
+  p.b_one = make_map_mn(&b0, w2, F, d, E);
+  if (!p.b_one && !make_map(&b0, w2, F, d, E, 64, 64)) return BTX_ERR_CUDA;
   p.n_tiles = (pl.F + BN - 1) / BN; p.kb_total = (pl.d + BK - 1) / BK; p.N = pl.F;
   p.h1 = (const __nv_bfloat16*)b.h1; p.h3 = (const __nv_bfloat16*)b.h3;
   p.o0 = (__nv_bfloat16*)b.dh1; p.o1 = (__nv_bfloat16*)b.dh3; p.o2 = (__nv_bfloat16*)b.ga; p.dg_part = b.dg_part;
@@ -538,9 +557,9 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   if ((s = launch_tc<G_DACT>(a0, a0, b0, b0, p, pl.mt_max * p.n_tiles, 0, st)) != BTX_OK) return s;
   mark_stage(2, st);
   // dgrad-1: dXs = dh1 W1 + dh3 W3 (weights read N-major), scatter to t*k+slot rows
-  if (!make_map(&a0, b.dh1, F, RP, 0, 64, 128) || !make_map(&a1, b.dh3, F, RP, 0, 64, 128) ||
-      !make_map(&b0, w1, d, F, E, 64, 64) || !make_map(&b1, w3, d, F, E, 64, 64))
-    return BTX_ERR_CUDA;
+  if (!make_map(&a0, b.dh1, F, RP, 0, 64, 128) || !make_map(&a1, b.dh3, F, RP, 0, 64, 128)) return BTX_ERR_CUDA;
+  p.b_one = make_map_mn(&b0, w1, d, F, E) && make_map_mn(&b1, w3, d, F, E);
+  if (!p.b_one && (!make_map(&b0, w1, d, F, E, 64, 64) || !make_map(&b1, w3, d, F, E, 64, 64))) return BTX_ERR_CUDA;
   p.n_tiles = (pl.d + BN - 1) / BN; p.kb_half = (pl.F + BK - 1) / BK; p.kb_total = 2 * p.kb_half; p.N = pl.d;
   p.of = b.dxp; p.wide = aligned32(b.dxp);
   if ((s = launch_tc<G_DX>(a0, a1, b0, b1, p, pl.mt_max * p.n_tiles, 1, st)) != BTX_OK) return s;
@@ -551,12 +570,17 @@ btx_status launch_expert_backward_bf16(const Plan& pl, const void* w1, const voi
   // indexed by the gradient's contiguous (column) index goes on the M side, so that the 32 lanes of
   // an epilogue warp write 32 neighbouring columns of one gradient row.
   p.accumulate = accumulate;
-  if (!make_map(&a0, b.ga, F, RP, 0, 64, 64) || !make_map(&b0, b.dys, d, RP, 0, 64, 64)) return BTX_ERR_CUDA;
+  p.a_one = make_map_mn(&a0, b.ga, F, RP, 0);
+  p.b_one = make_map_mn(&b0, b.dys, d, RP, 0);
+  if ((!p.a_one && !make_map(&a0, b.ga, F, RP, 0, 64, 64)) || (!p.b_one && !make_map(&b0, b.dys, d, RP, 0, 64, 64)))
+    return BTX_ERR_CUDA;
   p.M = pl.F; p.N = pl.d; p.m_tiles = (pl.F + kRowTile - 1) / kRowTile; p.n_tiles = (pl.d + BN - 1) / BN; p.of = dw2;
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, 2, st)) != BTX_OK) return s;
   mark_stage(4, st);
-  if (!make_map(&a0, b.xs, d, RP, 0, 64, 64) || !make_map(&b0, b.dh1, F, RP, 0, 64, 64) ||
-      !make_map(&b1, b.dh3, F, RP, 0, 64, 64))
+  p.a_one = make_map_mn(&a0, b.xs, d, RP, 0);
+  p.b_one = make_map_mn(&b0, b.dh1, F, RP, 0) && make_map_mn(&b1, b.dh3, F, RP, 0);
+  if ((!p.a_one && !make_map(&a0, b.xs, d, RP, 0, 64, 64)) ||
+      (!p.b_one && (!make_map(&b0, b.dh1, F, RP, 0, 64, 64) || !make_map(&b1, b.dh3, F, RP, 0, 64, 64))))
     return BTX_ERR_CUDA;
   p.M = pl.d; p.N = pl.F; p.m_tiles = (pl.d + kRowTile - 1) / kRowTile; p.n_tiles = (pl.F + BN - 1) / BN; p.of = dw1;
   if ((s = launch_tc<G_WGRAD>(a0, a0, b0, b0, p, pl.E * p.m_tiles * p.n_tiles, 3, st)) != BTX_OK) return s;

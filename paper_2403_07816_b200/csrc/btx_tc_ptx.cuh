@@ -113,6 +113,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // arrive (once the MMAs issued so far have retired) on the barrier at this offset in both CTAs
@@ -228,6 +236,25 @@ inline bool make_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t r
   const cuuint32_t rank = experts > 0 ? 3 : 2;
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The same tensor seen as [E,] cols/64 chunks x rows x 64 columns, for operands the tensor core reads MN-major:
+// one box of (64 columns, 64 rows, 2 chunks) lands in shared memory as two consecutive 64x64 MN-major tiles,
+// i.e. a 128-wide operand tile per TMA operation instead of one operation per 64 columns.  Needs cols to be a
+// multiple of 64 (the chunk dimension must tile the row exactly); returns false otherwise, or when the driver
+// refuses the strides, and the caller then loads the two tiles separately.
+// Coordinates: (0, row, chunk[, expert]).
+inline bool make_map_mn(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t experts) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || cols % 64 != 0) return false;
+  cuuint64_t dims[4] = {64, rows, cols / 64, experts};
+  cuuint64_t strides[3] = {cols * 2, 128, cols * rows * 2};
+  cuuint32_t box[4] = {64, 64, 2, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  const cuuint32_t rank = experts > 0 ? 4 : 3;
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
