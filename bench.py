@@ -45,11 +45,11 @@ ALPHA = 0.01
 SOAK_S = 2.0             # untimed run of the same step before the warm-up: power state and clocks settle
 E2E_STEPS = 50
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core GEMM launches of one training
-# step, from the ncu capture summarised under profiles/ (taken at T=4096 and scaled by 4 to T=16384: every
-# operand and output of these launches grows in proportion to T).  The figure belongs to the kernel sources
-# whose hash is recorded with it; with any other sources the bench reports traffic = null.
-TC_GEMM_TRAFFIC = {"bytes_per_step_T16384": 33.81e9, "sources_sha256_16": "unset"}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the seven tensor-core GEMM launches of one training
+# step at T=16384, from the one-pass ncu capture summarised in profiles/tc_gemm_kernel_fwd_bwd_T16384_dram.txt
+# (the traffic does not grow in proportion to T, so the T=4096 capture is not scaled).  The figure belongs to the
+# kernel sources whose hash is recorded with it; with any other sources the bench reports traffic = null.
+TC_GEMM_TRAFFIC = {"bytes_per_step_T16384": 33.93e9, "sources_sha256_16": "cfc18d776dac8077"}
 TC_GEMM_SOURCES = ("btx_gemm_tc.cu", "btx_tc_ptx.cuh", "btx_common.cuh")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
