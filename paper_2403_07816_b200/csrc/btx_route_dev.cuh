@@ -41,8 +41,11 @@ template <> struct Vec<__nv_bfloat16> {
   }
 };
 
-// Selection, gates and softmax for one token from the logits z[0..E) in shared memory (all lanes of
-// the calling warp take part).  The experts are chosen on z as it stands; the softmaxes are those of
+// Selection, gates and softmax for one token from the logits z[0..E) in shared memory, by the 32 lanes of
+// the calling warp together: lane l owns experts l and l + 32.  Top-k is k rounds of a warp arg-max over
+// (value descending, index ascending), so ties go to the lower index; the sums of the two softmaxes run over
+// the experts (resp. the slots) in ascending order, one addition at a time, so the result does not depend on
+// how the lanes are laid out.  The experts are chosen on z as it stands; the softmaxes are those of
 // z * scale (scale = 1 except for Sample Top-1, whose temperature must not touch the arg-max: a
 // rounded product could merge two distinct perturbed logits into a tie).  On return lane l holds the
 // dense gate and probability of experts l (index 0) and l + 32 (index 1).
@@ -50,47 +53,67 @@ __device__ __forceinline__ void route_select(int t, int E, int k, int routing, f
                                              int32_t* __restrict__ topk,
                                              float* __restrict__ gates, float* __restrict__ probs, float (&my_g)[2],
                                              float (&my_p)[2]) {
-  unsigned long long taken = 0;
-  int sel[kMaxExperts];
+  constexpr unsigned kAll = 0xffffffffu;
+  const bool have[2] = {lane < E, lane + 32 < E};
+  const float zv[2] = {have[0] ? z[lane] : 0.f, have[1] ? z[lane + 32] : 0.f};
+  int slot[2] = {-1, -1};          // the slot in which this lane's expert was selected
+  int sel[2] = {0, 0};             // lane j keeps the expert of slots j and j + 32
   int first = 0;
-  // repeated arg-max: strict '>' keeps the lower index on ties
+  float zmax = 0.f;
   for (int j = 0; j < k; ++j) {
-    int best = -1;
-    float zb = 0.f;
-    for (int e = 0; e < E; ++e) {
-      if ((taken >> e) & 1ull) continue;
-      float ze = z[e];
-      if (best < 0 || ze > zb) { best = e; zb = ze; }
+    // this lane's candidate: its lower expert wins a tie ('>' is strict)
+    int bi = -1;
+    float bv = 0.f;
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      if (have[h] && slot[h] < 0 && (bi < 0 || zv[h] > bv)) { bi = lane + 32 * h; bv = zv[h]; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(kAll, bv, o);
+      const int oi = __shfl_xor_sync(kAll, bi, o);
+      if (oi >= 0 && (bi < 0 || ov > bv || (ov == bv && oi < bi))) { bi = oi; bv = ov; }
     }
-    taken |= 1ull << best;
-    sel[j] = best;
-    if (j == 0) first = best;
+    if (j == 0) { first = bi; zmax = bv; }
+    if ((bi & 31) == lane) slot[bi >> 5] = j;
+    if ((j & 31) == lane) sel[j >> 5] = bi;
   }
-  const float zmax = z[first];
+  float ex[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) ex[h] = have[h] ? expf((zv[h] - zmax) * scale) : 0.f;
   float psum = 0.f;
-  for (int e = 0; e < E; ++e) psum += expf((z[e] - zmax) * scale);
+  for (int e = 0; e < min(E, 32); ++e) psum += __shfl_sync(kAll, ex[0], e);
+  for (int e = 32; e < E; ++e) psum += __shfl_sync(kAll, ex[1], e - 32);
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    const int e = lane + 32 * h;
-    my_p[h] = (e < E) ? expf((z[e] - zmax) * scale) / psum : 0.f;
+    my_p[h] = have[h] ? ex[h] / psum : 0.f;
     my_g[h] = 0.f;
   }
   if (routing == BTX_ROUTE_SWITCH) {
-    float g0 = expf((z[first] - zmax) * scale) / psum;
-    if ((first & 31) == lane) my_g[first >> 5] = g0;
-    if (lane == 0) { topk[t] = first; gates[t] = g0; }
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      if (slot[h] == 0) {          // the lane that owns the arg-max: the gate is its full-softmax probability
+        my_g[h] = ex[h] / psum;
+        topk[t] = first;
+        gates[t] = my_g[h];
+      }
   } else {
     float gsum = 0.f;
-    for (int j = 0; j < k; ++j) gsum += expf((z[sel[j]] - zmax) * scale);
     for (int j = 0; j < k; ++j) {
-      float gj = expf((z[sel[j]] - zmax) * scale) / gsum;
-      if ((sel[j] & 31) == lane) my_g[sel[j] >> 5] = gj;
-      if (lane == 0) { topk[(size_t)t * k + j] = sel[j]; gates[(size_t)t * k + j] = gj; }
+      const int s = __shfl_sync(kAll, sel[j >> 5], j & 31);
+      const float e0 = __shfl_sync(kAll, ex[0], s & 31), e1 = __shfl_sync(kAll, ex[1], s & 31);
+      gsum += s < 32 ? e0 : e1;
     }
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      if (slot[h] >= 0) {          // the lane that owns a selected expert writes that slot
+        my_g[h] = ex[h] / gsum;
+        topk[(size_t)t * k + slot[h]] = lane + 32 * h;
+        gates[(size_t)t * k + slot[h]] = my_g[h];
+      }
   }
 #pragma unroll
   for (int h = 0; h < 2; ++h)
-    if (lane + 32 * h < E) probs[(size_t)t * E + lane + 32 * h] = my_p[h];
+    if (have[h]) probs[(size_t)t * E + lane + 32 * h] = my_p[h];
   __syncwarp();
 }
 

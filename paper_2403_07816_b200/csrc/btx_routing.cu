@@ -128,7 +128,14 @@ __device__ __forceinline__ void lb_finalize(int Tn, int E, int nblocks, float al
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int pair = warp; pair < 2 * E; pair += kRouterWarps) {
     double s = 0.0;
-    for (int b = lane; b < nblocks; b += 32) s += (double)__ldcg(route_part + (size_t)b * 2 * E + pair);
+    for (int b0 = lane; b0 < nblocks; b0 += 8 * 32) {     // eight loads ahead, added in the same order as one by one
+      float v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = b0 + i * 32 < nblocks ? __ldcg(route_part + (size_t)(b0 + i * 32) * 2 * E + pair) : 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (b0 + i * 32 < nblocks) s += (double)v[i];
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     s /= (double)Tn;
