@@ -205,6 +205,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   cluster_sync_all();                                     // the peer's barriers exist before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Launched as a programmatic dependent: everything above ran while the kernel before this one may still have
+  // been running; nothing below (which reads what that kernel wrote) starts before it has completed.
+  allow_dependents();
+  grid_dependency_wait();
   const int n_total = total_tiles<MODE>(p);
 
   if (warp == 0) {
@@ -484,8 +488,9 @@ btx_status launch_tc(const CUtensorMap& a0, const CUtensorMap& a1, const CUtenso
   int pairs = sm_count() / 2;
   if (pairs > max_tiles) pairs = max_tiles;
   if (pairs < 1) pairs = 1;
-  tc_gemm_kernel<MODE><<<2 * pairs, TC_THREADS, SMEM_BYTES, st>>>(a0, a1, b0, b1, p);   // cluster dims are compiled in
-  return cudaGetLastError() == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
+  // cluster dims are compiled in
+  return launch_after_predecessor(tc_gemm_kernel<MODE>, dim3(2 * pairs), dim3(TC_THREADS), SMEM_BYTES, st, true, a0, a1, b0,
+                                  b1, p) == cudaSuccess ? BTX_OK : BTX_ERR_CUDA;
 }
 
 // One thread waits, with a 50 ms limit, on a barrier that nobody will ever arrive at.

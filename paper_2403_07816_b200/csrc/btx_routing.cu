@@ -690,7 +690,7 @@ cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int spl
   int blocks = (int)min((n + 255) / 256, (size_t)sm_count() * 32);
   const int32_t* kept = pl.capped ? b.flat2row : nullptr;
   if (dtype == BTX_BF16)
-    return launch_after_predecessor(combine_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, pl.small != 0, pl.T,
+    return launch_after_predecessor(combine_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, true, pl.T,
                                     pl.d, pl.k, pl.E, splits, rows, (const float*)nullptr,
                                     (const __nv_bfloat16*)nullptr, kept, (__nv_bfloat16*)y);
   combine_kernel<float><<<blocks, 256, 0, st>>>(pl.T, pl.d, pl.k, pl.E, splits, rows, nullptr, nullptr, kept, (float*)y);
