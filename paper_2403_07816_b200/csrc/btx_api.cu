@@ -246,13 +246,17 @@ extern "C" btx_status btx_moe_forward(const btx_moe_desc* desc, const void* x, c
   resolve(pl, sv, ws, &b);
 
   mark_stage(0, st);
+  // A handful of tokens, nothing kept: the whole layer is one cooperative kernel (it clears the status word
+  // itself).  Where that launch is refused (a device partition with too few multiprocessors for all its
+  // blocks to be resident at once, say) the launches below do the same work.
+  bool done = false;
   if (pl.dense) {
-    // a handful of tokens, nothing kept: the whole layer is one kernel (it clears the status word itself)
-    if ((s = launch_forward_small_fused_bf16(pl, er.routing, desc->lb_alpha, x, w_router, router_bias, noise, er.inv_tau,
-                                             w1, w3, w2, y, b, st)) != BTX_OK)
-      return s;
-    mark_stage(4, st);
-  } else {
+    done = launch_forward_small_fused_bf16(pl, er.routing, desc->lb_alpha, x, w_router, router_bias, noise, er.inv_tau, w1,
+                                           w3, w2, y, b, st) == BTX_OK;
+    if (done) mark_stage(4, st);
+    else cudaGetLastError();
+  }
+  if (!done) {
     const float* expert_rows = b.yp;
     int splits = 1;
     BTX_CUDA_OK(cudaMemsetAsync(b.status, 0, kStatusWords * 4, st));

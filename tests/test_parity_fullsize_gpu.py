@@ -158,6 +158,32 @@ def test_decode_shaped_T32_two_layers_seed4():
         assert rel_err(np64(fwd["y"]), ref["y"]) <= TOL
 
 
+@pytest.mark.parametrize("T,F_,E_,k,routing,cf", [
+    (48, 5504, 8, 2, B.ROUTE_TOPK, 0.0),       # split experts, top-2 of 8: MMA N = 48, eight experts streamed
+    (64, 11008, 4, 1, B.ROUTE_SWITCH, 1.0),    # the widest token tile (N = 64), Switch gate, capacity limit with drops
+    (9, 11008, 4, 4, B.ROUTE_SOFT, 0.0),       # every expert for every token, N = 16 with 9 real tokens
+])
+def test_decode_shaped_variants_full_width(T, F_, E_, k, routing, cf):
+    """The one-kernel inference forward at d = 4096 and the full hidden widths, in the launch configuration the
+    decode bench uses (74 CTA pairs, several tiles per pair): the whole output against the oracle."""
+    inp = synth.moe_inputs(T, D, F_, E_, 7, torch.bfloat16, DEV, with_dy=False)
+    bias = synth.skew_bias(E_, DEV) if cf > 0 else None
+    fwd = gpu_forward(inp, k, routing, ALPHA, bias, save=False, capacity_factor=cf)
+    cpu = {n: np64(t) for n, t in inp.items()}
+    z_gpu = fwd["routing"].logits.cpu().numpy()
+    kk = E_ if routing == B.ROUTE_SOFT else k
+    ref = o.moe_forward(cpu["x"], cpu["w_router"], cpu["w1"], cpu["w3"], cpu["w2"], kk, routing, ALPHA,
+                        router_bias=None if bias is None else np64(bias), logits=z_gpu, capacity_factor=cf)
+    r = fwd["routing"]
+    for name in ("topk_idx", "counts", "offsets", "perm", "inv_perm"):
+        assert np.array_equal(getattr(r, name).cpu().numpy(), ref[name]), name
+    if cf > 0:
+        assert not ref["keep"].all()
+    assert rel_err(r.gates.cpu().numpy(), ref["gates"]) <= TOL
+    assert abs(float(r.lb_loss.item()) - ref["lb_loss"]) <= TOL * max(abs(ref["lb_loss"]), 1e-30)
+    assert rel_err(np64(fwd["y"]), ref["y"]) <= TOL
+
+
 def test_merge_llama2_7b_shaped_tensors_seed4():
     """MiX merge at the sizes of the Llama-2-7B shape (Section 3.2): two layers plus embeddings, head and final
     norm of four BF16 parameter sets (5.4 GB read).  Averaged tensors against the fp64 mean rounded once;
