@@ -238,7 +238,7 @@ def free_device_memory():
 
 
 # kernels launched per call (memsets and copies are not counted)
-LAUNCHES_FWD = 9          # router, loss finalise, 3 permutation kernels, gather, GEMM-1, GEMM-2, combine
+LAUNCHES_FWD = 8          # router (its last block finalises the loss), 3 permutation kernels, gather, GEMM-1, GEMM-2, combine
 LAUNCHES_FWD_SMALL = 6    # one-launch routing, gather, pass 1, SwiGLU fix-up, pass 2, combine
 LAUNCHES_FWD_DENSE = 1    # inference with at most 64 tokens: the whole layer is one cooperative kernel
 LAUNCHES_BWD = 11         # dy gather, dgrad-2, dgrad-1, 3 weight gradients, row-sum, dz, dW_l partial, dx combine, reduce
