@@ -153,19 +153,24 @@ def run_reference(args):
     workload = args.workload if args.workload in ("fwd_bwd", "fwd") else "fwd_bwd"
     T, k = WORKLOADS[workload][0], WORKLOADS[workload][1]
     # A step of the oracle costs a fixed part (every expert's fp64 weights pass through the cores once, whatever
-    # the batch) plus a part per token.  Two calibration passes give both; the sample is then sized so that
-    # steps + warm-up take about two and a half minutes.
-    fn, _ = oracle_step_fn(workload, 16)
-    t0 = time.perf_counter(); fn(); c16 = time.perf_counter() - t0
-    fn, _ = oracle_step_fn(workload, 272)
-    t0 = time.perf_counter(); fn(); c272 = time.perf_counter() - t0
-    per_token = max((c272 - c16) / 256.0, 1e-5)
-    fixed = max(c16 - 16 * per_token, 0.0)
-    total = max(1, args.steps + args.warmup)
-    budget = 150.0 / total
+    # the batch) plus a part per token that grows a little faster than linearly.  Two calibration passes give
+    # both; the sample is sized, with a safety factor and a cap of 4096 tokens, so that steps + warm-up take
+    # about two and a half minutes, and one trial step at that size shrinks it further if it still runs long.
+    def timed(n_tok):
+        f, _ = oracle_step_fn(workload, n_tok)
+        t0 = time.perf_counter(); f(); return time.perf_counter() - t0
+    c_lo, c_hi = timed(64), timed(512)
+    per_token = 1.5 * max((c_hi - c_lo) / 448.0, 1e-5)
+    fixed = max(c_lo - 64 * per_token / 1.5, 0.0)
+    total = args.steps + args.warmup + 1                 # + the trial step
+    budget = 140.0 / total
     tokens = int((budget - fixed) / per_token) if budget > fixed else 16
-    tokens = max(16, min(T, tokens // 16 * 16))
+    tokens = max(16, min(T, 4096, tokens // 16 * 16))
     fn, n = oracle_step_fn(workload, tokens)
+    t0 = time.perf_counter(); fn(); trial = time.perf_counter() - t0
+    if trial > 1.3 * budget and tokens > 16:
+        tokens = max(16, int(tokens * budget / trial * 0.9) // 16 * 16)
+        fn, n = oracle_step_fn(workload, tokens)
     for _ in range(args.warmup):
         fn()
     t0 = time.perf_counter()
