@@ -329,6 +329,9 @@ def test_capacity_factor_small_batch_and_limits(dtype):
     (1, 128, 128, 1, 1, B.ROUTE_TOPK, 0.0),       # a single token, a single expert
     (40, 128, 264, 4, 2, B.ROUTE_TOPK, 0.5),      # capacity limit: dropped assignments are skipped in pass 2
     (48, 64, 72, 3, 1, B.ROUTE_SAMPLE1, 0.0),
+    (64, 64, 72, 64, 8, B.ROUTE_TOPK, 0.0),       # the expert limit: two experts per lane in the selection, 64 small experts
+    (40, 72, 40, 33, 33, B.ROUTE_SOFT, 0.0),      # one expert beyond a warp's lanes, every expert for every token
+    (64, 128, 136, 5, 2, B.ROUTE_TOPK, 0.4),      # tight capacity at N = 64: most assignments dropped
 ])
 def test_inference_forward_of_a_few_tokens(T, d, F, E, k, routing, cf):
     """BF16 forward that keeps nothing for backward, at most 64 tokens: every expert's weights meet all tokens
