@@ -404,3 +404,37 @@ def test_training_step_replays_from_a_cuda_graph():
     assert B.btx_device_status(ws) == B.BTX_OK
     for n, t in outs.items():
         assert torch.equal(t, direct[n]), n
+
+
+def test_inference_forward_replays_from_a_cuda_graph():
+    """The one-kernel forward of a few tokens is a single cooperative launch; three layers of it can be captured
+    once and replayed, with the direct calls' bits."""
+    T, d, F, E, k = 32, 1024, 2048, 4, 2
+    sets = [synth.moe_inputs(T, d, F, E, 4, torch.bfloat16, DEV, layer=l, with_dy=False) for l in range(3)]
+    desc = B.make_desc(T, d, F, E, k, torch.bfloat16, B.ROUTE_TOPK, 0.01, False, False)
+    ws, _ = B.alloc_buffers(desc, DEV)
+    ys = [torch.empty(T, d, dtype=torch.bfloat16, device=DEV) for _ in sets]
+
+    def step():
+        for inp, y in zip(sets, ys):
+            B.btx_moe_forward(desc, inp["x"], inp["w_router"], None, inp["w1"], inp["w3"], inp["w2"], y, None, None, ws)
+
+    step()
+    torch.cuda.synchronize()
+    direct = [y.clone() for y in ys]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for y in ys:
+        y.zero_()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert B.btx_device_status(ws) == B.BTX_OK
+    for got, want in zip(ys, direct):
+        assert torch.equal(got, want)
