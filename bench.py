@@ -49,7 +49,7 @@ E2E_STEPS = 50
 # step at T=16384, from the one-pass ncu capture summarised in profiles/tc_gemm_kernel_fwd_bwd_T16384_dram.txt
 # (the traffic does not grow in proportion to T, so the T=4096 capture is not scaled).  The figure belongs to the
 # kernel sources whose hash is recorded with it; with any other sources the bench reports traffic = null.
-TC_GEMM_TRAFFIC = {"bytes_per_step_T16384": 33.93e9, "sources_sha256_16": "cfc18d776dac8077"}
+TC_GEMM_TRAFFIC = {"bytes_per_step_T16384": 33.68e9, "sources_sha256_16": "4b5584b3b2e0e287"}
 TC_GEMM_SOURCES = ("btx_gemm_tc.cu", "btx_tc_ptx.cuh", "btx_common.cuh")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
