@@ -84,13 +84,14 @@ __device__ __forceinline__ void prefetch_map(const CUtensorMap* m) {
 
 // Work split.  The weight rows of a pass, all experts one after the other, are counted in units of 16 rows
 // and cut into chunks of `cap` units (one full tile of a CTA pair); chunk i goes to pair i mod n_pairs, so at
-// any time the pairs read neighbouring chunks (measured: with one contiguous range of rows per pair, i.e.
-// pairs reading megabytes apart, the same bytes stream 30-40 % slower, and a tile with fewer rows takes as long
-// per K block as a full one, so evening out the rows buys nothing).  A chunk that crosses the end of an
-// expert is walked as two tiles.  The first half of a tile's capacity belongs to the pair's first CTA; a CTA
-// fetches its units of a tile as boxes of 8, 4, 2 and 1 units, a full share as one box on a path of its own
-// (measured: every TMA operation the producer thread steps through, even one it skips under a predicate,
-// costs it about 80 ns, and three skipped ones per K block took the stream from 5.7 to 4.3 TB/s).
+// any time the pairs read neighbouring chunks.  At the Llama-2-7B shape the last round of pass 1 then has a
+// tile for 48 of the 74 pairs only; cutting what is left after the full rounds evenly among all pairs instead
+// was measured 3-7 % slower (a tile with fewer rows takes about as long per K block as a full one), so the
+// plain deal stayed.  A chunk that crosses the end of an expert is walked as two tiles.  The first half of a
+// tile's capacity belongs to the pair's first CTA; a CTA fetches its units of a tile as boxes of 8, 4, 2 and 1
+// units, a full share as one box on a path of its own (measured: every TMA operation the producer thread
+// steps through, even one it skips under a predicate, costs it about 80 ns, and three skipped ones per K
+// block took the stream from 5.7 to 4.3 TB/s).
 constexpr int XU = 16;                                   // rows per unit
 struct XTile { int e, u0, n; };                          // expert, first unit inside the expert, units of both CTAs
 struct XWalk {                                           // a pair's walk over its chunks
