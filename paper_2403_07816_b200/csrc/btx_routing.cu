@@ -18,8 +18,6 @@ namespace {
 
 using namespace routedev;
 
-constexpr int kRouteDepth = 2;        // 16-byte vectors of x per lane and token in flight in the router kernel
-constexpr int kRouteBlocksPerSm = 4;
 constexpr int kRouterThreads = 256;
 constexpr int kRouterWarps = kRouterThreads / 32;
 constexpr int kPermThreads = 256;
@@ -28,75 +26,71 @@ constexpr int kPermChunk = 1024;      // assignments per block of the permutatio
 // ---------------------------------------------------------------------------------------------
 // Router
 // ---------------------------------------------------------------------------------------------
-// Logits of two tokens by one warp (the second may be absent: t1 >= Tn): every lane takes each 32nd
-// 16-byte vector of both rows, so a router row vector fetched from L1 serves two tokens and twice as many
-// loads of x are in flight per warp.  z0/z1: the warp's shared scratch of kMaxExperts floats each.
-template <typename T>
-__device__ __forceinline__ void route_logits2(int t0, bool two, int d, int E, const T* __restrict__ x,
-                                              const T* __restrict__ wr, const float* __restrict__ bias,
-                                              const float* __restrict__ given_logits, float* z0, float* z1, int lane) {
-  constexpr int VN = Vec<T>::N;
+// Logits of up to four tokens t0 .. t0+nt-1 by one warp: every lane takes each 32nd 16-byte vector of the rows,
+// so one fetch of a router row vector serves four tokens.  With WS the router rows come from shared memory as
+// fp32, laid out [expert][quad of the vector][vector][4] so that the lanes of a warp read consecutive 16-byte
+// words; otherwise from global memory through L1.  z: the warp's shared scratch, kMaxExperts floats per token.
+constexpr int kRouteTokens = 4;
+template <typename T, bool WS>
+__device__ __forceinline__ void route_logits4(int t0, int nt, int d, int E, const T* __restrict__ x,
+                                              const T* __restrict__ wr, const float* ws, const float* __restrict__ bias,
+                                              const float* __restrict__ given_logits, float (*z)[kMaxExperts], int lane) {
+  constexpr int VN = Vec<T>::N, NT = kRouteTokens;
   if (given_logits != nullptr) {
     for (int e = lane; e < E; e += 32) {
       const float b = bias ? bias[e] : 0.f;
-      z0[e] = given_logits[(size_t)t0 * E + e] + b;
-      if (two) z1[e] = given_logits[(size_t)(t0 + 1) * E + e] + b;
+      for (int i = 0; i < nt; ++i) z[i][e] = given_logits[(size_t)(t0 + i) * E + e] + b;
     }
     return;
   }
-  const T* x0 = x + (size_t)t0 * d;
-  const T* x1 = two ? x0 + d : x0;
+  const T* xr[NT];
+#pragma unroll
+  for (int i = 0; i < NT; ++i) xr[i] = x + (size_t)(t0 + min(i, nt - 1)) * d;   // absent tokens repeat the last one
+  const int vecs = d / VN;
   for (int eb = 0; eb < E; eb += 8) {
-    float a0[8], a1[8];
+    float acc[NT][8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) { a0[j] = 0.f; a1[j] = 0.f; }
-    // A chunk is kRouteDepth 16-byte vectors per lane and token, all loaded before the first one is used.
-    // Measured at the Llama-2-7B shape: the kernel issues about 4600 instructions per token pair at 0.9 per
-    // cycle and multiprocessor, i.e. it is bound by instruction latency with the warps it has, not by the x
-    // stream: batches of 4 and 8 vectors (with the registers, hence fewer warps, they cost) were 7 and 19 %
-    // slower than 2.
-    for (int c0 = lane * VN; c0 < d; c0 += kRouteDepth * 32 * VN) {
-      uint4 q0[kRouteDepth], q1[kRouteDepth];
+    for (int i = 0; i < NT; ++i)
 #pragma unroll
-      for (int i = 0; i < kRouteDepth; ++i) {
-        const int c = c0 + i * 32 * VN;
-        if (c < d) {
-          q0[i] = __ldcs(reinterpret_cast<const uint4*>(x0 + c));   // streamed once: leave L1 to the router rows
-          q1[i] = __ldcs(reinterpret_cast<const uint4*>(x1 + c));
-        }
-      }
+      for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+#pragma unroll 2
+    for (int v = lane; v < vecs; v += 32) {
+      uint4 q[NT];
 #pragma unroll
-      for (int i = 0; i < kRouteDepth; ++i) {
-        const int c = c0 + i * 32 * VN;
-        if (c < d) {
-          float u0[VN], u1[VN];
-          Vec<T>::unpack(q0[i], u0);
-          Vec<T>::unpack(q1[i], u1);
+      for (int i = 0; i < NT; ++i) q[i] = __ldcs(reinterpret_cast<const uint4*>(xr[i]) + v);   // streamed once
+      float u[NT][VN];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            if (eb + j < E) {
-              float wv[VN];
-              Vec<T>::load(wr + (size_t)(eb + j) * d + c, wv);
+      for (int i = 0; i < NT; ++i) Vec<T>::unpack(q[i], u[i]);
 #pragma unroll
-              for (int v = 0; v < VN; ++v) { a0[j] = fmaf(u0[v], wv[v], a0[j]); a1[j] = fmaf(u1[v], wv[v], a1[j]); }
+      for (int j = 0; j < 8; ++j) {
+        if (eb + j < E) {
+          float wv[VN];
+          if (WS) {
+#pragma unroll
+            for (int h = 0; h < VN / 4; ++h) {
+              const float4 w4 = *reinterpret_cast<const float4*>(ws + (((size_t)(eb + j) * (VN / 4) + h) * vecs + v) * 4);
+              wv[4 * h] = w4.x; wv[4 * h + 1] = w4.y; wv[4 * h + 2] = w4.z; wv[4 * h + 3] = w4.w;
             }
+          } else {
+            Vec<T>::load(wr + (size_t)(eb + j) * d + (size_t)v * VN, wv);
           }
+#pragma unroll
+          for (int i = 0; i < NT; ++i)
+#pragma unroll
+            for (int c = 0; c < VN; ++c) acc[i][j] = fmaf(u[i][c], wv[c], acc[i][j]);
         }
       }
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       if (eb + j < E) {
-        float s0 = a0[j], s1 = a1[j];
+        const float b = bias ? bias[eb + j] : 0.f;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          s0 += __shfl_xor_sync(0xffffffffu, s0, o);
-          s1 += __shfl_xor_sync(0xffffffffu, s1, o);
-        }
-        if (lane == 0) {
-          const float b = bias ? bias[eb + j] : 0.f;
-          z0[eb + j] = s0 + b;
-          z1[eb + j] = s1 + b;
+        for (int i = 0; i < NT; ++i) {
+          float sum = acc[i][j];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+          if (lane == 0) z[i][eb + j] = sum + b;
         }
       }
     }
@@ -152,33 +146,42 @@ __device__ __forceinline__ void lb_finalize(int Tn, int E, int nblocks, float al
   }
 }
 
-// One warp per pair of tokens.  Every block leaves its partial sums of the gates and probabilities; the block
-// that finishes last (a ticket in the workspace status block, zero when the kernel starts) forms the batch
-// means and the loss from all of them.
-template <typename T>
-__global__ void __launch_bounds__(kRouterThreads, kRouteBlocksPerSm)   // at most 64 registers: the kernel needs the warps
+// One warp per four tokens; the blocks are persistent (two per multiprocessor) and, when the router matrix fits
+// (E*d fp32 values in at most 64 KB), keep it in shared memory as fp32, so the inner loop neither fetches nor
+// converts router rows per token.  Every block leaves its partial sums of the gates and probabilities; the
+// block that finishes last (a ticket in the workspace status block, zero when the kernel starts) forms the
+// batch means and the loss from all of them.
+template <typename T, bool WS>
+__global__ void __launch_bounds__(kRouterThreads, 2)
 router_kernel(int Tn, int d, int E, int k, int routing, float alpha, const T* __restrict__ x, const T* __restrict__ wr,
               const float* __restrict__ bias, const float* __restrict__ given_logits,
               const float* __restrict__ noise, float inv_tau,
               float* __restrict__ logits, int32_t* __restrict__ topk, float* __restrict__ gates,
               float* __restrict__ probs, float* route_part, float* __restrict__ u, float* __restrict__ p,
               float* __restrict__ loss, double* __restrict__ up64, int32_t* ticket) {
-  __shared__ float zs[kRouterWarps][2][kMaxExperts];
+  extern __shared__ __align__(16) float ws[];             // WS: the router rows as fp32
+  __shared__ float zs[kRouterWarps][kRouteTokens][kMaxExperts];
   __shared__ float red[kRouterWarps][kMaxExperts][2];
   __shared__ int is_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   allow_dependents();
+  if (WS) {
+    constexpr int VN = Vec<T>::N;
+    const int vecs = d / VN;
+    for (int idx = threadIdx.x; idx < E * d; idx += kRouterThreads) {
+      const int e = idx / d, c = idx - e * d, v = c / VN, r = c - v * VN;
+      ws[(((size_t)e * (VN / 4) + r / 4) * vecs + v) * 4 + (r & 3)] = to_f32(wr[idx]);
+    }
+    __syncthreads();
+  }
   float u_acc[2] = {0.f, 0.f}, p_acc[2] = {0.f, 0.f};   // lane l accumulates experts l and l + 32 over this warp's tokens
-  for (int t = (blockIdx.x * kRouterWarps + warp) * 2; t < Tn; t += gridDim.x * kRouterWarps * 2) {
-    const bool two = t + 1 < Tn;
-    route_logits2<T>(t, two, d, E, x, wr, bias, given_logits, zs[warp][0], zs[warp][1], lane);
+  for (int t = (blockIdx.x * kRouterWarps + warp) * kRouteTokens; t < Tn; t += gridDim.x * kRouterWarps * kRouteTokens) {
+    const int nt = min(kRouteTokens, Tn - t);
+    route_logits4<T, WS>(t, nt, d, E, x, wr, ws, bias, given_logits, zs[warp], lane);
     __syncwarp();
-    float my_g[2], my_p[2];
-    route_finish_token(t, E, k, routing, noise, inv_tau, zs[warp][0], lane, logits, topk, gates, probs, my_g, my_p);
-#pragma unroll
-    for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
-    if (two) {
-      route_finish_token(t + 1, E, k, routing, noise, inv_tau, zs[warp][1], lane, logits, topk, gates, probs, my_g, my_p);
+    for (int i = 0; i < nt; ++i) {
+      float my_g[2], my_p[2];
+      route_finish_token(t + i, E, k, routing, noise, inv_tau, zs[warp][i], lane, logits, topk, gates, probs, my_g, my_p);
 #pragma unroll
       for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
     }
@@ -623,21 +626,31 @@ router_dw_reduce_kernel(int d, int E, int chunks, const float* __restrict__ part
 // ---------------------------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------------------------
+template <typename T, bool WS>
+static cudaError_t launch_router_t(const Plan& pl, int routing, float alpha, const void* x, const void* w_router,
+                                   const float* bias, const float* given_logits, const float* noise, float inv_tau,
+                                   const Buffers& b, size_t smem, cudaStream_t st) {
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(router_kernel<T, WS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  // the ticket of the last-block finalisation is word 8 of the status block, zeroed by the caller
+  router_kernel<T, WS><<<pl.route_blocks, kRouterThreads, smem, st>>>(
+      pl.T, pl.d, pl.E, pl.k, routing, alpha, (const T*)x, (const T*)w_router, bias, given_logits, noise, inv_tau,
+      b.logits, b.topk, b.gates, b.probs, b.route_part, b.u, b.p, b.loss, b.up64, b.status + 8);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, const void* x, const void* w_router,
                           const float* bias, const float* given_logits, const float* noise, float inv_tau,
                           const Buffers& b, cudaStream_t st) {
-  // the ticket of the last-block finalisation is word 8 of the status block, zeroed by the caller
-  if (dtype == BTX_BF16) {
-    router_kernel<__nv_bfloat16><<<pl.route_blocks, kRouterThreads, 0, st>>>(
-        pl.T, pl.d, pl.E, pl.k, routing, alpha, (const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, bias,
-        given_logits, noise, inv_tau, b.logits, b.topk, b.gates, b.probs, b.route_part, b.u, b.p, b.loss, b.up64,
-        b.status + 8);
-  } else {
-    router_kernel<float><<<pl.route_blocks, kRouterThreads, 0, st>>>(
-        pl.T, pl.d, pl.E, pl.k, routing, alpha, (const float*)x, (const float*)w_router, bias, given_logits, noise,
-        inv_tau, b.logits, b.topk, b.gates, b.probs, b.route_part, b.u, b.p, b.loss, b.up64, b.status + 8);
-  }
-  return cudaGetLastError();
+  const size_t smem = (size_t)pl.E * pl.d * sizeof(float);
+  const bool in_smem = given_logits == nullptr && smem > 0 && smem <= 64 * 1024;
+  if (dtype == BTX_BF16)
+    return in_smem ? launch_router_t<__nv_bfloat16, true>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, smem, st)
+                   : launch_router_t<__nv_bfloat16, false>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, 0, st);
+  return in_smem ? launch_router_t<float, true>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, smem, st)
+                 : launch_router_t<float, false>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, 0, st);
 }
 
 bool route_permute_small_fits(const Plan& pl) { return pl.R <= kSmallMaxR; }
