@@ -117,6 +117,79 @@ __device__ __forceinline__ void route_select(int t, int E, int k, int routing, f
   __syncwarp();
 }
 
+// The same selection for up to 32 / G tokens at once when the layer has at most G <= 16 experts: G lanes per
+// token, lane (slot, e) = (lane / G, lane % G) owns expert e of token i0 + slot.  z: the warp's logits in shared
+// memory, kMaxExperts floats per token; tokens i0 .. min(i0 + 32 / G, nt) - 1 of the group starting at global
+// token t0 are routed, their (unperturbed) logits stored, the Sample Top-1 noise added before the selection.
+// Arithmetic and results per token are those of route_select.  On return lane e < E (slot 0) has had the gates
+// and probabilities of expert e over the routed tokens added to u_sum and p_sum.
+template <int G>
+__device__ __forceinline__ void route_select_group(int t0, int i0, int nt, int E, int k, int routing, float scale,
+                                                   const float* __restrict__ noise, float (*z)[kMaxExperts], int lane,
+                                                   float* __restrict__ logits, int32_t* __restrict__ topk,
+                                                   float* __restrict__ gates, float* __restrict__ probs, float& u_sum,
+                                                   float& p_sum) {
+  constexpr unsigned kAll = 0xffffffffu;
+  const int slot = lane / G, e = lane % G, i = i0 + slot;
+  const bool have = i < nt && e < E;
+  const size_t t = (size_t)t0 + i;
+  float zv = 0.f;
+  if (have) {
+    zv = z[i][e];
+    logits[t * E + e] = zv;                               // reported logits are unperturbed
+    if (noise != nullptr) zv = zv + noise[t * E + e];     // one fp32 addition decides the expert
+  }
+  int my_slot = -1;                // the slot in which this lane's expert was selected
+  int sel = 0;                     // lane j of a group keeps the expert of slot j
+  float zmax = 0.f;
+  for (int j = 0; j < k; ++j) {
+    int bi = have && my_slot < 0 ? e : -1;
+    float bv = zv;
+#pragma unroll
+    for (int o = G / 2; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(kAll, bv, o);
+      const int oi = __shfl_xor_sync(kAll, bi, o);
+      if (oi >= 0 && (bi < 0 || ov > bv || (ov == bv && oi < bi))) { bi = oi; bv = ov; }
+    }
+    if (j == 0) zmax = bv;
+    if (bi == e && have) my_slot = j;
+    if (j == e) sel = bi;
+  }
+  const float ex = have ? expf((zv - zmax) * scale) : 0.f;
+  float psum = 0.f;
+  for (int ee = 0; ee < E; ++ee) psum += __shfl_sync(kAll, ex, ee, G);
+  const float my_p = have ? ex / psum : 0.f;
+  float my_g = 0.f;
+  if (routing == BTX_ROUTE_SWITCH) {
+    if (my_slot == 0) {            // the lane that owns the arg-max: the gate is its full-softmax probability
+      my_g = ex / psum;
+      topk[t] = e;
+      gates[t] = my_g;
+    }
+  } else {
+    float gsum = 0.f;
+    for (int j = 0; j < k; ++j) {
+      const int sj = __shfl_sync(kAll, sel, j, G);
+      gsum += __shfl_sync(kAll, ex, sj < 0 ? 0 : sj, G);
+    }
+    if (my_slot >= 0) {            // the lane that owns a selected expert writes that slot
+      my_g = ex / gsum;
+      topk[t * k + my_slot] = e;
+      gates[t * k + my_slot] = my_g;
+    }
+  }
+  if (have) probs[t * E + e] = my_p;
+  // gates and probabilities of expert e over the tokens of this pass, gathered in the first group's lanes
+  float gs = my_g, ps = my_p;
+#pragma unroll
+  for (int o = 16; o >= G; o >>= 1) {
+    gs += __shfl_xor_sync(kAll, gs, o);
+    ps += __shfl_xor_sync(kAll, ps, o);
+  }
+  if (lane < E) { u_sum += gs; p_sum += ps; }
+  __syncwarp();
+}
+
 constexpr int kSmallThreads = 256;
 constexpr int kSmallMaxR = 1024;
 

@@ -97,6 +97,57 @@ __device__ __forceinline__ void route_logits4(int t0, int nt, int d, int E, cons
   }
 }
 
+// BF16: logits of up to sixteen tokens t0 .. t0+nt-1 by one warp on the tensor cores (mma.sync m16n8k16, fp32
+// accumulation): tokens are the rows, eight experts the columns.  Lane (g, tg) = (lane / 4, lane % 4) loads 16
+// bytes of rows g and g + 8 of x and of router row g at columns c0 + 8 tg, and feeds them to two MMAs as the
+// contraction slots its registers stand for; the order of the contraction index inside an MMA is free as long
+// as both operands use the same one, so nothing is shuffled or staged.  A warp instruction reads 64
+// contiguous bytes of each of 8 rows (whole sectors), x is streamed past L1, the 32 KB of router rows stay
+// in it.  About 70 instructions per token instead of 1800 with FMAs: the kernel becomes bound by the x stream.
+constexpr int kRouteMmaTokens = 16;
+__device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                 uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void route_logits16_mma(int t0, int nt, int d, int E, const __nv_bfloat16* __restrict__ x,
+                                                   const __nv_bfloat16* __restrict__ wr, const float* __restrict__ bias,
+                                                   float (*z)[kMaxExperts], int lane) {
+  const int g = lane >> 2, tg = lane & 3;
+  const __nv_bfloat16* x0 = x + (size_t)(t0 + min(g, nt - 1)) * d;        // absent tokens repeat the last one
+  const __nv_bfloat16* x1 = x + (size_t)(t0 + min(g + 8, nt - 1)) * d;
+  for (int eb = 0; eb < E; eb += 8) {
+    const __nv_bfloat16* w = wr + (size_t)min(eb + g, E - 1) * d;          // absent experts repeat the last one
+    float c[4] = {0.f, 0.f, 0.f, 0.f};
+    // the trip count is the same for all lanes (the MMAs need the whole warp); a lane whose 8 columns lie past
+    // the end of the rows (d is a multiple of 8, not necessarily of 32) contributes zeros
+#pragma unroll 8
+    for (int cb = 0; cb < d; cb += 32) {
+      const int c0 = cb + tg * 8;
+      uint4 lo = make_uint4(0, 0, 0, 0), hi = lo, b = lo;
+      if (c0 < d) {
+        lo = __ldcs(reinterpret_cast<const uint4*>(x0 + c0));
+        hi = __ldcs(reinterpret_cast<const uint4*>(x1 + c0));
+        b = __ldg(reinterpret_cast<const uint4*>(w + c0));
+      }
+      mma_bf16_16x8x16(c, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
+      mma_bf16_16x8x16(c, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
+    }
+    // c[0], c[1]: token g, experts eb + 2 tg, + 1; c[2], c[3]: token g + 8, the same experts
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int e = eb + 2 * tg + i;
+      if (e < E) {
+        const float bv = bias ? bias[e] : 0.f;
+        z[g][e] = c[i] + bv;
+        z[g + 8][e] = c[2 + i] + bv;
+      }
+    }
+  }
+}
+
 // Stores the (unperturbed) logits of token t, adds the Sample Top-1 noise, and routes: top-k by repeated
 // arg-max with ties to the lower index, gates, full softmax.  On return lane l holds the dense gate and the
 // probability of experts l and l + 32.
@@ -151,7 +202,7 @@ __device__ __forceinline__ void lb_finalize(int Tn, int E, int nblocks, float al
 // converts router rows per token.  Every block leaves its partial sums of the gates and probabilities; the
 // block that finishes last (a ticket in the workspace status block, zero when the kernel starts) forms the
 // batch means and the loss from all of them.
-template <typename T, bool WS>
+template <typename T, bool WS, bool MMA>
 __global__ void __launch_bounds__(kRouterThreads, 2)
 router_kernel(int Tn, int d, int E, int k, int routing, float alpha, const T* __restrict__ x, const T* __restrict__ wr,
               const float* __restrict__ bias, const float* __restrict__ given_logits,
@@ -160,7 +211,8 @@ router_kernel(int Tn, int d, int E, int k, int routing, float alpha, const T* __
               float* __restrict__ probs, float* route_part, float* __restrict__ u, float* __restrict__ p,
               float* __restrict__ loss, double* __restrict__ up64, int32_t* ticket) {
   extern __shared__ __align__(16) float ws[];             // WS: the router rows as fp32
-  __shared__ float zs[kRouterWarps][kRouteTokens][kMaxExperts];
+  constexpr int NTOK = MMA ? kRouteMmaTokens : kRouteTokens;             // tokens a warp routes at a time
+  __shared__ float zs[kRouterWarps][NTOK][kMaxExperts];
   __shared__ float red[kRouterWarps][kMaxExperts][2];
   __shared__ int is_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -175,15 +227,28 @@ router_kernel(int Tn, int d, int E, int k, int routing, float alpha, const T* __
     __syncthreads();
   }
   float u_acc[2] = {0.f, 0.f}, p_acc[2] = {0.f, 0.f};   // lane l accumulates experts l and l + 32 over this warp's tokens
-  for (int t = (blockIdx.x * kRouterWarps + warp) * kRouteTokens; t < Tn; t += gridDim.x * kRouterWarps * kRouteTokens) {
-    const int nt = min(kRouteTokens, Tn - t);
-    route_logits4<T, WS>(t, nt, d, E, x, wr, ws, bias, given_logits, zs[warp], lane);
+  for (int t = (blockIdx.x * kRouterWarps + warp) * NTOK; t < Tn; t += gridDim.x * kRouterWarps * NTOK) {
+    const int nt = min(NTOK, Tn - t);
+    if constexpr (MMA) route_logits16_mma(t, nt, d, E, x, wr, bias, zs[warp], lane);
+    else route_logits4<T, WS>(t, nt, d, E, x, wr, ws, bias, given_logits, zs[warp], lane);
     __syncwarp();
-    for (int i = 0; i < nt; ++i) {
-      float my_g[2], my_p[2];
-      route_finish_token(t + i, E, k, routing, noise, inv_tau, zs[warp][i], lane, logits, topk, gates, probs, my_g, my_p);
+    const float scale = noise != nullptr ? inv_tau : 1.0f;
+    if (E <= 4) {                  // few experts: several tokens are routed side by side, one lane per (token, expert)
+      for (int i0 = 0; i0 < nt; i0 += 8)
+        route_select_group<4>(t, i0, nt, E, k, routing, scale, noise, zs[warp], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
+    } else if (E <= 8) {
+      for (int i0 = 0; i0 < nt; i0 += 4)
+        route_select_group<8>(t, i0, nt, E, k, routing, scale, noise, zs[warp], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
+    } else if (E <= 16) {
+      for (int i0 = 0; i0 < nt; i0 += 2)
+        route_select_group<16>(t, i0, nt, E, k, routing, scale, noise, zs[warp], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
+    } else {
+      for (int i = 0; i < nt; ++i) {
+        float my_g[2], my_p[2];
+        route_finish_token(t + i, E, k, routing, noise, inv_tau, zs[warp][i], lane, logits, topk, gates, probs, my_g, my_p);
 #pragma unroll
-      for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
+        for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
+      }
     }
   }
 #pragma unroll
@@ -626,16 +691,18 @@ router_dw_reduce_kernel(int d, int E, int chunks, const float* __restrict__ part
 // ---------------------------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------------------------
-template <typename T, bool WS>
+template <typename T, bool WS, bool MMA>
 static cudaError_t launch_router_t(const Plan& pl, int routing, float alpha, const void* x, const void* w_router,
                                    const float* bias, const float* given_logits, const float* noise, float inv_tau,
                                    const Buffers& b, size_t smem, cudaStream_t st) {
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(router_kernel<T, WS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(router_kernel<T, WS, MMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   // the ticket of the last-block finalisation is word 8 of the status block, zeroed by the caller
-  router_kernel<T, WS><<<pl.route_blocks, kRouterThreads, smem, st>>>(
+  int blocks = pl.route_blocks;                           // (the plan's count bounds the partial-sum buffer)
+  if (MMA) blocks = min(blocks, (pl.T + kRouterWarps * kRouteMmaTokens - 1) / (kRouterWarps * kRouteMmaTokens));
+  router_kernel<T, WS, MMA><<<blocks, kRouterThreads, smem, st>>>(
       pl.T, pl.d, pl.E, pl.k, routing, alpha, (const T*)x, (const T*)w_router, bias, given_logits, noise, inv_tau,
       b.logits, b.topk, b.gates, b.probs, b.route_part, b.u, b.p, b.loss, b.up64, b.status + 8);
   return cudaGetLastError();
@@ -646,11 +713,10 @@ cudaError_t launch_router(const Plan& pl, int dtype, int routing, float alpha, c
                           const Buffers& b, cudaStream_t st) {
   const size_t smem = (size_t)pl.E * pl.d * sizeof(float);
   const bool in_smem = given_logits == nullptr && smem > 0 && smem <= 64 * 1024;
-  if (dtype == BTX_BF16)
-    return in_smem ? launch_router_t<__nv_bfloat16, true>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, smem, st)
-                   : launch_router_t<__nv_bfloat16, false>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, 0, st);
-  return in_smem ? launch_router_t<float, true>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, smem, st)
-                 : launch_router_t<float, false>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, 0, st);
+  if (dtype == BTX_BF16)          // BF16 activations: the logits come from the tensor cores
+    return launch_router_t<__nv_bfloat16, false, true>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, 0, st);
+  return in_smem ? launch_router_t<float, true, false>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, smem, st)
+                 : launch_router_t<float, false, false>(pl, routing, alpha, x, w_router, bias, given_logits, noise, inv_tau, b, 0, st);
 }
 
 bool route_permute_small_fits(const Plan& pl) { return pl.R <= kSmallMaxR; }
