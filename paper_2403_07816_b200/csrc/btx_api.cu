@@ -43,8 +43,8 @@ btx_status make_plan(const btx_moe_desc* desc, Plan* pl, bool routing_only) {
   p.r_pad_max = (int)align_up((size_t)p.R + (size_t)p.E * (kRowTile - 1), kRowTile);
   p.mt_max = p.r_pad_max / kRowTile;
   p.nt_dact = desc->dtype == BTX_BF16 ? 2 * ((p.F + 255) / 256) : (p.F + 63) / 64;   // row-dot partials per row
-  p.route_blocks = (p.T + 31) / 32;                       // a router block routes 32 tokens at a time; the blocks are
-  if (p.route_blocks > 2 * sm_count()) p.route_blocks = 2 * sm_count();   // persistent, two per multiprocessor
+  p.route_blocks = (p.T + 15) / 16;                       // a router block routes 16 (BF16) or 32 tokens at a time; the
+  if (p.route_blocks > 4 * sm_count()) p.route_blocks = 4 * sm_count();   // blocks are persistent, up to four per multiprocessor
   if (p.route_blocks > kMaxRouteBlocks) p.route_blocks = kMaxRouteBlocks;
   p.perm_blocks = (p.R + 1023) / 1024;
   p.wr_chunks = (p.T + 127) / 128;

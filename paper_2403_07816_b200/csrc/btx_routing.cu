@@ -103,7 +103,9 @@ __device__ __forceinline__ void route_logits4(int t0, int nt, int d, int E, cons
 // contraction slots its registers stand for; the order of the contraction index inside an MMA is free as long
 // as both operands use the same one, so nothing is shuffled or staged.  A warp instruction reads 64
 // contiguous bytes of each of 8 rows (whole sectors), x is streamed past L1, the 32 KB of router rows stay
-// in it.  About 70 instructions per token instead of 1800 with FMAs: the kernel becomes bound by the x stream.
+// in it.  A block takes sixteen tokens at a time and its eight warps an eighth of the columns each (short load
+// chains, a block per 16 tokens to spread over the multiprocessors); the partial sums meet in shared memory
+// and are added in warp order.  About 70 instructions per token instead of 1800 with FMAs.
 constexpr int kRouteMmaTokens = 16;
 __device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                  uint32_t b0, uint32_t b1) {
@@ -112,39 +114,30 @@ __device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], uint32_t a0, uin
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ void route_logits16_mma(int t0, int nt, int d, int E, const __nv_bfloat16* __restrict__ x,
-                                                   const __nv_bfloat16* __restrict__ wr, const float* __restrict__ bias,
-                                                   float (*z)[kMaxExperts], int lane) {
+// Partial logits over the column blocks c_begin, c_begin + c_step, ... (32 columns each) of tokens t0 ..
+// t0+nt-1 and experts eb .. eb+7.  c[0], c[1]: token g, experts eb + 2 tg, + 1; c[2], c[3]: token g + 8.
+__device__ __forceinline__ void route_mma_partial(int t0, int nt, int d, int E, int eb, int c_begin, int c_step,
+                                                  const __nv_bfloat16* __restrict__ x,
+                                                  const __nv_bfloat16* __restrict__ wr, int lane, float (&c)[4]) {
   const int g = lane >> 2, tg = lane & 3;
   const __nv_bfloat16* x0 = x + (size_t)(t0 + min(g, nt - 1)) * d;        // absent tokens repeat the last one
   const __nv_bfloat16* x1 = x + (size_t)(t0 + min(g + 8, nt - 1)) * d;
-  for (int eb = 0; eb < E; eb += 8) {
-    const __nv_bfloat16* w = wr + (size_t)min(eb + g, E - 1) * d;          // absent experts repeat the last one
-    float c[4] = {0.f, 0.f, 0.f, 0.f};
-    // the trip count is the same for all lanes (the MMAs need the whole warp); a lane whose 8 columns lie past
-    // the end of the rows (d is a multiple of 8, not necessarily of 32) contributes zeros
-#pragma unroll 8
-    for (int cb = 0; cb < d; cb += 32) {
-      const int c0 = cb + tg * 8;
-      uint4 lo = make_uint4(0, 0, 0, 0), hi = lo, b = lo;
-      if (c0 < d) {
-        lo = __ldcs(reinterpret_cast<const uint4*>(x0 + c0));
-        hi = __ldcs(reinterpret_cast<const uint4*>(x1 + c0));
-        b = __ldg(reinterpret_cast<const uint4*>(w + c0));
-      }
-      mma_bf16_16x8x16(c, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
-      mma_bf16_16x8x16(c, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
-    }
-    // c[0], c[1]: token g, experts eb + 2 tg, + 1; c[2], c[3]: token g + 8, the same experts
+  const __nv_bfloat16* w = wr + (size_t)min(eb + g, E - 1) * d;            // absent experts repeat the last one
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int e = eb + 2 * tg + i;
-      if (e < E) {
-        const float bv = bias ? bias[e] : 0.f;
-        z[g][e] = c[i] + bv;
-        z[g + 8][e] = c[2 + i] + bv;
-      }
+  for (int i = 0; i < 4; ++i) c[i] = 0.f;
+  // the trip count is the same for all lanes (the MMAs need the whole warp); a lane whose 8 columns lie past
+  // the end of the rows (d is a multiple of 8, not necessarily of 32) contributes zeros
+#pragma unroll 4
+  for (int cb = c_begin; cb < d; cb += c_step) {
+    const int c0 = cb + tg * 8;
+    uint4 lo = make_uint4(0, 0, 0, 0), hi = lo, b = lo;
+    if (c0 < d) {
+      lo = __ldcs(reinterpret_cast<const uint4*>(x0 + c0));
+      hi = __ldcs(reinterpret_cast<const uint4*>(x1 + c0));
+      b = __ldg(reinterpret_cast<const uint4*>(w + c0));
     }
+    mma_bf16_16x8x16(c, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
+    mma_bf16_16x8x16(c, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
   }
 }
 
@@ -203,7 +196,7 @@ __device__ __forceinline__ void lb_finalize(int Tn, int E, int nblocks, float al
 // block that finishes last (a ticket in the workspace status block, zero when the kernel starts) forms the
 // batch means and the loss from all of them.
 template <typename T, bool WS, bool MMA>
-__global__ void __launch_bounds__(kRouterThreads, 2)
+__global__ void __launch_bounds__(kRouterThreads, MMA ? 4 : 2)
 router_kernel(int Tn, int d, int E, int k, int routing, float alpha, const T* __restrict__ x, const T* __restrict__ wr,
               const float* __restrict__ bias, const float* __restrict__ given_logits,
               const float* __restrict__ noise, float inv_tau,
@@ -212,7 +205,8 @@ router_kernel(int Tn, int d, int E, int k, int routing, float alpha, const T* __
               float* __restrict__ loss, double* __restrict__ up64, int32_t* ticket) {
   extern __shared__ __align__(16) float ws[];             // WS: the router rows as fp32
   constexpr int NTOK = MMA ? kRouteMmaTokens : kRouteTokens;             // tokens a warp routes at a time
-  __shared__ float zs[kRouterWarps][NTOK][kMaxExperts];
+  __shared__ float zs[MMA ? 1 : kRouterWarps][NTOK][kMaxExperts];
+  __shared__ float part[MMA ? kRouterWarps : 1][kRouteMmaTokens][8];      // MMA: partial logits of the warps
   __shared__ float red[kRouterWarps][kMaxExperts][2];
   __shared__ int is_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -227,27 +221,69 @@ router_kernel(int Tn, int d, int E, int k, int routing, float alpha, const T* __
     __syncthreads();
   }
   float u_acc[2] = {0.f, 0.f}, p_acc[2] = {0.f, 0.f};   // lane l accumulates experts l and l + 32 over this warp's tokens
-  for (int t = (blockIdx.x * kRouterWarps + warp) * NTOK; t < Tn; t += gridDim.x * kRouterWarps * NTOK) {
-    const int nt = min(NTOK, Tn - t);
-    if constexpr (MMA) route_logits16_mma(t, nt, d, E, x, wr, bias, zs[warp], lane);
-    else route_logits4<T, WS>(t, nt, d, E, x, wr, ws, bias, given_logits, zs[warp], lane);
-    __syncwarp();
-    const float scale = noise != nullptr ? inv_tau : 1.0f;
-    if (E <= 4) {                  // few experts: several tokens are routed side by side, one lane per (token, expert)
-      for (int i0 = 0; i0 < nt; i0 += 8)
-        route_select_group<4>(t, i0, nt, E, k, routing, scale, noise, zs[warp], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
-    } else if (E <= 8) {
-      for (int i0 = 0; i0 < nt; i0 += 4)
-        route_select_group<8>(t, i0, nt, E, k, routing, scale, noise, zs[warp], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
-    } else if (E <= 16) {
-      for (int i0 = 0; i0 < nt; i0 += 2)
-        route_select_group<16>(t, i0, nt, E, k, routing, scale, noise, zs[warp], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
-    } else {
-      for (int i = 0; i < nt; ++i) {
-        float my_g[2], my_p[2];
-        route_finish_token(t + i, E, k, routing, noise, inv_tau, zs[warp][i], lane, logits, topk, gates, probs, my_g, my_p);
+  const float scale = noise != nullptr ? inv_tau : 1.0f;
+  if constexpr (MMA) {
+    // ---- BF16: a block per sixteen tokens, the columns split over its warps ----
+    for (int grp = blockIdx.x; grp * NTOK < Tn; grp += gridDim.x) {
+      const int t = grp * NTOK, nt = min(NTOK, Tn - t);
+      for (int eb = 0; eb < E; eb += 8) {
+        float c[4];
+        route_mma_partial(t, nt, d, E, eb, warp * 32, kRouterWarps * 32, x, wr, lane, c);
+        const int g = lane >> 2, tg = lane & 3;
+        part[warp][g][2 * tg] = c[0]; part[warp][g][2 * tg + 1] = c[1];
+        part[warp][g + 8][2 * tg] = c[2]; part[warp][g + 8][2 * tg + 1] = c[3];
+        __syncthreads();
+        if (threadIdx.x < NTOK * 8) {
+          const int tok = threadIdx.x >> 3, e = eb + (threadIdx.x & 7);
+          if (e < E) {
+            float a = 0.f;
+            for (int w = 0; w < kRouterWarps; ++w) a += part[w][tok][threadIdx.x & 7];
+            zs[0][tok][e] = a + (bias ? bias[e] : 0.f);
+          }
+        }
+        __syncthreads();
+      }
+      // few experts: several tokens are routed side by side, one lane per (token, expert); the passes go to
+      // different warps
+      if (E <= 4) {
+        if (warp * 8 < nt)
+          route_select_group<4>(t, warp * 8, nt, E, k, routing, scale, noise, zs[0], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
+      } else if (E <= 8) {
+        if (warp * 4 < nt)
+          route_select_group<8>(t, warp * 4, nt, E, k, routing, scale, noise, zs[0], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
+      } else if (E <= 16) {
+        if (warp * 2 < nt)
+          route_select_group<16>(t, warp * 2, nt, E, k, routing, scale, noise, zs[0], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
+      } else {
+        for (int i = warp; i < nt; i += kRouterWarps) {
+          float my_g[2], my_p[2];
+          route_finish_token(t + i, E, k, routing, noise, inv_tau, zs[0][i], lane, logits, topk, gates, probs, my_g, my_p);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
+          for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
+        }
+      }
+      __syncthreads();                                    // zs is written again for the next sixteen tokens
+    }
+  } else {
+    // ---- FP32 (or given logits): a warp per four tokens ----
+    for (int t = (blockIdx.x * kRouterWarps + warp) * NTOK; t < Tn; t += gridDim.x * kRouterWarps * NTOK) {
+      const int nt = min(NTOK, Tn - t);
+      route_logits4<T, WS>(t, nt, d, E, x, wr, ws, bias, given_logits, zs[warp], lane);
+      __syncwarp();
+      if (E <= 4) {
+        route_select_group<4>(t, 0, nt, E, k, routing, scale, noise, zs[warp], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
+      } else if (E <= 8) {
+        route_select_group<8>(t, 0, nt, E, k, routing, scale, noise, zs[warp], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
+      } else if (E <= 16) {
+        for (int i0 = 0; i0 < nt; i0 += 2)
+          route_select_group<16>(t, i0, nt, E, k, routing, scale, noise, zs[warp], lane, logits, topk, gates, probs, u_acc[0], p_acc[0]);
+      } else {
+        for (int i = 0; i < nt; ++i) {
+          float my_g[2], my_p[2];
+          route_finish_token(t + i, E, k, routing, noise, inv_tau, zs[warp][i], lane, logits, topk, gates, probs, my_g, my_p);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) { u_acc[h] += my_g[h]; p_acc[h] += my_p[h]; }
+        }
       }
     }
   }
@@ -701,7 +737,7 @@ static cudaError_t launch_router_t(const Plan& pl, int routing, float alpha, con
   }
   // the ticket of the last-block finalisation is word 8 of the status block, zeroed by the caller
   int blocks = pl.route_blocks;                           // (the plan's count bounds the partial-sum buffer)
-  if (MMA) blocks = min(blocks, (pl.T + kRouterWarps * kRouteMmaTokens - 1) / (kRouterWarps * kRouteMmaTokens));
+  if (!MMA) blocks = min(blocks, (pl.T + kRouterWarps * kRouteTokens - 1) / (kRouterWarps * kRouteTokens));
   router_kernel<T, WS, MMA><<<blocks, kRouterThreads, smem, st>>>(
       pl.T, pl.d, pl.E, pl.k, routing, alpha, (const T*)x, (const T*)w_router, bias, given_logits, noise, inv_tau,
       b.logits, b.topk, b.gates, b.probs, b.route_part, b.u, b.p, b.loss, b.up64, b.status + 8);
