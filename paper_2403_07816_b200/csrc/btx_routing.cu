@@ -480,30 +480,37 @@ route_permute_small_kernel(int Tn, int d, int E, int k, int routing, float alpha
 // ---------------------------------------------------------------------------------------------
 // Gather into the padded sorted layout, combine out of it
 // ---------------------------------------------------------------------------------------------
+// A warp per token: the row is read once (eight 16-byte loads in flight per lane) and written to the sorted row
+// of each of its k assignments (none for a dropped one); then a warp per padding row writes zeros.
 __global__ void __launch_bounds__(256)
-gather_rows_kernel(int k, int row_vecs, const uint4* __restrict__ src, uint4* __restrict__ dst,
-                   const int32_t* __restrict__ rowmap, const int32_t* __restrict__ pad_offsets, int E) {
+gather_rows_kernel(int Tn, int k, int row_vecs, const uint4* __restrict__ src, uint4* __restrict__ dst,
+                   const int32_t* __restrict__ rowmap, const int32_t* __restrict__ flat2row,
+                   const int32_t* __restrict__ pad_offsets, int E) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   allow_dependents();
   grid_dependency_wait();
-  const int total = pad_offsets[E];
-  for (int rp = blockIdx.x * 8 + warp; rp < total; rp += gridDim.x * 8) {
-    int flat = rowmap[rp];
-    uint4* o = dst + (size_t)rp * row_vecs;
-    if (flat < 0) {
-      for (int c = lane; c < row_vecs; c += 32) o[c] = make_uint4(0, 0, 0, 0);
-    } else {
-      const uint4* s = src + (size_t)(flat / k) * row_vecs;
-      for (int c0 = lane; c0 < row_vecs; c0 += 8 * 32) {   // eight loads in flight per lane, then eight stores
-        uint4 q[8];
+  for (int t = blockIdx.x * 8 + warp; t < Tn; t += gridDim.x * 8) {
+    const uint4* s = src + (size_t)t * row_vecs;
+    for (int c0 = lane; c0 < row_vecs; c0 += 8 * 32) {
+      uint4 q[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-          if (c0 + i * 32 < row_vecs) q[i] = s[c0 + i * 32];
+      for (int i = 0; i < 8; ++i)
+        if (c0 + i * 32 < row_vecs) q[i] = __ldcs(s + c0 + i * 32);
+      for (int sl = 0; sl < k; ++sl) {
+        const int rp = flat2row[(size_t)t * k + sl];
+        if (rp < 0) continue;
+        uint4* o = dst + (size_t)rp * row_vecs;
 #pragma unroll
         for (int i = 0; i < 8; ++i)
           if (c0 + i * 32 < row_vecs) o[c0 + i * 32] = q[i];
       }
     }
+  }
+  const int total = pad_offsets[E];
+  for (int rp = blockIdx.x * 8 + warp; rp < total; rp += gridDim.x * 8) {
+    if (rowmap[rp] >= 0) continue;
+    uint4* o = dst + (size_t)rp * row_vecs;
+    for (int c = lane; c < row_vecs; c += 32) o[c] = make_uint4(0, 0, 0, 0);
   }
 }
 
@@ -794,9 +801,9 @@ cudaError_t launch_gather_rows(const Plan& pl, const void* src, void* dst_sorted
   int row_vecs = pl.d * pl.esize / 16;
   int blocks = min(pl.r_pad_max / 8, sm_count() * 16);
   // the gather's launch overlaps the run of the kernel before it
-  return launch_after_predecessor(gather_rows_kernel, dim3(blocks), dim3(256), 0, st, true, pl.k, row_vecs,
+  return launch_after_predecessor(gather_rows_kernel, dim3(blocks), dim3(256), 0, st, true, pl.T, pl.k, row_vecs,
                                   (const uint4*)src, (uint4*)dst_sorted, (const int32_t*)b.rowmap,
-                                  (const int32_t*)b.pad_offsets, pl.E);
+                                  (const int32_t*)b.flat2row, (const int32_t*)b.pad_offsets, pl.E);
 }
 
 cudaError_t launch_combine(const Plan& pl, int dtype, const float* rows, int splits, void* y, const Buffers& b,
