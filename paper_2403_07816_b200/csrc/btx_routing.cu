@@ -1,10 +1,10 @@
 // Router, load-balancing loss, token permutation, row gather / combine and router backward.
 // These are the bandwidth- and latency-bound steps around the expert GEMMs.
 //
-//   router      logits = W_l x (Section 3.2), top-k by repeated arg-max with ties to the lower
-//               index, gate softmax over the selected logits, full softmax, partial sums for
-//               the batch means u and p of Section 3.3
-//   finalize    u, p, L_LB = alpha E sum_i u_i p_i
+//   router      logits = W_l x (Section 3.2; BF16: on the tensor cores), top-k by repeated arg-max with
+//               ties to the lower index, gate softmax over the selected logits, full softmax, partial
+//               sums for the batch means u and p of Section 3.3; the last block to finish forms
+//               u, p and L_LB = alpha E sum_i u_i p_i
 //   permutation histogram -> exclusive scan -> stable scatter of the R assignments into
 //               (expert ascending, token ascending) order; expert segments padded to whole 256-row tiles
 //   gather      rows of x (or dy) copied into the padded expert-sorted layout
