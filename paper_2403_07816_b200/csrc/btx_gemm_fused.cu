@@ -46,14 +46,15 @@ namespace cg = cooperative_groups;
 constexpr int XW = 128;                                  // weight rows per CTA and stage (256 per pair)
 constexpr int XN_MAX = 64;                               // tokens at most (MMA N)
 constexpr int XA_BYTES = XW * BK * 2;
-constexpr int X_STAGES = 8;
+constexpr int X_STAGES = 10;
 constexpr int X_RING_BYTES = X_STAGES * (XA_BYTES + (XN_MAX / 2) * BK * 2);
 constexpr int X_EPI_WARPS = 8;
 constexpr int X_EPI_THREADS = X_EPI_WARPS * 32;
 constexpr int X_THREADS = 64 + X_EPI_THREADS + 64;        // warps 10 and 11: two more TMA producers
-constexpr int X_CTL_BYTES = 256;
+constexpr int X_CTL_BYTES = 384;
 constexpr int X_XCHG_FLOATS = 2 * 32 * 64;               // [column half][column][row of the lower lanes]
 constexpr int X_SMEM_BYTES = X_RING_BYTES + 1024 + X_CTL_BYTES + X_XCHG_FLOATS * 4;
+static_assert(16 * X_STAGES + 112 <= X_CTL_BYTES, "barriers and control words fit the control block");
 static_assert(X_EPI_THREADS == kSmallThreads, "the epilogue warps run the routing code of a 256-thread block");
 
 struct FusedParams {
@@ -147,14 +148,14 @@ tc_small_forward_kernel(const __grid_constant__ XMaps tm, const FusedParams p) {
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t ring = (raw + 1023u) & ~1023u;
   uint8_t* ctl = smem_raw + (ring - raw) + X_RING_BYTES;
-  const uint32_t bar_full = smem_u32(ctl);                              // 8 x 8 B (used in the leader)
-  const uint32_t bar_empty = bar_full + X_STAGES * 8;                   // 8 x 8 B
+  const uint32_t bar_full = smem_u32(ctl);                              // X_STAGES x 8 B (used in the leader)
+  const uint32_t bar_empty = bar_full + X_STAGES * 8;                   // X_STAGES x 8 B
   const uint32_t bar_tfull = bar_empty + X_STAGES * 8;                  // 2 x 8 B
   const uint32_t bar_tempty = bar_tfull + 16;                           // 2 x 8 B (used in the leader)
   const uint32_t bar_xfull = bar_tempty + 16;                           // 4 x 8 B: h3 of a warp pair is in shared memory
   const uint32_t bar_xfree = bar_xfull + 32;                            // 4 x 8 B: ... and has been read
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + 224);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + 232);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + 16 * X_STAGES + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + 16 * X_STAGES + 104);
   float* xchg = reinterpret_cast<float*>(ctl + X_CTL_BYTES);
   const uint32_t stage_bytes = XA_BYTES + (uint32_t)(p.N / 2) * (BK * 2);
 
@@ -211,6 +212,7 @@ tc_small_forward_kernel(const __grid_constant__ XMaps tm, const FusedParams p) {
 
   // per-thread pipeline state of whichever role this thread has; it carries over from pass 1 to pass 2
   uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0, xphase = 0;
+  int w2_ahead = 0;                      // K blocks of W2 that the first loader put into the ring before pass 2 began
   bool ok = true;
 
   // code left in status word 1 by the first wait that runs out: which wait, in which pass, in which block
@@ -230,40 +232,61 @@ tc_small_forward_kernel(const __grid_constant__ XMaps tm, const FusedParams p) {
       // about 350): warp 0 arms the stage's barrier and loads W1 (pass 2: W2), warp 10 loads W3, warp 11 the
       // token tile; each waits for the stage to be free on its own.
       if (lane == 0 && !(prod == 1 && pass == 2)) {
-        while (ok && x_next_tile(walk, tl)) {
-          const int mine = rank == 0 ? min(tl.n, hu) : max(0, tl.n - hu);   // this CTA's units of the tile
-          const int row = (tl.u0 + (int)rank * hu) * XU;
-          const uint32_t tx = (uint32_t)tl.n * (XU * BK * 2) * (pass == 1 ? 2u : 1u) + 2u * (stage_bytes - XA_BYTES);
+        // K blocks [kb0, kb1) of tile t of pass ps
+        auto load_tile = [&](int ps, const XTile& t, int kb0, int kb1) {
+          const int thu = ps == 1 ? 4 : 8;
+          const int mine = rank == 0 ? min(t.n, thu) : max(0, t.n - thu);   // this CTA's units of the tile
+          const int row = (t.u0 + (int)rank * thu) * XU;
+          const uint32_t tx = (uint32_t)t.n * (XU * BK * 2) * (ps == 1 ? 2u : 1u) + 2u * (stage_bytes - XA_BYTES);
           // A thread with nothing to load for this tile (the second CTA's weight loaders when the tile fits into
           // the first CTA's share) only counts the stages: the MMAs do not depend on it, so it must not wait
           // on barriers that may complete more than one phase ahead of it.
           const bool idle = prod != 2 && mine == 0;
-          for (int kb = 0; kb < kb_total; ++kb) {
+          for (int kb = kb0; kb < kb1; ++kb) {
             if (idle) {
               if (++stage == X_STAGES) { stage = 0; phase ^= 1u; }
               continue;
             }
-            if (!(ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status, kWaitLimitNs, SITE(1)))) break;
+            if (!(ok = mbar_wait(bar_empty + stage * 8, phase ^ 1u, abort_flag, p.status, kWaitLimitNs,
+                                 1 | (ps << 4) | ((int)blockIdx.x << 8))))
+              break;
             const uint32_t full_local = bar_full + stage * 8;
             const uint32_t full = map_to_cta(full_local, 0);             // the leader collects both CTAs' bytes
             const uint32_t sA = ring + stage * stage_bytes, sB = sA + XA_BYTES;
             if (prod == 0) {
               if (rank == 0) mbar_expect_tx(full_local, tx);
-              if (pass == 1) {                            // this CTA: up to 64 rows of W1 ...
-                if (mine == hu) tma_load_3d(sA, &tm.w1[2], kb * BK, row, tl.e, full);
-                else x_load_units<2>(sA, tm.w1, mine, kb, row, tl.e, full);
+              if (ps == 1) {                              // this CTA: up to 64 rows of W1 ...
+                if (mine == thu) tma_load_3d(sA, &tm.w1[2], kb * BK, row, t.e, full);
+                else x_load_units<2>(sA, tm.w1, mine, kb, row, t.e, full);
               } else {
-                if (mine == hu) tma_load_3d(sA, &tm.w2[3], kb * BK, row, tl.e, full);
-                else x_load_units<3>(sA, tm.w2, mine, kb, row, tl.e, full);
+                if (mine == thu) tma_load_3d(sA, &tm.w2[3], kb * BK, row, t.e, full);
+                else x_load_units<3>(sA, tm.w2, mine, kb, row, t.e, full);
               }
             } else if (prod == 1) {                       // ... over the same rows of W3
-              if (mine == hu) tma_load_3d(sA + 64 * BK * 2, &tm.w3[2], kb * BK, row, tl.e, full);
-              else x_load_units<2>(sA + 64 * BK * 2, tm.w3, mine, kb, row, tl.e, full);
+              if (mine == thu) tma_load_3d(sA + 64 * BK * 2, &tm.w3[2], kb * BK, row, t.e, full);
+              else x_load_units<2>(sA + 64 * BK * 2, tm.w3, mine, kb, row, t.e, full);
             } else {                                      // this CTA's half of the N token rows
-              if (pass == 1) tma_load_2d(sB, &tm.x, kb * BK, (int)rank * (p.N / 2), full);
-              else tma_load_2d(sB, &tm.act, kb * BK, tl.e * p.N + (int)rank * (p.N / 2), full);
+              if (ps == 1) tma_load_2d(sB, &tm.x, kb * BK, (int)rank * (p.N / 2), full);
+              else tma_load_2d(sB, &tm.act, kb * BK, t.e * p.N + (int)rank * (p.N / 2), full);
             }
             if (++stage == X_STAGES) { stage = 0; phase ^= 1u; }
+          }
+        };
+        bool first = true;
+        while (ok && x_next_tile(walk, tl)) {
+          load_tile(pass, tl, (first && prod == 0) ? w2_ahead : 0, kb_total);
+          first = false;
+        }
+        w2_ahead = 0;
+        if (pass == 1 && prod == 0 && ok) {
+          // W2 does not depend on pass 1: the first K blocks of this pair's first pass-2 tile enter the ring as
+          // the last MMAs of pass 1 free its stages, ahead of the grid barrier; the stage barriers complete once
+          // the act tiles, loaded after the barrier, have arrived as well.
+          XWalk walk2 = x_walk(pair, n_pairs, p.E, (p.d + XU - 1) / XU, 16);
+          XTile t2;
+          if (x_next_tile(walk2, t2)) {
+            w2_ahead = min(X_STAGES, (p.F + BK - 1) / BK);
+            load_tile(2, t2, 0, w2_ahead);
           }
         }
         if (pass == 2 && prod == 0)
