@@ -16,7 +16,7 @@
 //            sits in accumulator lanes 0..63 and h3 in lanes 64..127, the epilogue warps of the upper
 //            lanes hand h3 to those of the lower lanes through shared memory, and the product is
 //            written as bf16: no partial sums
-//   -------- grid barrier --------
+//   -------- grid barrier (the first K blocks of W2, which depend on nothing, enter the ring before it) --------
 //   pass 2   rows[t*k+slot] = gate * W2_e act[e][t], written for the (token, expert) pairs the router
 //            selected (and, under a capacity limit, kept), found in the epilogue from topk.  Meanwhile the
 //            epilogue warps of block 0 form the batch means, the loss and the permutation
