@@ -51,6 +51,10 @@ E2E_STEPS = 50
 # kernel sources whose hash is recorded with it; with any other sources the bench reports traffic = null.
 TC_GEMM_TRAFFIC = {"bytes_per_step_T16384": 33.68e9, "sources_sha256_16": "4b5584b3b2e0e287"}
 TC_GEMM_SOURCES = ("btx_gemm_tc.cu", "btx_tc_ptx.cuh", "btx_common.cuh")
+# The same for one launch (one layer) of the one-kernel decode-shaped forward, from the capture summarised in
+# profiles/tc_small_forward_kernel_decode_T32_full.txt (1.0864 GB read + 0.0070 GB written).
+SMALL_FWD_TRAFFIC = {"bytes_per_layer_T32": 1.0934e9, "sources_sha256_16": "59f3acb607798dbb"}
+SMALL_FWD_SOURCES = ("btx_gemm_fused.cu", "btx_tc_ptx.cuh", "btx_route_dev.cuh", "btx_common.cuh")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -66,9 +70,9 @@ def load_peaks():
     return p
 
 
-def kernel_sources_hash():
+def kernel_sources_hash(names=TC_GEMM_SOURCES):
     h = hashlib.sha256()
-    for name in TC_GEMM_SOURCES:
+    for name in names:
         with open(os.path.join(ROOT, "paper_2403_07816_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:16]
@@ -492,9 +496,12 @@ def moe_result(run, ms, clocks, stages, soaked, K, W, world, peaks, with_counts)
     if run.workload == "decode":
         w_bytes = run.layers * 3 * N_EXPERTS * D_MODEL * D_FF * 2
         gbs = w_bytes / (ms * 1e-3) / 1e9
+        traffic = None                       # per launch = per layer, like `achieved`
+        if run.T == 32 and kernel_sources_hash(SMALL_FWD_SOURCES) == SMALL_FWD_TRAFFIC["sources_sha256_16"]:
+            traffic = SMALL_FWD_TRAFFIC["bytes_per_layer_T32"]
         res.update(metric="moe_ffn_decode_weight_stream_GBps", value=gbs * world, unit="GB/s",
                    roofline={"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                             "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0, "traffic": None,
+                             "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0, "traffic": traffic,
                              "peak_source": peaks["_source"],
                              "kernel": "tc_small_forward_kernel (one launch per layer) over the whole step"})
     else:
