@@ -47,3 +47,26 @@ def test_reference_arm_is_silent_on_other_ranks():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
                           "--warmup", "0"], capture_output=True, text=True, timeout=120, env=env, cwd=ROOT)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_clock_sampler_reads_clocks_power_and_reasons(tmp_path, monkeypatch):
+    """The bench's clock record comes from nvidia-smi's csv lines; a stand-in on PATH prints three samples."""
+    import stat
+    import time
+    fake = tmp_path / "nvidia-smi"
+    fake.write_text("#!/bin/sh\n"
+                    "echo '1200, 1965, 990.5, Not Active, Not Active, Not Active, Active'\n"
+                    "echo '1100, 1965, 1001.0, Not Active, Not Active, Not Active, Active'\n"
+                    "echo '1300, 1965, [N/A], Not Active, Not Active, Not Active, Not Active'\n"
+                    "sleep 30\n")
+    fake.chmod(fake.stat().st_mode | stat.S_IEXEC)
+    monkeypatch.setenv("PATH", str(tmp_path) + os.pathsep + os.environ["PATH"])
+    sys.path.insert(0, ROOT)
+    import bench
+    s = bench.ClockSampler(0)
+    s.start()
+    time.sleep(0.5)
+    rec = s.stop()
+    assert rec["samples"] == 3 and rec["sm_mhz"] == 1200 and rec["sm_max_mhz"] == 1965
+    assert rec["reasons"] == ["sw_power_cap"]
+    assert rec["power_w"] == (990.5 + 1001.0) / 2          # the unreadable sample is left out
